@@ -1,0 +1,201 @@
+/*
+ * dsn.h -- C ABI of the dynamic-weight-slicing inference library (NVIDIA B200, sm_100a).
+ *
+ * The library runs the batched inference path of DS-Net++ ("Dynamic Weight Slicing"):
+ * a per-sample gate picks one of T paths, samples are grouped by path, every group runs a
+ * dense contraction against the leading slice W[:k_out, :k_in] of the statically stored
+ * full weight, and results return in input order.
+ *
+ * Conventions
+ *   - Every function returns DSN_OK (0) or a negative dsn_status code.  No exceptions, no abort.
+ *   - "device" pointers are CUDA device memory of the context's GPU; "host" pointers are
+ *     ordinary host memory.  The caller owns every buffer; the library owns only dsn_ctx.
+ *     No entry point allocates memory per call unless its comment says so.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     Errors the host can detect are returned at once and nothing is launched.  Conditions only
+ *     the device can detect (routing index out of range, a bounded wait that ran out, non-finite
+ *     gate scores) are recorded in a device status word read by dsn_get_status().
+ *   - Weights are stored [out][in] (linear) or [out][KH][KW][in] (convolution, "OHWI"),
+ *     row-major, and are never modified, copied or repacked.  Activations are [B][R][C]
+ *     (tokens) or [B][H][W][C] (channels last); R = H*W.
+ *   - Paths are numbered 0..T-1 (the paper numbers them 1..|t|, smallest first).
+ */
+#ifndef DSN_H
+#define DSN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dsn_ctx dsn_ctx;
+
+enum dsn_status {
+  DSN_OK = 0,
+  DSN_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, k > C, T out of range ...   */
+  DSN_ERR_ALIGNMENT = -2,   /* a pointer or leading dimension breaks the stated alignment  */
+  DSN_ERR_WORKSPACE = -3,   /* workspace missing or smaller than dsn_*_workspace_bytes      */
+  DSN_ERR_UNSUPPORTED = -4, /* a combination this build has no kernel for                  */
+  DSN_ERR_BAD_INDEX = -5,   /* (device) a routing index outside [0, T)                     */
+  DSN_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed                         */
+  DSN_ERR_TIMEOUT = -7,     /* (device) a bounded wait inside a kernel ran out             */
+  DSN_ERR_NONFINITE = -8    /* (device) a gate score was NaN or infinite                   */
+};
+
+enum dsn_dtype { DSN_F32 = 0, DSN_BF16 = 1 };
+enum dsn_act { DSN_ACT_NONE = 0, DSN_ACT_RELU = 1, DSN_ACT_GELU = 2 /* exact erf form */ };
+enum dsn_order { DSN_INPUT_ORDER = 0, DSN_GROUPED = 1 };
+enum dsn_tail { DSN_TAIL_UNTOUCHED = 0, DSN_TAIL_ZERO = 1 };
+enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1 };
+
+#define DSN_MAX_SLICES 64   /* largest T                                               */
+#define DSN_MAX_GROUPS 4096 /* largest G of a caller-built group list                  */
+#define DSN_MAX_CHAIN 4     /* layers per dsn_layer_forward call                       */
+
+/* Batch grouping (not in the paper, which defines only per-sample behaviour, Eq. (dyn_net):
+ * every input runs the path its own gate picks).  Grouped position p holds sample perm[p];
+ * group g occupies positions offsets[g] .. offsets[g+1]-1 and uses slice group_slice[g]
+ * (slice g when group_slice is NULL).  dsn_route() fills it with G = T; a caller may instead
+ * build any list of G <= DSN_MAX_GROUPS groups, several of which may share a slice.
+ * All five arrays are device memory. */
+typedef struct dsn_routing {
+  int32_t B;                  /* samples                                                 */
+  int32_t G;                  /* groups                                                  */
+  int32_t* counts;            /* [G]                                                     */
+  int32_t* offsets;           /* [G+1], exclusive prefix sum of counts                   */
+  int32_t* perm;              /* [B]                                                     */
+  int32_t* inv_perm;          /* [B], inv_perm[perm[p]] = p                              */
+  const int32_t* group_slice; /* [G] or NULL                                             */
+} dsn_routing;
+
+/* Gate routing head (Sec. 3.5): X_E = mean over the R positions; scores = W2 ReLU(W1 X_E);
+ * index = first position of the maximum score. */
+typedef struct dsn_gate_desc {
+  int32_t dtype;   /* dtype of x: DSN_BF16 or DSN_F32                                    */
+  int32_t B, R;    /* samples, positions per sample                                      */
+  int32_t C_full;  /* columns of W1                                                      */
+  int32_t c_valid; /* leading channels of x that are read (elastic input), <= C_full     */
+  int32_t C_mlp;   /* hidden width                                                       */
+  int32_t T;       /* number of paths, 1..DSN_MAX_SLICES                                 */
+  int64_t ldx;     /* elements between consecutive positions of x, >= c_valid            */
+  const float* W1; /* device [C_mlp][C_full] fp32                                        */
+  const float* b1; /* device [C_mlp] or NULL                                             */
+  const float* W2; /* device [T][C_mlp] fp32                                             */
+  const float* b2; /* device [T] or NULL                                                 */
+} dsn_gate_desc;
+
+/* Sliced linear layer (Eq. (weight_slicing); ViT forms in Sec. 3.4):
+ * y[i][r][o] = act(bias[o] + sum_{c < k_in[t]} x[i][r][c] * W[o][c]),  o < k_out[t],  t = path of i. */
+typedef struct dsn_linear_desc {
+  int32_t dtype;        /* DSN_BF16 (x, W, y bf16; fp32 accumulate) or DSN_F32 (all fp32, plain FMA) */
+  int32_t R;            /* rows per sample                                               */
+  int32_t C_in, C_out;  /* full extents                                                  */
+  int64_t ldx, ldw, ldy;/* elements between rows of x, W, y.  bf16: multiples of 8       */
+  int32_t T;
+  const int32_t* k_in;  /* host [T], 1..C_in                                             */
+  const int32_t* k_out; /* host [T], 1..C_out                                            */
+  const void* W;        /* device [C_out][ldw]; bf16: 16-byte aligned                    */
+  const float* bias;    /* device [C_out] fp32 or NULL                                   */
+  int32_t act;          /* dsn_act                                                       */
+  int32_t in_order;     /* dsn_order of x: INPUT_ORDER [B][R][ldx] by sample, or GROUPED by position */
+  int32_t out_order;    /* dsn_order of y                                                */
+  int32_t tail;         /* dsn_tail: columns >= k_out[t] left untouched, or zero-filled up to C_out */
+} dsn_linear_desc;
+
+/* Slice-able convolution, filter-number / input-channel slicing (Sec. 3.3):
+ * y = W[:k_out, :k_in] * x, cross-correlation, zero padding, stride 1, K = 2*pad+1 in {1, 3}. */
+typedef struct dsn_conv_desc {
+  int32_t dtype;        /* DSN_BF16 only                                                 */
+  int32_t H, W_;        /* spatial size (output = input size)                            */
+  int32_t K, pad;       /* kernel size 1 (pad 0) or 3 (pad 1)                            */
+  int32_t C_in, C_out;
+  int64_t ldx, ldy;     /* elements between pixels of x, y; multiples of 8               */
+  int32_t T;
+  const int32_t* k_in;  /* host [T]                                                      */
+  const int32_t* k_out; /* host [T]                                                      */
+  const void* W;        /* device [C_out][K][K][C_in] bf16, dense, 16-byte aligned, C_in % 8 == 0 */
+  const float* bias;
+  int32_t act;
+  int32_t in_order, out_order, tail;
+} dsn_conv_desc;
+
+/* One dynamic block: optional gate, routing, then up to DSN_MAX_CHAIN layers that all inherit
+ * the block's routing (Sec. 5, "inherit the control signal").  Layer j reads layer j-1's output;
+ * layer 0 reads x in input order, the last layer writes y in input order; intermediate
+ * activations live in the workspace in grouped order. */
+typedef struct dsn_layer_desc {
+  const dsn_gate_desc* gate;        /* NULL: gate bypassed, idx_in supplies the path of every sample */
+  int32_t B;
+  int32_t T;
+  int32_t n_layers;                 /* 1..DSN_MAX_CHAIN                                  */
+  int32_t kind[DSN_MAX_CHAIN];      /* dsn_layer_kind                                    */
+  const void* layer[DSN_MAX_CHAIN]; /* dsn_linear_desc* or dsn_conv_desc* (order fields are ignored) */
+} dsn_layer_desc;
+
+/* ---- context ------------------------------------------------------------------------- */
+/* Creates a context on CUDA device `device` (allocates a few hundred bytes of device memory
+ * for the status word; the only allocation the library ever makes). */
+int dsn_create(dsn_ctx** ctx, int device);
+int dsn_destroy(dsn_ctx* ctx);
+const char* dsn_strerror(int code);
+/* Waits for `stream`, returns the first device-detected condition since the last call
+ * (code = DSN_OK if none; detail = a count or position) and clears it. */
+int dsn_get_status(dsn_ctx* ctx, void* stream, int32_t* code, int32_t* detail);
+
+/* Ratio list -> channel counts (host only).  granule g = 0 picks g = min(8, C/32);
+ * k = g*floor(r*C/g + 1/2) clamped to [g, C].  The paper lists channel counts, not a rounding
+ * rule; this rule reproduces its DS-MBNet list 224..640 step 32 from ratios 0.35..1.0. */
+int dsn_widths_from_ratios(int32_t C, const double* ratios, int32_t T, int32_t granule,
+                           int32_t* widths_out /* host [T] */);
+
+/* Multiply-adds the sliced layer executes for a routing histogram (Sec. 4.3, MAdds on the fly):
+ * sum_t counts[t] * R * k_in[t] * k_out[t] * K*K.  Host arrays. */
+int64_t dsn_executed_macs(const int32_t* counts, int32_t T, int32_t R, const int32_t* k_in,
+                          const int32_t* k_out, int32_t K);
+
+/* ---- gate (Sec. 3.5) ------------------------------------------------------------------ */
+size_t dsn_gate_workspace_bytes(const dsn_gate_desc* g);
+/* x: device [B][R][ldx].  idx_out: device [B].  logits_out: device [B][T] fp32 or NULL.
+ * workspace: device, 16-byte aligned, >= dsn_gate_workspace_bytes (partial sums of the pooling). */
+int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out,
+             float* logits_out, void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- routing (stable grouping by path index; one-hot routing of Sec. 3.1) -------------- */
+/* idx: device [B], values in [0, T).  Fills out->counts/offsets/perm/inv_perm (device arrays the
+ * caller allocated, G = T, B as given); integer-exact and deterministic.  A value outside
+ * [0, T) sets DSN_ERR_BAD_INDEX in the status word; that sample joins no group and the unused
+ * tail of perm is set to -1. */
+int dsn_route(dsn_ctx* ctx, const int32_t* idx, int32_t B, int32_t T, dsn_routing* out, void* stream);
+
+/* ---- gather / scatter between input order and grouped order ---------------------------- */
+/* Copies, for every sample, R rows of the leading k[t] columns (t = its path; k host [T]).
+ * to_grouped = 1: dst position p <- src sample perm[p]; 0: dst sample perm[p] <- src position p. */
+int dsn_permute_rows(dsn_ctx* ctx, const dsn_routing* r, int32_t dtype, int32_t R, int32_t T,
+                     const int32_t* k /* host [T] */, const void* src, int64_t ld_src, void* dst,
+                     int64_t ld_dst, int32_t to_grouped, void* stream);
+
+/* ---- sliced layers --------------------------------------------------------------------- */
+size_t dsn_linear_workspace_bytes(const dsn_linear_desc* d, int32_t B);
+size_t dsn_conv_workspace_bytes(const dsn_conv_desc* d, int32_t B);
+/* x, y: device, 16-byte aligned, laid out as d->in_order / d->out_order say.  r: routing of the
+ * batch (r->B samples).  workspace may be NULL when the size query returns 0. */
+int dsn_sliced_linear(dsn_ctx* ctx, const dsn_linear_desc* d, const dsn_routing* r, const void* x,
+                      void* y, void* workspace, size_t ws_bytes, void* stream);
+int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, const void* x,
+                    void* y, void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- whole dynamic block (Eq. (dyn_net)) ------------------------------------------------ */
+size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L);
+/* x, y in input order.  idx_in: device [B], required when L->gate is NULL, ignored otherwise.
+ * r_out (optional): receives pointers into the workspace holding the block's routing arrays
+ * (valid until the workspace is reused).  idx_out (optional): device [B], the gate's choice. */
+int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, const int32_t* idx_in,
+                      void* y, dsn_routing* r_out, int32_t* idx_out, void* workspace, size_t ws_bytes,
+                      void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSN_H */

@@ -1,0 +1,583 @@
+// C ABI of libdsn: context, argument validation, tensor-map construction, kernel selection and
+// the chained dsn_layer_forward.  Every compute step runs in this library's own CUDA kernels;
+// there is no host or library fallback.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "dsn_internal.cuh"
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+// bf16 tensor map of rank `rank` (3 or 4); dims/strides innermost first, strides[0] implied.
+int encode_map(const dsn_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+               const uint64_t* strides_bytes /* rank-1 */, const uint32_t* box) {
+  cuuint64_t gd[4], gs[3];
+  cuuint32_t bx[4], es[4];
+  for (int i = 0; i < rank; ++i) {
+    gd[i] = dims[i];
+    bx[i] = box[i];
+    es[i] = 1;
+    if (box[i] == 0 || box[i] > 256 || dims[i] == 0) return DSN_ERR_INVALID_ARG;
+  }
+  for (int i = 0; i + 1 < rank; ++i) {
+    gs[i] = strides_bytes[i];
+    if (gs[i] % 16 != 0 || gs[i] == 0) return DSN_ERR_ALIGNMENT;
+  }
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? DSN_OK : DSN_ERR_CUDA;
+}
+
+// One sliced layer in the form the kernels take.
+struct LayerCall {
+  int dtype;
+  int H, W, K, pad;      // linear: H = 1, W = R, K = 1
+  int C_in, C_out;
+  int64_t ldx, ldy;      // elements between rows (pixels)
+  int64_t w_row, w_tap;  // elements between output rows / taps of the weight
+  int T;
+  const int32_t *k_in, *k_out;
+  const void* Wt;
+  const float* bias;
+  int act, in_order, out_order, tail;
+};
+
+int check_slices(int T, const int32_t* k_in, const int32_t* k_out, int C_in, int C_out) {
+  if (T < 1 || T > DSN_MAX_SLICES || !k_in || !k_out) return DSN_ERR_INVALID_ARG;
+  for (int t = 0; t < T; ++t)
+    if (k_in[t] < 1 || k_in[t] > C_in || k_out[t] < 1 || k_out[t] > C_out) return DSN_ERR_INVALID_ARG;
+  return DSN_OK;
+}
+
+int check_routing(const dsn_routing* r, int T) {
+  if (!r || r->B < 0 || r->G < 1 || r->G > DSN_MAX_GROUPS) return DSN_ERR_INVALID_ARG;
+  if (!r->offsets || !r->perm) return DSN_ERR_INVALID_ARG;
+  if (!r->group_slice && r->G > T) return DSN_ERR_INVALID_ARG;
+  return DSN_OK;
+}
+
+int validate_call(const LayerCall& c, const dsn_routing* r, const void* x, const void* y) {
+  if (!x || !y || !c.Wt) return DSN_ERR_INVALID_ARG;
+  if (c.dtype != DSN_BF16 && c.dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
+  if (c.H < 1 || c.W < 1 || c.C_in < 1 || c.C_out < 1 || c.C_in > 32767 || c.C_out > 32767) return DSN_ERR_INVALID_ARG;
+  if (c.act < DSN_ACT_NONE || c.act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
+  if ((c.in_order != DSN_INPUT_ORDER && c.in_order != DSN_GROUPED) ||
+      (c.out_order != DSN_INPUT_ORDER && c.out_order != DSN_GROUPED) ||
+      (c.tail != DSN_TAIL_UNTOUCHED && c.tail != DSN_TAIL_ZERO))
+    return DSN_ERR_INVALID_ARG;
+  if (c.ldx < c.C_in || c.ldy < c.C_out || c.w_row < (int64_t)c.C_in * c.K * c.K) return DSN_ERR_INVALID_ARG;
+  int e = check_slices(c.T, c.k_in, c.k_out, c.C_in, c.C_out);
+  if (e) return e;
+  e = check_routing(r, c.T);
+  if (e) return e;
+  if ((int64_t)r->B * c.H * c.W > 0x7fffffffLL) return DSN_ERR_INVALID_ARG;
+  if (c.dtype == DSN_BF16) {
+    if (!aligned16(x) || !aligned16(y) || !aligned16(c.Wt)) return DSN_ERR_ALIGNMENT;
+    if (c.ldx % 8 || c.ldy % 8 || c.w_row % 8 || c.w_tap % 8) return DSN_ERR_ALIGNMENT;
+    if (!(c.K == 1 && c.pad == 0) && !(c.K == 3 && c.pad == 1)) return DSN_ERR_UNSUPPORTED;
+  } else {
+    if (c.K != 1) return DSN_ERR_UNSUPPORTED;
+  }
+  return DSN_OK;
+}
+
+void fill_slice_table(SliceTable& st, const LayerCall& c) {
+  memset(&st, 0, sizeof(st));
+  for (int t = 0; t < c.T; ++t) {
+    st.k_in[t] = c.k_in[t];
+    st.k_out[t] = c.k_out[t];
+  }
+}
+
+// Tile geometry for the bf16 kernel.
+void choose_geometry(const LayerCall& c, GemmGeom& g) {
+  memset(&g, 0, sizeof(g));
+  g.H = c.H;
+  g.W = c.W;
+  g.R = c.H * c.W;
+  g.taps = c.K * c.K;
+  g.KW = c.K;
+  g.pad = c.pad;
+  g.a_input_order = c.in_order == DSN_INPUT_ORDER;
+  g.y_input_order = c.out_order == DSN_INPUT_ORDER;
+  int max_ko = 1;
+  for (int t = 0; t < c.T; ++t) max_ko = c.k_out[t] > max_ko ? c.k_out[t] : max_ko;
+  g.BN = max_ko > 128 ? 256 : (max_ko > 64 ? 128 : 64);
+  g.stages = g.BN == 256 ? 4 : (g.BN == 128 ? 6 : 8);
+  if (c.K == 1 && !g.a_input_order) {
+    g.flat = 1;  // grouped rows are contiguous: tile them without regard to sample boundaries
+    g.bw = DSN_GEMM_BM;
+    g.bh = g.nb = g.tiles_x = g.tiles_y = 1;
+    return;
+  }
+  if (c.K == 1) {  // input order: a sample's R rows form one "image" of height 1
+    g.H = 1;
+    g.W = g.R;
+  }
+  g.bw = g.W < DSN_GEMM_BM ? g.W : DSN_GEMM_BM;
+  g.bh = DSN_GEMM_BM / g.bw;
+  if (g.bh > g.H) g.bh = g.H;
+  if (g.bh > 1) {  // balance the row bands of an image
+    const int bands = (g.H + g.bh - 1) / g.bh;
+    g.bh = (g.H + bands - 1) / bands;
+  }
+  g.nb = 1;
+  if (!g.a_input_order && g.bh == g.H && g.bw == g.W) {
+    g.nb = DSN_GEMM_BM / (g.bw * g.bh);
+    if (g.nb < 1) g.nb = 1;
+  }
+  g.tiles_x = (g.W + g.bw - 1) / g.bw;
+  g.tiles_y = (g.H + g.bh - 1) / g.bh;
+}
+
+int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  choose_geometry(c, p.g);
+  const GemmGeom& g = p.g;
+  p.B = r->B;
+  p.G = r->G;
+  p.T = c.T;
+  p.offsets = r->offsets;
+  p.perm = r->perm;
+  p.group_slice = r->group_slice;
+  p.y = static_cast<__nv_bfloat16*>(y);
+  p.ldy = c.ldy;
+  p.bias = c.bias;
+  p.act = c.act;
+  p.status = ctx->d_status;
+  for (int t = 0; t < c.T; ++t) {
+    p.k_in[t] = (int16_t)c.k_in[t];
+    p.k_out[t] = (int16_t)c.k_out[t];
+  }
+  const size_t smem = dsn_gemm_smem_bytes(g.BN, g.stages);
+
+  // distinct k_in values, DSN_GEMM_MAX_MAPS per launch
+  int done[DSN_MAX_SLICES];
+  memset(done, 0, sizeof(done));
+  int remaining = c.T;
+  while (remaining > 0) {
+    int nmaps = 0;
+    int map_k[DSN_GEMM_MAX_MAPS];
+    memset(p.map_id, 0xFF, sizeof(p.map_id));
+    for (int t = 0; t < c.T; ++t) {
+      if (done[t]) continue;
+      int id = -1;
+      for (int m = 0; m < nmaps; ++m)
+        if (map_k[m] == c.k_in[t]) id = m;
+      if (id < 0) {
+        if (nmaps == DSN_GEMM_MAX_MAPS) continue;  // next launch
+        id = nmaps++;
+        map_k[id] = c.k_in[t];
+      }
+      p.map_id[t] = (uint8_t)id;
+      done[t] = 1;
+      --remaining;
+    }
+    for (int m = 0; m < nmaps; ++m) {
+      const uint64_t kv = (uint64_t)map_k[m];
+      int e;
+      if (g.flat) {
+        const uint64_t rows = (uint64_t)r->B * g.R;
+        const uint64_t dims[4] = {kv, rows, 1, 1};
+        const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * rows, (uint64_t)c.ldx * 2 * rows};
+        const uint32_t box[4] = {DSN_GEMM_BK, DSN_GEMM_BM, 1, 1};
+        e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
+      } else {
+        const uint64_t dims[4] = {kv, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)r->B};
+        const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * g.W, (uint64_t)c.ldx * 2 * g.W * g.H};
+        const uint32_t box[4] = {DSN_GEMM_BK, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.nb};
+        e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
+      }
+      if (e) return e;
+      const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)c.C_out};
+      const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
+      const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)g.BN};
+      e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
+      if (e) return e;
+    }
+    if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
+  }
+  return DSN_OK;
+}
+
+int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
+  if (!ctx) return DSN_ERR_INVALID_ARG;
+  int e = validate_call(c, r, x, y);
+  if (e) return e;
+  if (r->B == 0) return DSN_OK;
+  SliceTable st;
+  fill_slice_table(st, c);
+  if (c.dtype == DSN_BF16) {
+    e = run_bf16(ctx, c, r, x, y, s);
+    if (e) return e;
+  } else {
+    if (dsn_launch_linear_f32(st, c.T, c.H * c.W, static_cast<const float*>(x), c.ldx,
+                              static_cast<const float*>(c.Wt), c.w_row, static_cast<float*>(y), c.ldy, c.bias, c.act,
+                              c.in_order == DSN_INPUT_ORDER, c.out_order == DSN_INPUT_ORDER, r->B, r->G, r->offsets,
+                              r->perm, r->group_slice, ctx->sm_count, s) != cudaSuccess)
+      return DSN_ERR_CUDA;
+  }
+  if (c.tail == DSN_TAIL_ZERO) {
+    if (dsn_launch_zero_tail(st, c.dtype == DSN_BF16 ? 2 : 4, c.H * c.W, c.C_out, y, c.ldy,
+                             c.out_order == DSN_INPUT_ORDER, r->B, r->G, r->offsets, r->perm, r->group_slice,
+                             s) != cudaSuccess)
+      return DSN_ERR_CUDA;
+  }
+  return DSN_OK;
+}
+
+LayerCall from_linear(const dsn_linear_desc* d) {
+  LayerCall c;
+  c.dtype = d->dtype;
+  c.H = 1; c.W = d->R; c.K = 1; c.pad = 0;
+  c.C_in = d->C_in; c.C_out = d->C_out;
+  c.ldx = d->ldx; c.ldy = d->ldy;
+  c.w_row = d->ldw; c.w_tap = d->ldw;
+  c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
+  c.Wt = d->W; c.bias = d->bias;
+  c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
+  return c;
+}
+
+LayerCall from_conv(const dsn_conv_desc* d) {
+  LayerCall c;
+  c.dtype = d->dtype;
+  c.H = d->H; c.W = d->W_; c.K = d->K; c.pad = d->pad;
+  c.C_in = d->C_in; c.C_out = d->C_out;
+  c.ldx = d->ldx; c.ldy = d->ldy;
+  c.w_row = (int64_t)d->K * d->K * d->C_in; c.w_tap = d->C_in;
+  c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
+  c.Wt = d->W; c.bias = d->bias;
+  c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
+  return c;
+}
+
+int check_gate(const dsn_gate_desc* g) {
+  if (!g || !g->W1 || !g->W2) return DSN_ERR_INVALID_ARG;
+  if (g->dtype != DSN_BF16 && g->dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
+  if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
+      g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
+    return DSN_ERR_INVALID_ARG;
+  if ((size_t)4 * 4 * ((size_t)g->c_valid + g->C_mlp + g->T) > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  return DSN_OK;
+}
+
+// workspace carving for dsn_layer_forward
+struct LayerPlan {
+  size_t off_idx, off_counts, off_offsets, off_perm, off_inv, off_gate, off_buf[2], off_gather, total;
+  size_t elem;
+  bool gather_first;
+};
+
+int layer_call_of(const dsn_layer_desc* L, int j, LayerCall& c) {
+  if (!L->layer[j]) return DSN_ERR_INVALID_ARG;
+  if (L->kind[j] == DSN_LAYER_LINEAR) c = from_linear(static_cast<const dsn_linear_desc*>(L->layer[j]));
+  else if (L->kind[j] == DSN_LAYER_CONV) c = from_conv(static_cast<const dsn_conv_desc*>(L->layer[j]));
+  else return DSN_ERR_INVALID_ARG;
+  return DSN_OK;
+}
+
+int plan_layer(const dsn_layer_desc* L, LayerPlan& pl) {
+  if (!L || L->B < 0 || L->T < 1 || L->T > DSN_MAX_SLICES || L->n_layers < 1 || L->n_layers > DSN_MAX_CHAIN)
+    return DSN_ERR_INVALID_ARG;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t B = (size_t)L->B;
+  pl.off_idx = take(4 * B);
+  pl.off_counts = take(4 * (size_t)L->T);
+  pl.off_offsets = take(4 * ((size_t)L->T + 1));
+  pl.off_perm = take(4 * B);
+  pl.off_inv = take(4 * B);
+  pl.off_gate = take(L->gate ? dsn_gate_workspace_bytes(L->gate) : 0);
+  size_t need[2] = {0, 0};
+  LayerCall first;
+  int e = layer_call_of(L, 0, first);
+  if (e) return e;
+  pl.elem = first.dtype == DSN_BF16 ? 2 : 4;
+  int prev_out = 0, prev_R = 0;
+  for (int j = 0; j < L->n_layers; ++j) {
+    LayerCall c;
+    e = layer_call_of(L, j, c);
+    if (e) return e;
+    if (c.T != L->T || c.dtype != first.dtype) return DSN_ERR_INVALID_ARG;
+    if (j > 0 && (c.C_in != prev_out || c.H * c.W != prev_R)) return DSN_ERR_INVALID_ARG;
+    prev_out = c.C_out;
+    prev_R = c.H * c.W;
+    if (j + 1 < L->n_layers) {
+      const size_t bytes = B * (size_t)prev_R * (size_t)c.C_out * pl.elem;
+      if (bytes > need[j & 1]) need[j & 1] = bytes;
+    }
+  }
+  pl.off_buf[0] = take(need[0]);
+  pl.off_buf[1] = take(need[1]);
+  // a physical gather pays when a sample has too few rows to fill a 128-row tile on its own
+  pl.gather_first = first.dtype == DSN_BF16 && first.H * first.W <= 64;
+  pl.off_gather = take(pl.gather_first ? B * (size_t)(first.H * first.W) * (size_t)first.C_in * pl.elem : 0);
+  pl.total = off;
+  return DSN_OK;
+}
+
+}  // namespace
+
+// ================================================================================== C ABI
+extern "C" {
+
+const char* dsn_strerror(int code) {
+  switch (code) {
+    case DSN_OK: return "ok";
+    case DSN_ERR_INVALID_ARG: return "invalid argument";
+    case DSN_ERR_ALIGNMENT: return "pointer or leading dimension not aligned as required";
+    case DSN_ERR_WORKSPACE: return "workspace missing or too small";
+    case DSN_ERR_UNSUPPORTED: return "unsupported combination";
+    case DSN_ERR_BAD_INDEX: return "routing index out of range";
+    case DSN_ERR_CUDA: return "CUDA call failed";
+    case DSN_ERR_TIMEOUT: return "bounded device wait ran out";
+    case DSN_ERR_NONFINITE: return "non-finite gate score";
+    default: return "unknown dsn status";
+  }
+}
+
+int dsn_create(dsn_ctx** out, int device) {
+  if (!out) return DSN_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return DSN_ERR_CUDA;
+  if (cudaSetDevice(device) != cudaSuccess) return DSN_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return DSN_ERR_CUDA;
+  if (prop.major != 10) return DSN_ERR_UNSUPPORTED;  // the kernels are sm_100a only
+  dsn_ctx* c = static_cast<dsn_ctx*>(calloc(1, sizeof(dsn_ctx)));
+  if (!c) return DSN_ERR_INVALID_ARG;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || !c->encode_tiled) {
+    free(c);
+    return DSN_ERR_CUDA;
+  }
+  if (cudaMalloc(&c->d_status, sizeof(int32_t) * DSN_STATUS_WORDS) != cudaSuccess ||
+      cudaMemset(c->d_status, 0, sizeof(int32_t) * DSN_STATUS_WORDS) != cudaSuccess) {
+    free(c);
+    return DSN_ERR_CUDA;
+  }
+  *out = c;
+  return DSN_OK;
+}
+
+int dsn_destroy(dsn_ctx* ctx) {
+  if (!ctx) return DSN_ERR_INVALID_ARG;
+  cudaFree(ctx->d_status);
+  free(ctx);
+  return DSN_OK;
+}
+
+int dsn_get_status(dsn_ctx* ctx, void* stream, int32_t* code, int32_t* detail) {
+  if (!ctx) return DSN_ERR_INVALID_ARG;
+  int32_t h[DSN_STATUS_WORDS];
+  cudaStream_t s = as_stream(stream);
+  if (cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DSN_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->d_status, 0, sizeof(h), s) != cudaSuccess) return DSN_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DSN_ERR_CUDA;
+  if (code) *code = h[0];
+  if (detail) *detail = h[1];
+  return DSN_OK;
+}
+
+int dsn_widths_from_ratios(int32_t C, const double* ratios, int32_t T, int32_t granule, int32_t* widths_out) {
+  if (C < 1 || !ratios || !widths_out || T < 1 || granule < 0) return DSN_ERR_INVALID_ARG;
+  int g = granule;
+  if (g == 0) {
+    g = C / 32 < 8 ? C / 32 : 8;
+    if (g < 1) g = 1;
+  }
+  for (int t = 0; t < T; ++t) {
+    if (!(ratios[t] > 0.0) || ratios[t] > 1.0) return DSN_ERR_INVALID_ARG;
+    long k = (long)g * (long)floor(ratios[t] * C / g + 0.5 + 1e-9);
+    if (k < g) k = g;
+    if (k > C) k = C;
+    widths_out[t] = (int32_t)k;
+  }
+  return DSN_OK;
+}
+
+int64_t dsn_executed_macs(const int32_t* counts, int32_t T, int32_t R, const int32_t* k_in, const int32_t* k_out,
+                          int32_t K) {
+  if (!counts || !k_in || !k_out || T < 1) return -1;
+  int64_t total = 0;
+  for (int t = 0; t < T; ++t) total += (int64_t)counts[t] * R * k_in[t] * k_out[t] * K * K;
+  return total;
+}
+
+size_t dsn_gate_workspace_bytes(const dsn_gate_desc* g) {
+  if (check_gate(g)) return 0;
+  // the split count depends on the SM count; size for the largest count the launcher can pick
+  int splits = g->R / 8 > 0 ? g->R / 8 : 1;
+  if (splits > 64) splits = 64;
+  return align_up((size_t)g->B * splits * g->c_valid * sizeof(float), 256) + 256;
+}
+
+int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out, float* logits_out,
+             void* workspace, size_t ws_bytes, void* stream) {
+  if (!ctx || !x || !idx_out) return DSN_ERR_INVALID_ARG;
+  int e = check_gate(g);
+  if (e) return e;
+  if (g->B == 0) return DSN_OK;
+  const int splits = dsn_gate_splits(*g, ctx->sm_count);
+  const size_t need = (size_t)g->B * splits * g->c_valid * sizeof(float);
+  if (!workspace || ws_bytes < need) return DSN_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return DSN_ERR_ALIGNMENT;
+  if (dsn_launch_gate(*g, x, idx_out, logits_out, static_cast<float*>(workspace), splits, ctx->d_status,
+                      as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_route(dsn_ctx* ctx, const int32_t* idx, int32_t B, int32_t T, dsn_routing* out, void* stream) {
+  if (!ctx || !idx || !out || B < 0 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (!out->counts || !out->offsets || !out->perm || !out->inv_perm) return DSN_ERR_INVALID_ARG;
+  out->B = B;
+  out->G = T;
+  out->group_slice = nullptr;
+  if (dsn_launch_route(idx, B, T, out->counts, out->offsets, out->perm, out->inv_perm, ctx->d_status,
+                       as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_permute_rows(dsn_ctx* ctx, const dsn_routing* r, int32_t dtype, int32_t R, int32_t T, const int32_t* k,
+                     const void* src, int64_t ld_src, void* dst, int64_t ld_dst, int32_t to_grouped, void* stream) {
+  if (!ctx || !src || !dst || !k || R < 1 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (dtype != DSN_BF16 && dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
+  int e = check_routing(r, T);
+  if (e) return e;
+  SliceTable st;
+  memset(&st, 0, sizeof(st));
+  for (int t = 0; t < T; ++t) {
+    if (k[t] < 1 || k[t] > ld_src || k[t] > ld_dst) return DSN_ERR_INVALID_ARG;
+    st.k_in[t] = k[t];
+  }
+  if (dsn_launch_permute_rows(st, dtype == DSN_BF16 ? 2 : 4, R, src, ld_src, dst, ld_dst, to_grouped ? 1 : 0, r->B,
+                              r->G, r->offsets, r->perm, r->group_slice, as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+size_t dsn_linear_workspace_bytes(const dsn_linear_desc* d, int32_t B) {
+  (void)d; (void)B;
+  return 0;  // the tile schedule is rebuilt inside the kernel from the group offsets
+}
+size_t dsn_conv_workspace_bytes(const dsn_conv_desc* d, int32_t B) {
+  (void)d; (void)B;
+  return 0;
+}
+
+int dsn_sliced_linear(dsn_ctx* ctx, const dsn_linear_desc* d, const dsn_routing* r, const void* x, void* y,
+                      void* workspace, size_t ws_bytes, void* stream) {
+  (void)workspace; (void)ws_bytes;
+  if (!d || d->R < 1) return DSN_ERR_INVALID_ARG;
+  return run_layer(ctx, from_linear(d), r, x, y, as_stream(stream));
+}
+
+int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, const void* x, void* y,
+                    void* workspace, size_t ws_bytes, void* stream) {
+  (void)workspace; (void)ws_bytes;
+  if (!d) return DSN_ERR_INVALID_ARG;
+  if (d->dtype != DSN_BF16) return DSN_ERR_UNSUPPORTED;
+  return run_layer(ctx, from_conv(d), r, x, y, as_stream(stream));
+}
+
+size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L) {
+  LayerPlan pl;
+  if (plan_layer(L, pl)) return 0;
+  return pl.total + 256;
+}
+
+int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, const int32_t* idx_in, void* y,
+                      dsn_routing* r_out, int32_t* idx_out, void* workspace, size_t ws_bytes, void* stream) {
+  if (!ctx || !L || !x || !y) return DSN_ERR_INVALID_ARG;
+  LayerPlan pl;
+  int e = plan_layer(L, pl);
+  if (e) return e;
+  if (!L->gate && !idx_in) return DSN_ERR_INVALID_ARG;
+  if (L->gate && (L->gate->B != L->B || L->gate->T != L->T)) return DSN_ERR_INVALID_ARG;
+  if (!workspace || ws_bytes < pl.total) return DSN_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSN_ERR_ALIGNMENT;
+  char* ws = static_cast<char*>(workspace);
+  cudaStream_t s = as_stream(stream);
+
+  // validate every layer before the first launch
+  LayerCall calls[DSN_MAX_CHAIN];
+  dsn_routing r;
+  r.B = L->B;
+  r.G = L->T;
+  r.counts = reinterpret_cast<int32_t*>(ws + pl.off_counts);
+  r.offsets = reinterpret_cast<int32_t*>(ws + pl.off_offsets);
+  r.perm = reinterpret_cast<int32_t*>(ws + pl.off_perm);
+  r.inv_perm = reinterpret_cast<int32_t*>(ws + pl.off_inv);
+  r.group_slice = nullptr;
+  const void* src = x;
+  for (int j = 0; j < L->n_layers; ++j) {
+    LayerCall& c = calls[j];
+    layer_call_of(L, j, c);
+    const bool first = j == 0, last = j + 1 == L->n_layers;
+    c.in_order = (first && !pl.gather_first) ? DSN_INPUT_ORDER : DSN_GROUPED;
+    c.out_order = last ? DSN_INPUT_ORDER : DSN_GROUPED;
+    if (first && pl.gather_first) c.ldx = c.C_in;
+    if (!first) c.ldx = calls[j - 1].C_out;
+    if (!last) c.ldy = c.C_out;
+    const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
+                           : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
+    void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
+    e = validate_call(c, &r, in, out);
+    if (e) return e;
+  }
+  (void)src;
+
+  const int32_t* idx = idx_in;
+  if (L->gate) {
+    int32_t* gi = idx_out ? idx_out : reinterpret_cast<int32_t*>(ws + pl.off_idx);
+    e = dsn_gate(ctx, L->gate, x, gi, nullptr, ws + pl.off_gate, dsn_gate_workspace_bytes(L->gate), stream);
+    if (e) return e;
+    idx = gi;
+  } else if (idx_out && L->B > 0) {
+    if (cudaMemcpyAsync(idx_out, idx_in, 4 * (size_t)L->B, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+      return DSN_ERR_CUDA;
+  }
+  e = dsn_route(ctx, idx, L->B, L->T, &r, stream);
+  if (e) return e;
+  if (r_out) *r_out = r;
+
+  if (pl.gather_first) {
+    const LayerCall& c0 = calls[0];
+    const dsn_linear_desc* dl = L->kind[0] == DSN_LAYER_LINEAR ? static_cast<const dsn_linear_desc*>(L->layer[0]) : nullptr;
+    const int64_t ld_src = dl ? dl->ldx : static_cast<const dsn_conv_desc*>(L->layer[0])->ldx;
+    e = dsn_permute_rows(ctx, &r, c0.dtype, c0.H * c0.W, c0.T, c0.k_in, x, ld_src, ws + pl.off_gather, c0.C_in, 1,
+                         stream);
+    if (e) return e;
+  }
+  for (int j = 0; j < L->n_layers; ++j) {
+    const bool first = j == 0, last = j + 1 == L->n_layers;
+    const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
+                           : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
+    void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
+    e = run_layer(ctx, calls[j], &r, in, out, s);
+    if (e) return e;
+  }
+  return DSN_OK;
+}
+
+}  // extern "C"

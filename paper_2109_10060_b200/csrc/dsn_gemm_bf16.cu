@@ -1,0 +1,452 @@
+// Ragged grouped sliced GEMM, bf16 operands, fp32 accumulation, for sm_100a.
+//
+//   for every group g (samples routed to one path, slice (k_in, k_out)):
+//       Y[rows of g, :k_out] = act( X[rows of g, :k_in] * W[:k_out, :k_in]^T + bias )
+//
+// The same kernel covers linear layers, 1x1 convolutions and 3x3 convolutions as implicit GEMM
+// over channels-last activations: the reduction runs over (tap, channel chunk) and the activation
+// tile of tap (r, s) is the output tile's pixel rectangle shifted by (r - pad, s - pad); the TMA
+// unit zero-fills what falls outside the image, which is the convolution's zero padding.
+//
+// Operands are read in place.  Every distinct k_in has its own pair of tensor maps whose
+// innermost extent is k_in but whose strides are those of the full tensors, so the channels
+// beyond the slice arrive in shared memory as zeros and are never multiplied.
+//
+// Structure of a CTA (persistent, one per SM, 192 threads):
+//   warp 0      one lane issues the TMA loads into a ring of shared-memory stages
+//   warp 1      one lane issues tcgen05.mma (M = 128, N = 16..256, K = 16) into a TMEM accumulator;
+//               two accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
+//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), bias / activation,
+//               bf16 rounding, stores to the grouped or the input-order (scattered) output
+// Every mbarrier wait is bounded; on a timeout the CTA records DSN_ERR_TIMEOUT, stops issuing
+// work, lets its copies land, frees its TMEM and returns.
+#include "dsn_internal.cuh"
+#include "dsn_tiles.cuh"
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int BM = DSN_GEMM_BM;
+constexpr int BK = DSN_GEMM_BK;
+constexpr uint32_t kABytes = BM * BK * 2;  // 16 KB: 128 rows of 128 bytes
+constexpr uint32_t kCtrlBytes = 1024;
+constexpr int kMaxStages = 8;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+// ---------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this or another thread ran out of time).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            int32_t* status, int where) {
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 31u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        dsn_set_status(status, DSN_ERR_TIMEOUT, where);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          int32_t* status, int where) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, where);
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the mbarrier receives one arrival once every tcgen05.mma issued so far by this thread is done
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, 8-row groups
+// 1024 bytes apart (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
+__device__ __forceinline__ uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ float apply_act(float v, int act) {
+  if (act == DSN_ACT_RELU) return fmaxf(v, 0.f);
+  if (act == DSN_ACT_GELU) return 0.5f * v * (1.f + erff(v * 0.70710678118654752f));
+  return v;
+}
+
+// ---------------------------------------------------------------------------------- tile decode
+struct TileInfo {
+  int map, ki, ko, n0;
+  int p_end;            // one past the group's last grouped position
+  int row0, rows_end;   // flat: first grouped row of the tile, one past the group's last row
+  int b0, x0, y0;       // per-image tiling: first position, pixel origin
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int32_t* s_prefix, int tile) {
+  TileInfo t;
+  const GemmGeom& g = p.g;
+  const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
+  const int grp = p.G - 1 - j;
+  const int sl = p.group_slice ? p.group_slice[grp] : grp;
+  t.map = p.map_id[sl];
+  t.ki = p.k_in[sl];
+  t.ko = p.k_out[sl];
+  const int p0 = p.offsets[grp];
+  t.p_end = p.offsets[grp + 1];
+  const int ntn = (t.ko + g.BN - 1) / g.BN;
+  const int local = tile - s_prefix[j];
+  const int nt = local % ntn, mt = local / ntn;
+  t.n0 = nt * g.BN;
+  if (g.flat) {
+    t.row0 = p0 * g.R + mt * BM;
+    t.rows_end = t.p_end * g.R;
+    t.b0 = t.x0 = t.y0 = 0;
+  } else {
+    const int per_img = g.tiles_x * g.tiles_y;
+    const int ib = mt / per_img, rem = mt - ib * per_img;
+    const int ty = rem / g.tiles_x, tx = rem - ty * g.tiles_x;
+    t.b0 = p0 + ib * g.nb;
+    t.y0 = ty * g.bh;
+    t.x0 = tx * g.bw;
+    t.row0 = t.rows_end = 0;
+  }
+  return t;
+}
+
+// ---------------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const GemmGeom& g = p.g;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+
+  // control block
+  const uint32_t bar_full = base;                       // [kMaxStages]
+  const uint32_t bar_empty = base + 8 * kMaxStages;     // [kMaxStages]
+  const uint32_t bar_tfull = base + 16 * kMaxStages;    // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;           // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16 * kMaxStages + 32);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxStages + 36);
+
+  const int stages = g.stages;
+  const uint32_t b_bytes = (uint32_t)g.BN * BK * 2;
+  const uint32_t stage_bytes = kABytes + b_bytes;
+  const uint32_t tiles_base = base + kCtrlBytes;
+  int32_t* s_prefix = reinterpret_cast<int32_t*>(smem + kCtrlBytes + (size_t)stages * stage_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tmem_cols = 2u * (uint32_t)g.BN;  // 128, 256 or 512: a power of two >= 32
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), tmem_cols);
+    tmem_relinquish();
+  }
+
+  auto ntiles_of = [&](int grp) {
+    const int sl = p.group_slice ? p.group_slice[grp] : grp;
+    if (sl < 0 || sl >= p.T || p.map_id[sl] == 0xFF) return 0;
+    const int cnt = p.offsets[grp + 1] - p.offsets[grp];
+    if (cnt <= 0) return 0;
+    const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
+    return mt * ((p.k_out[sl] + g.BN - 1) / g.BN);
+  };
+  dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);  // contains __syncthreads
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = s_prefix[p.G];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x) {
+        const TileInfo t = decode_tile(p, s_prefix, tile);
+        const CUtensorMap* mA = &p.mapA[t.map];
+        const CUtensorMap* mB = &p.mapB[t.map];
+        const int nkc = (t.ki + BK - 1) / BK;
+        int bsel = t.b0;
+        if (g.a_input_order) bsel = p.perm[t.b0];
+        for (int tap = 0; ok && tap < g.taps; ++tap) {
+          const int r = tap / g.KW, s = tap - r * g.KW;
+          for (int kc = 0; kc < nkc; ++kc) {
+            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+            const uint32_t full = bar_full + 8 * stage;
+            mbar_expect_tx(full, a_box_bytes + b_bytes);
+            const uint32_t sa = tiles_base + stage * stage_bytes;
+            if (g.flat) tma_load_4d(sa, mA, kc * BK, t.row0, 0, 0, full);
+            else tma_load_4d(sa, mA, kc * BK, t.x0 + s - g.pad, t.y0 + r - g.pad, bsel, full);
+            tma_load_3d(sa + kABytes, mB, kc * BK, tap, t.n0, full);
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        // let copies already issued land before the CTA gives up its shared memory
+        for (int s = 0; s < stages; ++s) {
+          const uint64_t t0 = globaltimer_ns();
+          const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+          while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < 1000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
+        const TileInfo t = decode_tile(p, s_prefix, tile);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
+        tc_fence_after();
+        int n_inst = t.ko - t.n0;
+        n_inst = n_inst > g.BN ? g.BN : ((n_inst + 15) & ~15);
+        const uint32_t idesc = make_idesc(BM, n_inst);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
+        const int nkc = (t.ki + BK - 1) / BK;
+        uint32_t accumulate = 0;
+        for (int tap = 0; ok && tap < g.taps; ++tap) {
+          for (int kc = 0; kc < nkc; ++kc) {
+            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 3)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = tiles_base + stage * stage_bytes;
+            const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kABytes);
+            const int krem = t.ki - kc * BK;
+            const int nks = krem >= BK ? BK / 16 : (krem + 15) >> 4;
+            for (int ks = 0; ks < nks; ++ks) {
+              umma_bf16(d_tmem, da + 2u * ks, db + 2u * ks, idesc, accumulate);  // +32 bytes per K step
+              accumulate = 1;
+            }
+            umma_commit(bar_empty + 8 * stage);
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+        if (ok) umma_commit(bar_tfull + 8 * acc);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;          // TMEM lane quarter this warp may read
+    const int m = q * 32 + lane;     // accumulator row of this thread
+    int it = 0;
+    bool ok = true;
+    const int box_rows = g.bw * g.bh * g.nb, img_rows = g.bw * g.bh;
+    for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
+      const TileInfo t = decode_tile(p, s_prefix, tile);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+
+      bool valid;
+      int64_t out_row;
+      if (g.flat) {
+        const int gr = t.row0 + m;
+        valid = gr < t.rows_end;
+        out_row = gr;
+        if (valid && g.y_input_order) {
+          const int pp = gr / g.R;
+          out_row = (int64_t)p.perm[pp] * g.R + (gr - pp * g.R);
+        }
+      } else {
+        const int bi = m / img_rows, rem = m - bi * img_rows;
+        const int yy = t.y0 + rem / g.bw, xx = t.x0 + rem % g.bw;
+        const int pp = t.b0 + bi;
+        valid = m < box_rows && yy < g.H && xx < g.W && pp < t.p_end;
+        out_row = 0;
+        if (valid) {
+          const int smp = g.y_input_order ? p.perm[pp] : pp;
+          out_row = (int64_t)smp * g.R + yy * g.W + xx;
+        }
+      }
+      __nv_bfloat16* yrow = p.y + out_row * p.ldy + t.n0;
+      const float* brow = p.bias ? p.bias + t.n0 : nullptr;
+      int ncols = t.ko - t.n0;
+      ncols = ncols > g.BN ? g.BN : ncols;
+
+      // every lane waits, then the warp takes one decision so that tcgen05.ld stays warp-wide
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 4));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
+      for (int c0 = 0; c0 < ncols; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + c0, v);
+        tmem_ld_wait();
+        if (valid) {
+          const int nv = ncols - c0 < 32 ? ncols - c0 : 32;
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float a = __uint_as_float(v[2 * i]), b = __uint_as_float(v[2 * i + 1]);
+            if (brow) {
+              if (2 * i < nv) a += __ldg(brow + c0 + 2 * i);
+              if (2 * i + 1 < nv) b += __ldg(brow + c0 + 2 * i + 1);
+            }
+            a = apply_act(a, p.act);
+            b = apply_act(b, p.act);
+            __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+            packed[i] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          __nv_bfloat16* dst = yrow + c0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (8 * i + 8 <= nv) {
+              reinterpret_cast<uint4*>(dst)[i] =
+                  make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+            } else if (8 * i < nv) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                if (8 * i + e < nv) {
+                  const uint32_t w = packed[4 * i + e / 2];
+                  reinterpret_cast<uint16_t*>(dst)[8 * i + e] = (e & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xffffu);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+}  // namespace
+
+size_t dsn_gemm_smem_bytes(int BN, int stages) {
+  return 1024 /* alignment slack */ + kCtrlBytes + (size_t)stages * (kABytes + (size_t)BN * BK * 2) +
+         sizeof(int32_t) * (DSN_MAX_GROUPS + 1);
+}
+
+cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s) {
+  static size_t configured = 0;
+  if (smem_bytes > configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) return e;
+    configured = smem_bytes;
+  }
+  gemm_bf16_kernel<<<sm_count, kThreads, smem_bytes, s>>>(p);
+  return cudaGetLastError();
+}

@@ -1,0 +1,96 @@
+// Internal declarations shared by the translation units of libdsn (never installed).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dsn.h"
+
+// Device status word: [0] = first condition code, [1] = detail, [2] = count of non-finite gate
+// scores, [3] = count of out-of-range routing indices.
+#define DSN_STATUS_WORDS 4
+
+struct dsn_ctx {
+  int device;
+  int sm_count;
+  int32_t* d_status;   // DSN_STATUS_WORDS ints
+  void* encode_tiled;  // cuTensorMapEncodeTiled entry point
+};
+
+__device__ __forceinline__ void dsn_set_status(int32_t* status, int code, int detail) {
+  if (status && atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Grouped GEMM parameters (bf16, tcgen05).  One launch covers every group whose slice has a
+// tensor map in this launch (map_id != 0xFF).
+// ----------------------------------------------------------------------------------------------
+#define DSN_GEMM_MAX_MAPS 16
+#define DSN_GEMM_BM 128
+#define DSN_GEMM_BK 64
+
+struct GemmGeom {
+  // activation tensor seen as [Bdim][H][W][C]; a linear layer is H = 1 (rows along W)
+  int32_t H, W;            // "image" extents of one sample (input-order / per-image tiling)
+  int32_t R;               // rows per sample = H*W
+  int32_t taps, KW, pad;   // taps = K*K
+  int32_t bw, bh, nb;      // A box = bw x bh pixels x nb images  (bw*bh*nb <= 128)
+  int32_t tiles_x, tiles_y;
+  int32_t flat;            // 1: grouped rows tiled without regard to sample boundaries
+  int32_t a_input_order;   // A read by sample index perm[p] (needs nb == 1, flat == 0)
+  int32_t y_input_order;   // rows scattered to sample perm[p]
+  int32_t BN;              // n-tile (64, 128, 256) = rows of the weight box
+  int32_t stages;
+};
+
+struct GemmParams {
+  CUtensorMap mapA[DSN_GEMM_MAX_MAPS];
+  CUtensorMap mapB[DSN_GEMM_MAX_MAPS];
+  int16_t k_in[DSN_MAX_SLICES];
+  int16_t k_out[DSN_MAX_SLICES];
+  uint8_t map_id[DSN_MAX_SLICES];
+  GemmGeom g;
+  int32_t B, G, T;
+  const int32_t* offsets;
+  const int32_t* perm;
+  const int32_t* group_slice;
+  __nv_bfloat16* y;
+  int64_t ldy;
+  const float* bias;
+  int32_t act;
+  int32_t* status;
+};
+
+// launchers implemented in the .cu files
+cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
+size_t dsn_gemm_smem_bytes(int BN, int stages);
+
+cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_out, float* logits_out,
+                            float* partial, int splits, int32_t* status, cudaStream_t s);
+int dsn_gate_splits(const dsn_gate_desc& g, int sm_count);
+
+cudaError_t dsn_launch_route(const int32_t* idx, int B, int T, int32_t* counts, int32_t* offsets,
+                             int32_t* perm, int32_t* inv_perm, int32_t* status, cudaStream_t s);
+
+struct SliceTable {
+  int32_t k_in[DSN_MAX_SLICES];
+  int32_t k_out[DSN_MAX_SLICES];
+};
+
+cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const float* x, int64_t ldx,
+                                  const float* W, int64_t ldw, float* y, int64_t ldy, const float* bias,
+                                  int act, int x_input_order, int y_input_order, int B, int G,
+                                  const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
+                                  int sm_count, cudaStream_t s);
+
+cudaError_t dsn_launch_permute_rows(const SliceTable& st, int elem_bytes, int R, const void* src,
+                                    int64_t ld_src, void* dst, int64_t ld_dst, int to_grouped, int B, int G,
+                                    const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
+                                    cudaStream_t s);
+
+// Zero columns k_out[t] .. C_out-1 of every row (dsn_tail = ZERO).
+cudaError_t dsn_launch_zero_tail(const SliceTable& st, int elem_bytes, int R, int C_out, void* y, int64_t ldy,
+                                 int y_input_order, int B, int G, const int32_t* offsets, const int32_t* perm,
+                                 const int32_t* group_slice, cudaStream_t s);

@@ -1,0 +1,197 @@
+"""GPU parity of dsn_sliced_conv and dsn_layer_forward chains against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import dsn_workloads as wl
+from oracle import dsn_oracle as O
+from gpu_util import (DEV, SENTINEL, assert_tail_untouched, check_status, down, group_errors, route_on_gpu, up_bf16,
+                      up_f32, up_i32)
+
+pytestmark = pytest.mark.gpu
+TOL_BF16 = 5e-3
+
+
+@pytest.fixture(scope="module")
+def ctx(dsn):
+    return dsn.Context(0)
+
+
+def ohwi(W):
+    """[C_O][C_I][K][K] (the paper's indexing) -> [C_O][K][K][C_I] (the library's storage)."""
+    return np.ascontiguousarray(np.transpose(W, (0, 2, 3, 1)))
+
+
+def _run_conv(dsn, ctx, x, W, idx, k_in, k_out, pad, in_order=0, out_order=0, act=0, bias=None):
+    B, H, Wd, Ci = x.shape
+    Co, _, K, _ = W.shape
+    T = len(k_in)
+    r = route_on_gpu(dsn, ctx, idx, T)
+    perm = O.route(idx, T)[2]
+    xs = x[perm] if in_order else x
+    y = torch.full((B, H, Wd, Co), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    d = dsn.make_conv_desc(dsn.BF16, H, Wd, K, pad, Ci, Co, k_in, k_out, up_bf16(ohwi(W)),
+                           bias=None if bias is None else up_f32(bias), act=act, in_order=in_order, out_order=out_order)
+    dsn.dsn_sliced_conv(ctx, d, r, up_bf16(xs), y)
+    check_status(ctx, dsn)
+    got = down(y)
+    if out_order:
+        tmp = np.empty_like(got)
+        tmp[perm] = got
+        got = tmp
+    return got
+
+
+@pytest.mark.parametrize("hw,C,B,orders", [(14, 256, 20, (0, 0)), (14, 256, 20, (1, 1)), (7, 512, 21, (1, 0)),
+                                           (7, 512, 9, (0, 1)), (28, 128, 6, (1, 1)), (56, 64, 3, (0, 0)),
+                                           (56, 64, 3, (1, 1))])
+def test_conv3x3_resnet_stage_shapes(dsn, ctx, hw, C, B, orders):
+    """3x3, pad 1, w -> w with the 14 ResNet-50 widths of that stage (22, 26, ... are no multiple of 16)."""
+    g = np.random.default_rng(hw * 1000 + C + B)
+    widths = wl.WIDTHS_14[C]
+    T = len(widths)
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    x = wl.normal(g, (B, hw, hw, C), relu=True)
+    W = wl.normal(g, (C, C, 3, 3), std=(9 * C) ** -0.5)
+    bias = g.standard_normal(C).astype(np.float32) * 0.2
+    got = _run_conv(dsn, ctx, x, W, idx, widths, widths, 1, orders[0], orders[1], act=dsn.ACT_RELU, bias=bias)
+    ref = O.round_bf16(O.sliced_conv(x, W, idx, widths, widths, 1, bias=bias, act=O.ACT_RELU))
+    errs = group_errors(got, ref, idx, widths, T)
+    assert max(errs.values()) <= TOL_BF16, errs
+    assert_tail_untouched(got, idx, widths)
+
+
+@pytest.mark.parametrize("orders", [(0, 0), (1, 1), (0, 1)])
+def test_conv1x1_both_directions(dsn, ctx, orders):
+    g = np.random.default_rng(77)
+    B, hw, C, Ci = 24, 14, 1024, 256
+    widths = wl.WIDTHS_14[Ci]
+    T = len(widths)
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    x = wl.normal(g, (B, hw, hw, C), relu=True)
+    W1 = wl.normal(g, (Ci, C, 1, 1), std=C ** -0.5)
+    got = _run_conv(dsn, ctx, x, W1, idx, [C] * T, widths, 0, orders[0], orders[1], act=dsn.ACT_RELU)
+    ref = O.round_bf16(O.sliced_conv(x, W1, idx, [C] * T, widths, 0, act=O.ACT_RELU))
+    assert max(group_errors(got, ref, idx, widths, T).values()) <= TOL_BF16
+    assert_tail_untouched(got, idx, widths)
+    x2 = wl.normal(g, (B, hw, hw, Ci), relu=True)
+    W3 = wl.normal(g, (C, Ci, 1, 1), std=Ci ** -0.5)
+    got = _run_conv(dsn, ctx, x2, W3, idx, widths, [C] * T, 0, orders[0], orders[1])
+    ref = O.round_bf16(O.sliced_conv(x2, W3, idx, widths, [C] * T, 0))
+    assert max(group_errors(got, ref, idx, [C] * T, T).values()) <= TOL_BF16
+
+
+def test_conv3x3_delta_and_padding_on_device(dsn, ctx):
+    """Orientation (no kernel flip) and zero padding, checked on the device path itself."""
+    H = Wd = 5
+    C = 16
+    x = np.zeros((2, H, Wd, C), np.float32)
+    x[0, 2, 2, 0] = 1.0
+    x[1] = 1.0
+    W = np.zeros((C, C, 3, 3), np.float32)
+    W[0, 0] = np.arange(9, dtype=np.float32).reshape(3, 3)
+    W[1, :, :, :] = 1.0
+    got = _run_conv(dsn, ctx, x, W, np.array([0, 0], np.int32), [C], [C], 1)
+    ref = O.sliced_conv(x, W, [0, 0], [C], [C], 1)
+    np.testing.assert_array_equal(got, ref)
+    assert got[0, 1, 1, 0] == 8.0 and got[0, 3, 3, 0] == 0.0 and got[0, 1, 3, 0] == 6.0
+    assert got[1, 2, 2, 1] == 9 * C and got[1, 0, 2, 1] == 6 * C and got[1, 0, 0, 1] == 4 * C
+
+
+def _bottleneck_forward(dsn, ctx, cfg, with_gate):
+    B, H, Wd, C, Ci, T, widths = cfg["B"], cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"], cfg["widths"]
+    full = [C] * T
+    W1, W2, W3 = up_bf16(cfg["W1"].reshape(Ci, C)), up_bf16(ohwi(cfg["W2"])), up_bf16(cfg["W3"].reshape(C, Ci))
+    layers = [dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, Ci, full, widths, W1, act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 3, 1, Ci, Ci, widths, widths, W2, act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, Ci, C, widths, full, W3)]
+    gate = None
+    if with_gate:
+        gW1, gW2 = up_f32(cfg["gate_W1"]), up_f32(cfg["gate_W2"])
+        gate = dsn.make_gate_desc(dsn.BF16, B, H * Wd, C, gW1.shape[0], T, gW1, gW2)
+    L = dsn.make_layer_desc(B, T, layers, gate)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, H, Wd, C), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    idx_out = torch.full((B,), -1, dtype=torch.int32, device=DEV)
+    r_out = dsn.Routing()
+    dsn.dsn_layer_forward(ctx, L, up_bf16(cfg["x"]), None if with_gate else up_i32(cfg["idx"]), y, ws, r_out=r_out,
+                          idx_out=idx_out)
+    check_status(ctx, dsn)
+    return down(y), idx_out.cpu().numpy(), r_out, ws
+
+
+def test_layer_forward_bottleneck_with_gate(dsn, ctx):
+    """Config-2 style block end to end: gate -> route -> 1x1 -> 3x3 -> 1x1 -> input order."""
+    cfg = wl.config2(B=48)
+    got, idx_gpu, r_out, ws = _bottleneck_forward(dsn, ctx, cfg, with_gate=True)
+    B, R, C = cfg["B"], cfg["H"] * cfg["W"], cfg["C_outer"]
+    idx_ref, _, margin = O.gate(cfg["x"].reshape(B, R, C), cfg["gate_W1"], cfg["gate_W2"])
+    safe = margin >= 1e-4
+    np.testing.assert_array_equal(idx_gpu[safe], idx_ref[safe])
+    idx_used = np.where(safe, idx_ref, idx_gpu)            # inside the margin adopt the device's pick
+    assert np.all((idx_used >= 0) & (idx_used < cfg["T"]))
+    _, _, ref = O.bottleneck(cfg["x"], cfg["W1"], cfg["W2"], cfg["W3"], idx_used, cfg["widths"], mirror_bf16=True)
+    errs = group_errors(got, ref, idx_used, [C] * cfg["T"], cfg["T"])
+    assert max(errs.values()) <= TOL_BF16, errs
+    # routing arrays left in the workspace are the stable grouping of the gate's choice
+    assert r_out.B == B and r_out.G == cfg["T"]
+    base = ws.data_ptr()
+    def view(ptr, n):
+        off = ptr - base
+        return ws[off:off + 4 * n].view(torch.int32).cpu().numpy()
+    counts, offsets, perm, inv = O.route(idx_gpu, cfg["T"])
+    np.testing.assert_array_equal(view(r_out.counts, cfg["T"]), counts)
+    np.testing.assert_array_equal(view(r_out.offsets, cfg["T"] + 1), offsets)
+    np.testing.assert_array_equal(view(r_out.perm, B), perm)
+    np.testing.assert_array_equal(view(r_out.inv_perm, B), inv)
+
+
+@pytest.mark.parametrize("stage,B,routing", [(1, 4, "skewed14"), (2, 14, "uniform"), (4, 40, "uniform")])
+def test_layer_forward_bottleneck_resnet_stages(dsn, ctx, stage, B, routing):
+    hw, outer, inner = wl.RESNET_STAGES[stage]
+    cfg = wl.bottleneck(40 + stage, B, hw, hw, outer, inner, routing="iid" if routing == "skewed14" else routing,
+                        with_gate=False)
+    got, idx_gpu, _, _ = _bottleneck_forward(dsn, ctx, cfg, with_gate=False)
+    np.testing.assert_array_equal(idx_gpu, cfg["idx"])
+    _, _, ref = O.bottleneck(cfg["x"], cfg["W1"], cfg["W2"], cfg["W3"], cfg["idx"], cfg["widths"], mirror_bf16=True)
+    errs = group_errors(got, ref, cfg["idx"], [outer] * cfg["T"], cfg["T"])
+    assert max(errs.values()) <= TOL_BF16, errs
+
+
+def test_layer_forward_vit_mlp_and_config1(dsn, ctx):
+    cfg = wl.config3(B=64, routing="uniform")
+    B, R, De, Dm, T, paths = cfg["B"], cfg["R"], cfg["D_e"], cfg["D_mlp"], cfg["T"], cfg["paths"]
+    ki1, ko1 = wl.vit_layer_slices(paths, 64, "fc1")
+    ki2, ko2 = wl.vit_layer_slices(paths, 64, "fc2")
+    layers = [dsn.make_linear_desc(dsn.BF16, R, De, Dm, ki1, ko1, up_bf16(cfg["Wfc1"]), act=dsn.ACT_GELU),
+              dsn.make_linear_desc(dsn.BF16, R, Dm, De, ki2, ko2, up_bf16(cfg["Wfc2"]))]
+    gW1, gW2 = up_f32(cfg["gate_W1"]), up_f32(cfg["gate_W2"])
+    gate = dsn.make_gate_desc(dsn.BF16, B, R, De, gW1.shape[0], T, gW1, gW2)
+    L = dsn.make_layer_desc(B, T, layers, gate)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, R, De), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    idx_out = torch.zeros(B, dtype=torch.int32, device=DEV)
+    dsn.dsn_layer_forward(ctx, L, up_bf16(cfg["x"]), None, y, ws, idx_out=idx_out)
+    check_status(ctx, dsn)
+    idx_gpu = idx_out.cpu().numpy()
+    idx_ref, _, margin = O.gate(cfg["x"], cfg["gate_W1"], cfg["gate_W2"])
+    safe = margin >= 1e-4
+    np.testing.assert_array_equal(idx_gpu[safe], idx_ref[safe])
+    idx_used = np.where(safe, idx_ref, idx_gpu)
+    _, ref = O.vit_mlp(cfg["x"], cfg["Wfc1"], cfg["Wfc2"], idx_used, paths, mirror_bf16=True)
+    got = down(y)
+    errs = group_errors(got, ref, idx_used, ko2, T)
+    assert max(errs.values()) <= TOL_BF16, errs
+    assert_tail_untouched(got, idx_used, ko2)
+
+    # config 1: single fp32 layer, gate bypassed
+    c1 = wl.config1()
+    d = dsn.make_linear_desc(dsn.F32, 1, 256, 256, c1["k_in"], c1["k_out"], up_f32(c1["W"]))
+    L1 = dsn.make_layer_desc(c1["B"], 4, [d])
+    ws1 = torch.empty(dsn.dsn_layer_workspace_bytes(L1), dtype=torch.uint8, device=DEV)
+    y1 = torch.full((c1["B"], 1, 256), SENTINEL, dtype=torch.float32, device=DEV)
+    dsn.dsn_layer_forward(ctx, L1, up_f32(c1["x"]), up_i32(c1["idx"]), y1, ws1)
+    check_status(ctx, dsn)
+    ref1 = O.sliced_linear(c1["x"], c1["W"], c1["idx"], c1["k_in"], c1["k_out"])
+    assert max(group_errors(down(y1), ref1, c1["idx"], c1["k_out"], 4).values()) <= 1e-5
+    assert_tail_untouched(down(y1), c1["idx"], c1["k_out"])
