@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the dynamic-weight-slicing hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: gate (average pool,
+FC-ReLU-FC, arg-max) -> routing (stable grouping) -> the block's sliced grouped GEMMs -> outputs in
+input order.  Default workload: ResNet-50 stage-3 dynamic bottleneck, bf16 NHWC, batch 128, 14x14,
+1x1 1024->w, 3x3 w->w, 1x1 w->1024 with 14 inner widths, gate-driven routing.
+
+Prints ONE JSON line (see --help).  `value` is executed TFLOP/s of the whole step (2 x multiply-adds
+of the sliced layers actually run, divided by the step time, gate and routing included), inputs
+resident in HBM.  `e2e` is the same metric with the batch starting and ending in pinned host memory.
+`roofline` describes the grouped-GEMM kernel, `cpu_baseline` the fp64 CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# --------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.samples.append(line.strip())
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.samples:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- workloads
+class Bottleneck:
+    """ResNet-50-style dynamic bottleneck (configs 2 and 4)."""
+
+    def __init__(self, dsn, torch, dev, cfg, gate_driven=True, copies=None):
+        import dsn_workloads as wl
+        self.dsn, self.torch, self.dev, self.cfg = dsn, torch, dev, cfg
+        B, H, Wd, C, Ci, T = cfg["B"], cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"]
+        self.B, self.R, self.C, self.T, self.widths = B, H * Wd, C, T, cfg["widths"]
+        self.gate_driven = gate_driven
+        up = lambda a: torch.from_numpy(wl.bf16_bits(np.ascontiguousarray(a)).view(np.int16)).to(dev).view(torch.bfloat16)
+        self.x_host_bits = wl.bf16_bits(cfg["x"]).view(np.int16)
+        x_bytes = self.x_host_bits.nbytes
+        self.copies = copies or max(2, -(-2 * L2_BYTES // (2 * x_bytes)) + 1)   # inputs + outputs rotate past L2
+        self.xs = [torch.from_numpy(self.x_host_bits).to(dev).view(torch.bfloat16).reshape(B, H, Wd, C)
+                   for _ in range(self.copies)]
+        self.ys = [torch.zeros(B, H, Wd, C, dtype=torch.bfloat16, device=dev) for _ in range(self.copies)]
+        self.W1 = up(cfg["W1"].reshape(Ci, C))
+        self.W2 = up(np.transpose(cfg["W2"], (0, 2, 3, 1)))
+        self.W3 = up(cfg["W3"].reshape(C, Ci))
+        full = [C] * T
+        self.slices = [(full, self.widths, 1), (self.widths, self.widths, 3), (self.widths, full, 1)]
+        mk = dsn.make_conv_desc
+        self.layers = [mk(dsn.BF16, H, Wd, 1, 0, C, Ci, full, self.widths, self.W1, act=dsn.ACT_RELU),
+                       mk(dsn.BF16, H, Wd, 3, 1, Ci, Ci, self.widths, self.widths, self.W2, act=dsn.ACT_RELU),
+                       mk(dsn.BF16, H, Wd, 1, 0, Ci, C, self.widths, full, self.W3)]
+        self.gW1 = torch.from_numpy(cfg["gate_W1"]).to(dev)
+        self.gW2 = torch.from_numpy(cfg["gate_W2"]).to(dev)
+        self.gate = dsn.make_gate_desc(dsn.BF16, B, self.R, C, self.gW1.shape[0], T, self.gW1, self.gW2)
+        self.idx_given = torch.from_numpy(cfg["idx"]).to(dev)
+        self.L = dsn.make_layer_desc(B, T, self.layers, self.gate if gate_driven else None)
+        self.ws = torch.empty(dsn.dsn_layer_workspace_bytes(self.L), dtype=torch.uint8, device=dev)
+        self.idx_out = torch.zeros(B, dtype=torch.int32, device=dev)
+        # decomposed form (same kernels, one C call per step of the path) for per-kernel timing
+        self.gate_ws = torch.empty(dsn.dsn_gate_workspace_bytes(self.gate), dtype=torch.uint8, device=dev)
+        ints = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+        self.routing = dsn.make_routing(B, T, ints(T), ints(T + 1), ints(B), ints(B))
+        self.t1 = torch.zeros(B, H, Wd, Ci, dtype=torch.bfloat16, device=dev)
+        self.t2 = torch.zeros(B, H, Wd, Ci, dtype=torch.bfloat16, device=dev)
+        self.dec_layers = [
+            mk(dsn.BF16, H, Wd, 1, 0, C, Ci, full, self.widths, self.W1, act=dsn.ACT_RELU, in_order=0, out_order=1),
+            mk(dsn.BF16, H, Wd, 3, 1, Ci, Ci, self.widths, self.widths, self.W2, act=dsn.ACT_RELU, in_order=1, out_order=1),
+            mk(dsn.BF16, H, Wd, 1, 0, Ci, C, self.widths, full, self.W3, in_order=1, out_order=0)]
+        self.kernels_per_step = (2 if gate_driven else 0) + 1 + 3
+        self.name = cfg["name"]
+
+    def step(self, ctx, i):
+        k = i % self.copies
+        self.dsn.dsn_layer_forward(ctx, self.L, self.xs[k], None if self.gate_driven else self.idx_given, self.ys[k],
+                                   self.ws, idx_out=self.idx_out)
+
+    def decomposed_step(self, ctx, i, mark):
+        """Same path as separate C calls; mark(name) records a CUDA event after each."""
+        d, k = self.dsn, i % self.copies
+        mark("start")
+        if self.gate_driven:
+            d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)
+            mark("gate")
+            d.dsn_route(ctx, self.idx_out, self.B, self.T, self.routing)
+        else:
+            d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)
+        mark("route")
+        d.dsn_sliced_conv(ctx, self.dec_layers[0], self.routing, self.xs[k], self.t1)
+        mark("gemm:conv1_1x1")
+        d.dsn_sliced_conv(ctx, self.dec_layers[1], self.routing, self.t1, self.t2)
+        mark("gemm:conv2_3x3")
+        d.dsn_sliced_conv(ctx, self.dec_layers[2], self.routing, self.t2, self.ys[k])
+        mark("gemm:conv3_1x1")
+
+    def histogram(self):
+        return np.bincount(self.idx_out.cpu().numpy() if self.gate_driven else self.cfg["idx"], minlength=self.T)
+
+    def exec_flops(self, counts):
+        return sum(2 * self.dsn.dsn_executed_macs(counts.tolist(), self.R, ki, ko, K) for ki, ko, K in self.slices)
+
+    def gemm_bytes(self, counts):
+        """Algorithmic bytes of the three GEMM launches: sliced input read once, sliced output written
+        once, each used weight slice read once (bf16)."""
+        total = 0
+        for ki, ko, K in self.slices:
+            for t, n in enumerate(counts):
+                if n:
+                    total += 2 * (int(n) * self.R * (ki[t] + ko[t]) + ki[t] * ko[t] * K * K)
+        return total
+
+    def e2e_io(self):
+        t = self.torch
+        hx = t.from_numpy(self.x_host_bits.copy()).pin_memory()
+        hy = t.empty(self.ys[0].numel(), dtype=t.int16).pin_memory()
+        return hx, hy
+
+    def e2e_step(self, ctx, hx, hy):
+        t = self.torch
+        self.xs[0].view(t.int16).view(-1).copy_(hx.view(-1), non_blocking=True)
+        self.step(ctx, 0)
+        hy.copy_(self.ys[0].view(t.int16).view(-1), non_blocking=True)
+
+    def oracle_sample(self, n):
+        """Times the fp64 oracle on the first n samples (gate + bottleneck chain)."""
+        from oracle import dsn_oracle as O
+        cfg = self.cfg
+        x = cfg["x"][:n]
+        t0 = time.perf_counter()
+        idx, _, _ = O.gate(x.reshape(n, self.R, self.C), cfg["gate_W1"], cfg["gate_W2"])
+        if not self.gate_driven:
+            idx = cfg["idx"][:n]
+        O.route(idx, self.T)
+        O.bottleneck(x, cfg["W1"], cfg["W2"], cfg["W3"], idx, self.widths, mirror_bf16=True)
+        dt = time.perf_counter() - t0
+        flops = sum(2 * O.executed_macs(idx, self.R, ki, ko, K) for ki, ko, K in self.slices)
+        return flops, dt
+
+
+def make_workload(name, dsn, torch, dev, batch=None):
+    import dsn_workloads as wl
+    if name == "cfg2":
+        return Bottleneck(dsn, torch, dev, wl.config2(B=batch or 128), gate_driven=True)
+    if name.startswith("cfg4-stage"):
+        stage = int(name[len("cfg4-stage")])
+        routing = "uniform" if name.endswith("uniform") else "skewed"
+        return Bottleneck(dsn, torch, dev, wl.config4(stage, B=batch or 256, routing=routing), gate_driven=False)
+    raise SystemExit(f"unknown workload {name}")
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """Times the CPU oracle (the only 'reference implementation' this method has) on host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import dsn_workloads as wl
+    from oracle import dsn_oracle as O
+    cfg = wl.config2(B=128)
+    n = 8
+    R, C, T, widths = cfg["H"] * cfg["W"], cfg["C_outer"], cfg["T"], cfg["widths"]
+    full = [C] * T
+    slices = [(full, widths, 1), (widths, widths, 3), (widths, full, 1)]
+
+    def one(i):
+        x = cfg["x"][(i * n) % 128:(i * n) % 128 + n]
+        idx, _, _ = O.gate(x.reshape(n, R, C), cfg["gate_W1"], cfg["gate_W2"])
+        O.route(idx, T)
+        O.bottleneck(x, cfg["W1"], cfg["W2"], cfg["W3"], idx, widths, mirror_bf16=True)
+        return sum(2 * O.executed_macs(idx, R, ki, ko, K) for ki, ko, K in slices)
+
+    for i in range(args.warmup):
+        one(i)
+    flops, t0 = 0, time.perf_counter()
+    for i in range(args.steps):
+        flops += one(i)
+    dt = time.perf_counter() - t0
+    val = flops / dt / 1e12
+    cores = os.cpu_count()
+    print(json.dumps({
+        "impl": "reference", "metric": "sliced_gemm_executed_tflops", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg2 ResNet-50 stage-3 dynamic bottleneck, bf16-valued inputs, 14x14, 14 widths",
+                   "sample": f"{n} samples per step"},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{n} of 128 samples per step, {args.steps} steps"},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# --------------------------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="dsn", choices=["dsn", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2109_10060_b200.build import build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    import paper_2109_10060_b200 as dsn
+    torch.cuda.set_device(local_rank)
+    dev = torch.device(f"cuda:{local_rank}")
+    ctx = dsn.Context(local_rank)
+    peaks = load_peaks()
+
+    wlk = make_workload(args.workload, dsn, torch, dev, args.batch)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        wlk.step(ctx, i)
+    barrier()
+    code, detail = ctx.get_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
+    counts = wlk.histogram()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        wlk.step(ctx, i)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+
+    # per-kernel durations: same kernels, one C call per step of the path, events between calls
+    names, acc = [], {}
+    dec_steps = min(args.steps, 50)
+    for i in range(3 + dec_steps):
+        evs = []
+        def mark(n):
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record(stream)
+            evs.append((n, ev))
+        wlk.decomposed_step(ctx, i, mark)
+        torch.cuda.synchronize()
+        if i >= 3:
+            for (n0, a), (n1, b) in zip(evs[:-1], evs[1:]):
+                acc.setdefault(n1, []).append(a.elapsed_time(b))
+    clocks = sampler.stop()
+
+    # end to end: batch starts and ends in pinned host memory
+    hx, hy = wlk.e2e_io()
+    for _ in range(3):
+        wlk.e2e_step(ctx, hx, hy)
+    barrier()
+    e2e_steps = min(args.steps, 20)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        wlk.e2e_step(ctx, hx, hy)
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+    code, detail = ctx.get_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    t2 = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    ms_e2e = float(t2.item())
+    flops = wlk.exec_flops(counts)
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    e2e_value = world * flops / (ms_e2e * 1e-3) / 1e12
+
+    gemm_ms = sum(float(np.mean(v)) for k, v in acc.items() if k.startswith("gemm:"))
+    gemm_bytes = wlk.gemm_bytes(counts)
+    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
+    per_kernel = {k: round(float(np.mean(v)) * 1e3, 2) for k, v in acc.items()}
+    roofline = {"bound": "hbm", "kernel": "gemm_bf16_kernel (3 launches per step: conv1, conv2, conv3)",
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "peak_source": peaks["source"] + " copy bandwidth, burst", "traffic": None,
+                "algorithmic_bytes_per_step": gemm_bytes, "us_per_step": round(gemm_ms * 1e3, 2),
+                "executed_tflops": flops / (gemm_ms * 1e-3) / 1e12,
+                "frac_of_bf16_peak_burst": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+
+    if rank != 0:
+        return
+    out = {
+        "metric": "sliced_gemm_executed_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wlk.name}: batch {wlk.B} per GPU, gate-driven routing" if wlk.gate_driven
+                   else f"{wlk.name}: batch {wlk.B} per GPU, routing {wlk.cfg['routing']}",
+                   "path": "gate -> route -> 1x1 -> 3x3 -> 1x1 -> input order (dsn_layer_forward)",
+                   "l2": f"inputs and outputs rotate over {wlk.copies} buffers (> 126 MB L2)",
+                   "routing_histogram": counts.tolist(), "parallelism": f"batch shards x{world}, no collective"},
+        "samples_per_s": world * wlk.B / (ms_step * 1e-3),
+        "pct_bf16_peak_burst": 100 * value / world / peaks["bf16_tflops"],
+        "pct_bf16_peak_nominal": 100 * value / world / NOMINAL_BF16_TFLOPS,
+        "kernel_us": per_kernel,
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(hx.numel() * 2),
+                "d2h_bytes_per_step": int(hy.numel() * 2), "ms_per_step": ms_e2e},
+        "gpu_launches": wlk.kernels_per_step * args.steps,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        n = 16
+        f_cpu, dt = wlk.oracle_sample(n)
+        out["cpu_baseline"] = {"value": f_cpu / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                               "sample": f"first {n} of {wlk.B} samples, gate + route + bottleneck, fp64 numpy, {dt:.1f} s"}
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -10,6 +10,23 @@ from gpu_util import (DEV, SENTINEL, assert_tail_untouched, check_status, down, 
 
 pytestmark = pytest.mark.gpu
 TOL_BF16 = 5e-3
+# Chains store bf16 between layers.  Where the device's fp32 accumulator and the oracle's fp64 sum fall on
+# different sides of a bf16 rounding boundary the stored values differ by one ulp (<= 2^-7 of the value);
+# downstream layers then move a few final outputs across a boundary as well.  A chained output may
+# therefore sit one output ulp (<= 7.8e-3 of max|ref|) from the mirrored oracle, while the mean error
+# stays far below that because such flips are rare.
+TOL_CHAIN_MAX = 1e-2
+TOL_CHAIN_MEAN = 2e-4
+
+
+def chain_mean_error(got, ref, idx, k_out, T):
+    worst = 0.0
+    for t in range(T):
+        sel = np.nonzero(np.asarray(idx) == t)[0]
+        if len(sel):
+            g, r = got[sel][..., :k_out[t]], ref[sel][..., :k_out[t]]
+            worst = max(worst, float(np.mean(np.abs(g - r)) / np.max(np.abs(r))))
+    return worst
 
 
 @pytest.fixture(scope="module")
@@ -132,7 +149,8 @@ def test_layer_forward_bottleneck_with_gate(dsn, ctx):
     assert np.all((idx_used >= 0) & (idx_used < cfg["T"]))
     _, _, ref = O.bottleneck(cfg["x"], cfg["W1"], cfg["W2"], cfg["W3"], idx_used, cfg["widths"], mirror_bf16=True)
     errs = group_errors(got, ref, idx_used, [C] * cfg["T"], cfg["T"])
-    assert max(errs.values()) <= TOL_BF16, errs
+    assert max(errs.values()) <= TOL_CHAIN_MAX, errs
+    assert chain_mean_error(got, ref, idx_used, [C] * cfg["T"], cfg["T"]) <= TOL_CHAIN_MEAN
     # routing arrays left in the workspace are the stable grouping of the gate's choice
     assert r_out.B == B and r_out.G == cfg["T"]
     base = ws.data_ptr()
@@ -155,7 +173,8 @@ def test_layer_forward_bottleneck_resnet_stages(dsn, ctx, stage, B, routing):
     np.testing.assert_array_equal(idx_gpu, cfg["idx"])
     _, _, ref = O.bottleneck(cfg["x"], cfg["W1"], cfg["W2"], cfg["W3"], cfg["idx"], cfg["widths"], mirror_bf16=True)
     errs = group_errors(got, ref, cfg["idx"], [outer] * cfg["T"], cfg["T"])
-    assert max(errs.values()) <= TOL_BF16, errs
+    assert max(errs.values()) <= TOL_CHAIN_MAX, errs
+    assert chain_mean_error(got, ref, cfg["idx"], [outer] * cfg["T"], cfg["T"]) <= TOL_CHAIN_MEAN
 
 
 def test_layer_forward_vit_mlp_and_config1(dsn, ctx):
@@ -181,7 +200,8 @@ def test_layer_forward_vit_mlp_and_config1(dsn, ctx):
     _, ref = O.vit_mlp(cfg["x"], cfg["Wfc1"], cfg["Wfc2"], idx_used, paths, mirror_bf16=True)
     got = down(y)
     errs = group_errors(got, ref, idx_used, ko2, T)
-    assert max(errs.values()) <= TOL_BF16, errs
+    assert max(errs.values()) <= TOL_CHAIN_MAX, errs
+    assert chain_mean_error(got, ref, idx_used, ko2, T) <= TOL_CHAIN_MEAN
     assert_tail_untouched(got, idx_used, ko2)
 
     # config 1: single fp32 layer, gate bypassed
