@@ -162,6 +162,26 @@ size_t dsn_gate_workspace_bytes(const dsn_gate_desc* g);
 int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out,
              float* logits_out, void* workspace, size_t ws_bytes, void* stream);
 
+/* The same gate for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience).  Typical such callers: a serving loop that must never enter
+ * the CUDA allocator once it is running, a plug-in that is handed only its input and output
+ * buffers, code running while the process's memory pool is fully handed out.  The pooling scratch
+ * lives in a fixed 4 MiB array inside the library image (every GPU that loads the library keeps it
+ * until the process exits), so the call takes no workspace and performs no allocation of any kind.
+ *   - Limit: B * splits * c_valid <= 1,048,576 floats, where splits (1..64) is the row-band count
+ *     the gate picks for this GPU; larger problems return DSN_ERR_WORKSPACE and launch nothing.
+ *     All BASELINE workloads fit (128 x 5 x 1024, 1024 x 1 x 768).
+ *   - The context's device must be the current device (else DSN_ERR_INVALID_ARG).
+ *   - The first call on a device looks up the array's device address (a synchronous runtime
+ *     query); make that first call before starting any stream capture.
+ *   - All calls on one GPU share the array and it keeps the previous call's contents.  Nothing has
+ *     to start at zero (each call overwrites every value it later reads), but two calls that
+ *     overlap on the GPU (different streams, or different contexts of one process) race on it:
+ *     keep calls to this entry point ordered on one stream per GPU.
+ * Arguments and results are those of dsn_gate. */
+int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out,
+                    float* logits_out, void* stream);
+
 /* ---- routing (stable grouping by path index; one-hot routing of Sec. 3.1) -------------- */
 /* idx: device [B], values in [0, T).  Fills out->counts/offsets/perm/inv_perm (device arrays the
  * caller allocated, G = T, B as given); integer-exact and deterministic.  A value outside

@@ -25,7 +25,7 @@ MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
 
 EXPORTS = [
     "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_widths_from_ratios",
-    "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_route", "dsn_permute_rows",
+    "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_route", "dsn_permute_rows",
     "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
 ]
@@ -93,6 +93,7 @@ def load_library():
     lib.dsn_gate_workspace_bytes.argtypes = [C.POINTER(GateDesc)]
     lib.dsn_gate_workspace_bytes.restype = sz
     lib.dsn_gate.argtypes = [vp, C.POINTER(GateDesc), vp, vp, vp, vp, sz, vp]
+    lib.dsn_gate_static.argtypes = [vp, C.POINTER(GateDesc), vp, vp, vp, vp]
     lib.dsn_route.argtypes = [vp, vp, i32, i32, C.POINTER(Routing), vp]
     lib.dsn_permute_rows.argtypes = [vp, C.POINTER(Routing), i32, i32, i32, C.POINTER(i32), vp, i64, vp, i64, i32, vp]
     lib.dsn_linear_workspace_bytes.argtypes = [C.POINTER(LinearDesc), i32]
@@ -225,6 +226,15 @@ def dsn_gate(ctx: Context, g: GateDesc, x, idx_out, logits_out=None, workspace=N
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(ctx.lib.dsn_gate(ctx.handle, C.byref(g), _ptr(x), _ptr(idx_out), _ptr(logits_out), _ptr(workspace),
                             ws_bytes, _stream_handle(stream)), "dsn_gate")
+
+
+def dsn_gate_static(ctx: Context, g: GateDesc, x, idx_out, logits_out=None, stream=None):
+    """dsn_gate without a workspace: for callers that may not allocate device memory (a serving loop
+    that must stay out of the allocator, a plug-in that only receives its inputs and outputs).  The
+    scratch is a fixed 4 MiB array inside the library, shared by all calls on a GPU, so calls must not
+    overlap on the device, and problems beyond 1,048,576 scratch floats raise ERR_WORKSPACE."""
+    _check(ctx.lib.dsn_gate_static(ctx.handle, C.byref(g), _ptr(x), _ptr(idx_out), _ptr(logits_out),
+                                   _stream_handle(stream)), "dsn_gate_static")
 
 
 def dsn_route(ctx: Context, idx, B: int, T: int, routing: Routing, stream=None):

@@ -190,3 +190,61 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
                                                                   logits_out, status);
   return cudaGetLastError();
 }
+
+// ------------------------------------------------------------------------------------------------
+// dsn_gate_static: the gate for callers that cannot allocate device memory.
+//
+// The pooling partial sums normally live in a workspace the caller allocates.  Some callers have no
+// allocator to ask: code running inside a region where cudaMalloc is forbidden or would stall the
+// device (a latency-critical serving loop that must never touch the allocator, a plug-in that is
+// handed only its input and output buffers, a process whose memory pool has been handed out in
+// full).  For them the same kernels run with their scratch in a fixed array that is part of the
+// loaded library image: 4 MiB per GPU that loads the library, held until the process exits.
+// ------------------------------------------------------------------------------------------------
+#define DSN_GATE_STATIC_MAX_FLOATS (1u << 20)
+
+static __device__ __align__(256) float g_gate_static_scratch[DSN_GATE_STATIC_MAX_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices];  // device address of the array, per device, 0 = not looked up yet
+
+// The array's name is only a host-side handle; kernels need its device address, which is looked up
+// once per device while that device is current.
+int static_scratch_address(int device, float** out) {
+  if (device < 0 || device >= kMaxDevices) return DSN_ERR_INVALID_ARG;
+  int current = -1;
+  if (cudaGetDevice(&current) != cudaSuccess) return DSN_ERR_CUDA;
+  if (current != device) return DSN_ERR_INVALID_ARG;
+  if (!g_static_scratch_ptr[device]) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_gate_static_scratch) != cudaSuccess || !ptr)
+      return DSN_ERR_CUDA;
+    g_static_scratch_ptr[device] = ptr;
+  }
+  *out = g_static_scratch_ptr[device];
+  return DSN_OK;
+}
+}  // namespace
+
+extern "C" int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out,
+                               float* logits_out, void* stream) {
+  if (!ctx || !g || !x || !idx_out || !g->W1 || !g->W2) return DSN_ERR_INVALID_ARG;
+  if (g->dtype != DSN_BF16 && g->dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
+  if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
+      g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
+    return DSN_ERR_INVALID_ARG;
+  if ((size_t)4 * kSB * ((size_t)g->c_valid + g->C_mlp + g->T) > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  if (g->B == 0) return DSN_OK;
+  const int splits = dsn_gate_splits(*g, ctx->sm_count);
+  const size_t need = (size_t)g->B * splits * g->c_valid;
+  if (need > DSN_GATE_STATIC_MAX_FLOATS) return DSN_ERR_WORKSPACE;  // batch too large for the fixed scratch
+  float* scratch = nullptr;
+  const int e = static_scratch_address(ctx->device, &scratch);
+  if (e != DSN_OK) return e;
+  // every partial sum the second kernel reads is overwritten by the first one, so nothing needs clearing
+  if (dsn_launch_gate(*g, x, idx_out, logits_out, scratch, splits, ctx->d_status,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
