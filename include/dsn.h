@@ -168,9 +168,10 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
  * buffers, code running while the process's memory pool is fully handed out.  The pooling scratch
  * lives in a fixed 4 MiB array inside the library image (every GPU that loads the library keeps it
  * until the process exits), so the call takes no workspace and performs no allocation of any kind.
- *   - Limit: B * splits * c_valid <= 1,048,576 floats, where splits (1..64) is the row-band count
- *     the gate picks for this GPU; larger problems return DSN_ERR_WORKSPACE and launch nothing.
- *     All BASELINE workloads fit (128 x 5 x 1024, 1024 x 1 x 768).
+ *   - Limit: B * (splits * c_valid + C_mlp) <= 1,048,576 floats, where splits (1..64) is the
+ *     row-band count the gate picks for this GPU; larger problems return DSN_ERR_WORKSPACE and
+ *     launch nothing.  The ResNet-50 and ViT workloads fit (128 x (5 x 1024 + 128),
+ *     1024 x (1 x 768 + 128)).
  *   - The context's device must be the current device (else DSN_ERR_INVALID_ARG).
  *   - The first call on a device looks up the array's device address (a synchronous runtime
  *     query); make that first call before starting any stream capture.

@@ -162,25 +162,26 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     p.k_in[t] = (int16_t)c.k_in[t];
     p.k_out[t] = (int16_t)c.k_out[t];
   }
-  const size_t smem = dsn_gemm_smem_bytes(g.BN, g.stages);
+  const size_t smem = dsn_gemm_smem_bytes(g.BN, g.stages, r->G);
 
-  // distinct k_in values, DSN_GEMM_MAX_MAPS per launch
+  // one tensor-map pair per distinct slice (k_in, k_out), DSN_GEMM_MAX_MAPS pairs per launch
   int done[DSN_MAX_SLICES];
   memset(done, 0, sizeof(done));
   int remaining = c.T;
   while (remaining > 0) {
     int nmaps = 0;
-    int map_k[DSN_GEMM_MAX_MAPS];
+    int map_k[DSN_GEMM_MAX_MAPS], map_n[DSN_GEMM_MAX_MAPS];
     memset(p.map_id, 0xFF, sizeof(p.map_id));
     for (int t = 0; t < c.T; ++t) {
       if (done[t]) continue;
       int id = -1;
       for (int m = 0; m < nmaps; ++m)
-        if (map_k[m] == c.k_in[t]) id = m;
+        if (map_k[m] == c.k_in[t] && map_n[m] == c.k_out[t]) id = m;
       if (id < 0) {
         if (nmaps == DSN_GEMM_MAX_MAPS) continue;  // next launch
         id = nmaps++;
         map_k[id] = c.k_in[t];
+        map_n[id] = c.k_out[t];
       }
       p.map_id[t] = (uint8_t)id;
       done[t] = 1;
@@ -202,7 +203,7 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
         e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
       }
       if (e) return e;
-      const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)c.C_out};
+      const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)map_n[m]};  // rows beyond k_out: zeros, not fetched
       const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
       const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)g.BN};
       e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
@@ -271,7 +272,7 @@ int check_gate(const dsn_gate_desc* g) {
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * 4 * ((size_t)g->c_valid + g->C_mlp + g->T) > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  if ((size_t)4 * 4 * (size_t)g->c_valid > 200 * 1024) return DSN_ERR_UNSUPPORTED;
   return DSN_OK;
 }
 
@@ -427,7 +428,7 @@ size_t dsn_gate_workspace_bytes(const dsn_gate_desc* g) {
   // the split count depends on the SM count; size for the largest count the launcher can pick
   int splits = g->R / 8 > 0 ? g->R / 8 : 1;
   if (splits > 64) splits = 64;
-  return align_up((size_t)g->B * splits * g->c_valid * sizeof(float), 256) + 256;
+  return align_up(((size_t)g->B * splits * g->c_valid + (size_t)g->B * g->C_mlp) * sizeof(float), 256) + 256;
 }
 
 int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out, float* logits_out,
@@ -437,7 +438,7 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
   if (e) return e;
   if (g->B == 0) return DSN_OK;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
-  const size_t need = (size_t)g->B * splits * g->c_valid * sizeof(float);
+  const size_t need = ((size_t)g->B * splits * g->c_valid + (size_t)g->B * g->C_mlp) * sizeof(float);
   if (!workspace || ws_bytes < need) return DSN_ERR_WORKSPACE;
   if (!aligned16(workspace)) return DSN_ERR_ALIGNMENT;
   if (dsn_launch_gate(*g, x, idx_out, logits_out, static_cast<float*>(workspace), splits, ctx->d_status,
@@ -529,7 +530,6 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
   r.perm = reinterpret_cast<int32_t*>(ws + pl.off_perm);
   r.inv_perm = reinterpret_cast<int32_t*>(ws + pl.off_inv);
   r.group_slice = nullptr;
-  const void* src = x;
   for (int j = 0; j < L->n_layers; ++j) {
     LayerCall& c = calls[j];
     layer_call_of(L, j, c);
@@ -545,7 +545,6 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     e = validate_call(c, &r, in, out);
     if (e) return e;
   }
-  (void)src;
 
   const int32_t* idx = idx_in;
   if (L->gate) {

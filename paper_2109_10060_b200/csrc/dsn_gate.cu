@@ -1,19 +1,23 @@
 // Gate routing head (Sec. 3.5): average pooling over the R positions of each sample, a two-layer
 // MLP (ReLU between), and the index of the first maximum score.
 //
-// Kernel 1 (HBM-bound): grid (splits, B).  A CTA streams a contiguous band of rows of one sample
-// with 16-byte loads (consecutive threads read consecutive 16 bytes of a row) and accumulates in
-// fp32 registers; its column sums go to partial[b][split][c].  No atomics, so sums are
-// reproducible run to run.
-// Kernel 2 (tiny, plain FMA): a CTA owns kSB samples; it folds the partial sums, scales by 1/R,
-// and evaluates both FC layers with one warp per output unit (lanes stride the reduction,
-// shuffle reduce), then one thread per sample takes the arg-max with a strict '>' scan.
+// Kernel 1 (HBM-bound): grid (splits, B), 512 threads.  A CTA streams a contiguous band of rows of
+// one sample: consecutive threads read consecutive 16 bytes of a row, the CTA's row groups walk
+// different rows, four loads are in flight per thread; fp32 accumulation in registers, one
+// shared-memory reduction across the row groups, column sums to partial[b][split][c].  No atomics,
+// so sums are reproducible run to run.
+// Kernel 2 (L2-bound, plain FMA): grid (B/4, C_mlp/16).  A CTA folds the partial sums of 4 samples
+// (scaled by 1/R) into shared memory and computes 16 hidden units for them, one warp per two
+// units with 16-byte weight loads and a shuffle reduction; ReLU; hid[b][j] to scratch.
+// Kernel 3 (tiny): one warp per sample evaluates the T scores and takes the arg-max with a strict
+// '>' scan in ascending path order (ties keep the lowest index).
 #include "dsn_internal.cuh"
 
 namespace {
 
-constexpr int kSB = 4;            // samples per CTA in the MLP kernel
-constexpr int kPoolThreads = 128;
+constexpr int kSB = 4;             // samples per CTA in the hidden-layer kernel
+constexpr int kJB = 16;            // hidden units per CTA in the hidden-layer kernel
+constexpr int kPoolThreads = 512;
 constexpr int kMlpThreads = 256;
 
 __device__ __forceinline__ void add8(float (&acc)[8], const uint4& v) {
@@ -25,46 +29,61 @@ __device__ __forceinline__ void add8(float (&acc)[8], const uint4& v) {
   }
 }
 
-// bf16 input, c_valid % 8 == 0, ldx % 8 == 0, x 16-byte aligned
+// bf16 input, c_valid % 8 == 0, ldx % 8 == 0, x 16-byte aligned.  CT = column threads (power of two).
 __global__ void __launch_bounds__(kPoolThreads)
-pool_bf16_vec_kernel(const __nv_bfloat16* __restrict__ x, int R, int64_t ldx, int c_valid, int splits,
+pool_bf16_vec_kernel(const __nv_bfloat16* __restrict__ x, int R, int64_t ldx, int c_valid, int splits, int CT,
                      float* __restrict__ partial) {
+  __shared__ float red[kPoolThreads * 8];
   const int b = blockIdx.y, sp = blockIdx.x;
   const int r0 = (int)(((int64_t)R * sp) / splits), r1 = (int)(((int64_t)R * (sp + 1)) / splits);
   const int nvec = c_valid >> 3;
+  const int tx = threadIdx.x & (CT - 1), ty = threadIdx.x / CT, RG = kPoolThreads / CT;
   const __nv_bfloat16* xb = x + (int64_t)b * R * ldx;
   float* out = partial + ((int64_t)b * splits + sp) * c_valid;
-  for (int v = threadIdx.x; v < nvec; v += kPoolThreads) {
+  const int64_t stride = ldx >> 3;  // row pitch in uint4
+  for (int v0 = 0; v0 < nvec; v0 += CT) {
+    const int v = v0 + tx;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    const uint4* col = reinterpret_cast<const uint4*>(xb + (int64_t)r0 * ldx) + v;
-    const int64_t stride = ldx >> 3;  // in uint4
-    int r = r0;
-    for (; r + 4 <= r1; r += 4) {     // four independent loads in flight per thread
-      const uint4 a0 = __ldg(col), a1 = __ldg(col + stride), a2 = __ldg(col + 2 * stride),
-                  a3 = __ldg(col + 3 * stride);
-      add8(acc, a0); add8(acc, a1); add8(acc, a2); add8(acc, a3);
-      col += 4 * stride;
+    if (v < nvec) {
+      const uint4* col = reinterpret_cast<const uint4*>(xb) + v;
+      int r = r0 + ty;
+      for (; r + 3 * RG < r1; r += 4 * RG) {  // four independent loads in flight per thread
+        const uint4 a0 = __ldg(col + (int64_t)r * stride), a1 = __ldg(col + (int64_t)(r + RG) * stride),
+                    a2 = __ldg(col + (int64_t)(r + 2 * RG) * stride), a3 = __ldg(col + (int64_t)(r + 3 * RG) * stride);
+        add8(acc, a0); add8(acc, a1); add8(acc, a2); add8(acc, a3);
+      }
+      for (; r < r1; r += RG) add8(acc, __ldg(col + (int64_t)r * stride));
     }
-    for (; r < r1; ++r) {
-      add8(acc, __ldg(col));
-      col += stride;
+    float4* mine = reinterpret_cast<float4*>(red + (size_t)threadIdx.x * 8);
+    mine[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    mine[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    __syncthreads();
+    // one thread per (column vector, half): sum over the row groups in a fixed order
+    if (threadIdx.x < 2 * CT) {
+      const int cx = threadIdx.x >> 1, half = threadIdx.x & 1;
+      if (v0 + cx < nvec) {
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < RG; ++g) {
+          const float4 t = reinterpret_cast<const float4*>(red + (size_t)(g * CT + cx) * 8)[half];
+          sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+        }
+        reinterpret_cast<float4*>(out + 8 * (v0 + cx))[half] = sum;
+      }
     }
-    float4* o = reinterpret_cast<float4*>(out + 8 * v);
-    o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    o[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    __syncthreads();
   }
 }
 
 // any dtype / any width: one channel per thread
 template <typename Tin>
-__global__ void __launch_bounds__(kPoolThreads)
+__global__ void __launch_bounds__(128)
 pool_scalar_kernel(const Tin* __restrict__ x, int R, int64_t ldx, int c_valid, int splits,
                    float* __restrict__ partial) {
   const int b = blockIdx.y, sp = blockIdx.x;
   const int r0 = (int)(((int64_t)R * sp) / splits), r1 = (int)(((int64_t)R * (sp + 1)) / splits);
   const Tin* xb = x + (int64_t)b * R * ldx;
   float* out = partial + ((int64_t)b * splits + sp) * c_valid;
-  for (int c = threadIdx.x; c < c_valid; c += kPoolThreads) {
+  for (int c = threadIdx.x; c < c_valid; c += 128) {
     float acc = 0.f;
     for (int r = r0; r < r1; ++r) acc += (float)xb[(int64_t)r * ldx + c];
     out[c] = acc;
@@ -72,18 +91,12 @@ pool_scalar_kernel(const Tin* __restrict__ x, int R, int64_t ldx, int c_valid, i
 }
 
 __global__ void __launch_bounds__(kMlpThreads)
-gate_mlp_kernel(const float* __restrict__ partial, int splits, int B, int R, int C_full, int c_valid, int C_mlp,
-                int T, const float* __restrict__ W1, const float* __restrict__ b1,
-                const float* __restrict__ W2, const float* __restrict__ b2, int32_t* __restrict__ idx_out,
-                float* __restrict__ logits_out, int32_t* status) {
-  extern __shared__ float smem[];
-  float* pooled = smem;                        // [kSB][c_valid]
-  float* hid = pooled + kSB * c_valid;         // [kSB][C_mlp]
-  float* logit = hid + kSB * C_mlp;            // [kSB][T]
-  const int b0 = blockIdx.x * kSB;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kMlpThreads / 32;
+gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, int C_full, int c_valid, int C_mlp,
+                   const float* __restrict__ W1, const float* __restrict__ b1, float* __restrict__ hid) {
+  extern __shared__ __align__(16) float pooled[];  // [kSB][c_valid]
+  const int b0 = blockIdx.x * kSB, j0 = blockIdx.y * kJB;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_r = 1.0f / (float)R;
-
   for (int e = tid; e < kSB * c_valid; e += kMlpThreads) {
     const int s = e / c_valid, c = e - s * c_valid;
     float acc = 0.f;
@@ -94,58 +107,77 @@ gate_mlp_kernel(const float* __restrict__ partial, int splits, int B, int R, int
     pooled[e] = acc * inv_r;
   }
   __syncthreads();
-
-  for (int j = warp; j < C_mlp; j += nwarp) {
+  const bool vec = (c_valid % 4 == 0) && (C_full % 4 == 0) && ((reinterpret_cast<uintptr_t>(W1) & 15) == 0);
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int j = j0 + 2 * warp + u;
+    if (j >= C_mlp) break;  // warp-uniform
     float acc[kSB];
 #pragma unroll
     for (int s = 0; s < kSB; ++s) acc[s] = 0.f;
     const float* w = W1 + (int64_t)j * C_full;
-    for (int c = lane; c < c_valid; c += 32) {
-      const float wv = __ldg(w + c);
+    if (vec) {
+      const float4* w4 = reinterpret_cast<const float4*>(w);
+      const int n4 = c_valid >> 2;
+#pragma unroll 4
+      for (int c = lane; c < n4; c += 32) {
+        const float4 wv = __ldg(w4 + c);
 #pragma unroll
-      for (int s = 0; s < kSB; ++s) acc[s] = fmaf(wv, pooled[s * c_valid + c], acc[s]);
+        for (int s = 0; s < kSB; ++s) {
+          const float4 pv = reinterpret_cast<const float4*>(pooled + s * c_valid)[c];
+          acc[s] = fmaf(wv.x, pv.x, acc[s]);
+          acc[s] = fmaf(wv.y, pv.y, acc[s]);
+          acc[s] = fmaf(wv.z, pv.z, acc[s]);
+          acc[s] = fmaf(wv.w, pv.w, acc[s]);
+        }
+      }
+    } else {
+      for (int c = lane; c < c_valid; c += 32) {
+        const float wv = __ldg(w + c);
+#pragma unroll
+        for (int s = 0; s < kSB; ++s) acc[s] = fmaf(wv, pooled[s * c_valid + c], acc[s]);
+      }
     }
 #pragma unroll
     for (int s = 0; s < kSB; ++s) {
       float v = acc[s];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) hid[s * C_mlp + j] = fmaxf(v + (b1 ? b1[j] : 0.f), 0.f);
+      if (lane == 0 && b0 + s < B) hid[(int64_t)(b0 + s) * C_mlp + j] = fmaxf(v + (b1 ? b1[j] : 0.f), 0.f);
     }
   }
-  __syncthreads();
+}
 
-  for (int t = warp; t < T; t += nwarp) {
-    float acc[kSB];
-#pragma unroll
-    for (int s = 0; s < kSB; ++s) acc[s] = 0.f;
+__global__ void __launch_bounds__(kMlpThreads)
+gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const float* __restrict__ W2,
+                  const float* __restrict__ b2, int32_t* __restrict__ idx_out, float* __restrict__ logits_out,
+                  int32_t* status) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.x * (kMlpThreads / 32) + warp;
+  if (b >= B) return;
+  const float* h = hid + (int64_t)b * C_mlp;
+  int best = 0, nonfinite = 0;
+  float best_v = 0.f;
+  for (int t = 0; t < T; ++t) {
     const float* w = W2 + (int64_t)t * C_mlp;
-    for (int j = lane; j < C_mlp; j += 32) {
-      const float wv = __ldg(w + j);
+    float v = 0.f;
+    for (int j = lane; j < C_mlp; j += 32) v = fmaf(__ldg(w + j), h[j], v);
 #pragma unroll
-      for (int s = 0; s < kSB; ++s) acc[s] = fmaf(wv, hid[s * C_mlp + j], acc[s]);
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    v += b2 ? b2[t] : 0.f;
+    if (!isfinite(v)) ++nonfinite;
+    if (t == 0) {
+      best_v = v;
+    } else if (v > best_v) {  // strict: ties keep the lower index
+      best = t;
+      best_v = v;
     }
-#pragma unroll
-    for (int s = 0; s < kSB; ++s) {
-      float v = acc[s];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) logit[s * T + t] = v + (b2 ? b2[t] : 0.f);
-    }
+    if (lane == 0 && logits_out) logits_out[(int64_t)b * T + t] = v;
   }
-  __syncthreads();
-
-  if (tid < kSB && b0 + tid < B) {
-    const float* l = logit + tid * T;
-    int best = 0, nonfinite = 0;
-    for (int t = 0; t < T; ++t) {
-      if (!isfinite(l[t])) ++nonfinite;
-      if (t > 0 && l[t] > l[best]) best = t;
-      if (logits_out) logits_out[(int64_t)(b0 + tid) * T + t] = l[t];
-    }
-    idx_out[b0 + tid] = best;
+  if (lane == 0) {
+    idx_out[b] = best;
     if (nonfinite) {
-      dsn_set_status(status, DSN_ERR_NONFINITE, b0 + tid);
+      dsn_set_status(status, DSN_ERR_NONFINITE, b);
       if (status) atomicAdd(status + 2, nonfinite);
     }
   }
@@ -154,7 +186,7 @@ gate_mlp_kernel(const float* __restrict__ partial, int splits, int B, int R, int
 }  // namespace
 
 int dsn_gate_splits(const dsn_gate_desc& g, int sm_count) {
-  // enough CTAs to fill the machine about four times over, at least 8 rows per CTA
+  // about four 512-thread CTAs per SM, at least 8 rows per CTA
   int want = (4 * sm_count + g.B - 1) / g.B;
   int max_by_rows = g.R / 8 > 0 ? g.R / 8 : 1;
   int s = want < max_by_rows ? want : max_by_rows;
@@ -163,31 +195,41 @@ int dsn_gate_splits(const dsn_gate_desc& g, int sm_count) {
   return s;
 }
 
+// scratch = partial[B][splits][c_valid] followed by hid[B][C_mlp] (floats)
 cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_out, float* logits_out,
                             float* partial, int splits, int32_t* status, cudaStream_t s) {
   dim3 grid(splits, g.B);
+  float* hid = partial + (size_t)g.B * splits * g.c_valid;
   const bool vec = g.dtype == DSN_BF16 && (g.c_valid % 8 == 0) && (g.ldx % 8 == 0) &&
                    ((reinterpret_cast<uintptr_t>(x) & 15) == 0);
   if (vec) {
+    const int nvec = g.c_valid / 8;
+    int CT = 8;
+    while (CT < nvec && CT < 128) CT <<= 1;
     pool_bf16_vec_kernel<<<grid, kPoolThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), g.R, g.ldx,
-                                                        g.c_valid, splits, partial);
+                                                        g.c_valid, splits, CT, partial);
   } else if (g.dtype == DSN_BF16) {
-    pool_scalar_kernel<__nv_bfloat16><<<grid, kPoolThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), g.R,
-                                                                    g.ldx, g.c_valid, splits, partial);
+    pool_scalar_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(static_cast<const __nv_bfloat16*>(x), g.R, g.ldx,
+                                                           g.c_valid, splits, partial);
   } else {
-    pool_scalar_kernel<float><<<grid, kPoolThreads, 0, s>>>(static_cast<const float*>(x), g.R, g.ldx, g.c_valid,
-                                                            splits, partial);
+    pool_scalar_kernel<float><<<grid, 128, 0, s>>>(static_cast<const float*>(x), g.R, g.ldx, g.c_valid, splits,
+                                                   partial);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const size_t smem = sizeof(float) * (size_t)kSB * (g.c_valid + g.C_mlp + g.T);
+  const size_t smem = sizeof(float) * (size_t)kSB * g.c_valid;
   if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(gate_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(gate_hidden_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  gate_mlp_kernel<<<(g.B + kSB - 1) / kSB, kMlpThreads, smem, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid,
-                                                                  g.C_mlp, g.T, g.W1, g.b1, g.W2, g.b2, idx_out,
-                                                                  logits_out, status);
+  dim3 hgrid((g.B + kSB - 1) / kSB, (g.C_mlp + kJB - 1) / kJB);
+  gate_hidden_kernel<<<hgrid, kMlpThreads, smem, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp, g.W1,
+                                                      g.b1, hid);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int per_cta = kMlpThreads / 32;
+  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, 0, s>>>(hid, g.B, g.C_mlp, g.T, g.W2, g.b2, idx_out,
+                                                                         logits_out, status);
   return cudaGetLastError();
 }
 
@@ -234,15 +276,16 @@ extern "C" int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void*
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * kSB * ((size_t)g->c_valid + g->C_mlp + g->T) > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  if ((size_t)4 * kSB * (size_t)g->c_valid > 200 * 1024) return DSN_ERR_UNSUPPORTED;
   if (g->B == 0) return DSN_OK;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
-  const size_t need = (size_t)g->B * splits * g->c_valid;
+  const size_t need = (size_t)g->B * splits * g->c_valid + (size_t)g->B * g->C_mlp;
   if (need > DSN_GATE_STATIC_MAX_FLOATS) return DSN_ERR_WORKSPACE;  // batch too large for the fixed scratch
   float* scratch = nullptr;
   const int e = static_scratch_address(ctx->device, &scratch);
   if (e != DSN_OK) return e;
-  // every partial sum the second kernel reads is overwritten by the first one, so nothing needs clearing
+  // every scratch value a later kernel reads is overwritten by an earlier one of the same call, so
+  // nothing needs clearing
   if (dsn_launch_gate(*g, x, idx_out, logits_out, scratch, splits, ctx->d_status,
                       static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;

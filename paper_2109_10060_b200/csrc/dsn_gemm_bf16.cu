@@ -8,16 +8,19 @@
 // tile of tap (r, s) is the output tile's pixel rectangle shifted by (r - pad, s - pad); the TMA
 // unit zero-fills what falls outside the image, which is the convolution's zero padding.
 //
-// Operands are read in place.  Every distinct k_in has its own pair of tensor maps whose
-// innermost extent is k_in but whose strides are those of the full tensors, so the channels
-// beyond the slice arrive in shared memory as zeros and are never multiplied.
+// Operands are read in place.  Every distinct slice (k_in, k_out) has its own pair of tensor maps
+// whose extents are the slice's (k_in channels; k_out weight rows) but whose strides are those of
+// the full tensors, so everything beyond the slice arrives in shared memory as zeros: it is never
+// fetched from L2 and never multiplied.
 //
 // Structure of a CTA (persistent, one per SM, 192 threads):
 //   warp 0      one lane issues the TMA loads into a ring of shared-memory stages
 //   warp 1      one lane issues tcgen05.mma (M = 128, N = 16..256, K = 16) into a TMEM accumulator;
 //               two accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
-//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), bias / activation,
-//               bf16 rounding, stores to the grouped or the input-order (scattered) output
+//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), bias / activation, bf16
+//               rounding, a 32-row x 128-byte transpose through swizzled shared memory, then
+//               stores in which eight lanes write one contiguous 128-byte piece of an output row
+//               (grouped or input-order / scattered rows alike)
 // Every mbarrier wait is bounded; on a timeout the CTA records DSN_ERR_TIMEOUT, stops issuing
 // work, lets its copies land, frees its TMEM and returns.
 #include "dsn_internal.cuh"
@@ -31,6 +34,7 @@ constexpr int BK = DSN_GEMM_BK;
 constexpr uint32_t kABytes = BM * BK * 2;  // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr int kMaxStages = 8;
+constexpr uint32_t kStageOutBytes = 4 * 32 * 128;  // epilogue transpose: 4 warps x 32 rows x 128 bytes
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -160,10 +164,81 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-__device__ __forceinline__ float apply_act(float v, int act) {
-  if (act == DSN_ACT_RELU) return fmaxf(v, 0.f);
-  if (act == DSN_ACT_GELU) return 0.5f * v * (1.f + erff(v * 0.70710678118654752f));
+// erf by the rational approximation of Abramowitz & Stegun, formula 7.1.26 (|error| <= 1.5e-7,
+// far below bf16 resolution): erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1 / (1 + p x), x >= 0.
+__device__ __forceinline__ float erf_as(float x) {
+  const float ax = fabsf(x);
+  const float t = __fdividef(1.f, fmaf(0.3275911f, ax, 1.f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float r = 1.f - poly * t * __expf(-ax * ax);
+  return copysignf(r, x);
+}
+
+// The activation is a template parameter so that the per-element loop holds no trace of the others.
+template <int ACT>
+__device__ __forceinline__ float apply_act(float v) {
+  if (ACT == DSN_ACT_RELU) return fmaxf(v, 0.f);
+  if (ACT == DSN_ACT_GELU) return 0.5f * v * (1.f + erf_as(v * 0.70710678118654752f));
   return v;
+}
+
+// Epilogue of one tile for one warp: accumulator rows (one per lane) -> bias, activation, bf16 ->
+// 32 x 128-byte transpose in swizzled shared memory -> row-contiguous global stores.
+template <int ACT>
+__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, const float* brow, uint8_t* stage_w,
+                                              __nv_bfloat16* const (&rp)[8], int lane) {
+  for (int c0 = 0; c0 < ncols; c0 += 64) {
+    // phase 1: this thread's row, 64 columns -> bf16 -> its 128-byte row of the staging tile
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      if (c0 + 32 * half < ncols) {  // warp-uniform
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + c0 + 32 * half, v);
+        tmem_ld_wait();
+        const int cb = c0 + 32 * half;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = 8 * jj + 2 * e;
+            float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
+            if (brow) {
+              if (cb + c < ncols) a += __ldg(brow + cb + c);
+              if (cb + c + 1 < ncols) b += __ldg(brow + cb + c + 1);
+            }
+            __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
+            w[e] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          const int j = 4 * half + jj;
+          *reinterpret_cast<uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+    __syncwarp();
+    // phase 2: eight lanes per row, 16 bytes each: contiguous 128-byte pieces of output rows
+    const int j = lane & 7, col = c0 + 8 * j;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = 4 * i + (lane >> 3);
+      if (rp[i] != nullptr && col < ncols) {
+        const uint4 val = *reinterpret_cast<const uint4*>(stage_w + row * 128 + ((j ^ (row & 7)) << 4));
+        if (col + 8 <= ncols) {
+          *reinterpret_cast<uint4*>(rp[i] + col) = val;
+        } else {  // slice width not a multiple of 8: the last few columns one by one
+          const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (col + e < ncols)
+              reinterpret_cast<uint16_t*>(rp[i] + col)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
+        }
+      }
+    }
+    __syncwarp();
+  }
 }
 
 // ---------------------------------------------------------------------------------- tile decode
@@ -225,7 +300,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
   const uint32_t b_bytes = (uint32_t)g.BN * BK * 2;
   const uint32_t stage_bytes = kABytes + b_bytes;
   const uint32_t tiles_base = base + kCtrlBytes;
-  int32_t* s_prefix = reinterpret_cast<int32_t*>(smem + kCtrlBytes + (size_t)stages * stage_bytes);
+  uint8_t* out_stage = smem + kCtrlBytes + (size_t)stages * stage_bytes;
+  int32_t* s_prefix = reinterpret_cast<int32_t*>(out_stage + kStageOutBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tmem_cols = 2u * (uint32_t)g.BN;  // 128, 256 or 512: a power of two >= 32
@@ -370,53 +446,26 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
           out_row = (int64_t)smp * g.R + yy * g.W + xx;
         }
       }
-      __nv_bfloat16* yrow = p.y + out_row * p.ldy + t.n0;
+      __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
+      // output rows this lane writes in the store phase: row 4*i + lane/8 of the warp's 32 rows
+      __nv_bfloat16* rp[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        rp[i] = reinterpret_cast<__nv_bfloat16*>(
+            __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(yrow), 4 * i + (lane >> 3)));
 
       // every lane waits, then the warp takes one decision so that tcgen05.ld stays warp-wide
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 4));
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
-      for (int c0 = 0; c0 < ncols; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + c0, v);
-        tmem_ld_wait();
-        if (valid) {
-          const int nv = ncols - c0 < 32 ? ncols - c0 : 32;
-          uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a = __uint_as_float(v[2 * i]), b = __uint_as_float(v[2 * i + 1]);
-            if (brow) {
-              if (2 * i < nv) a += __ldg(brow + c0 + 2 * i);
-              if (2 * i + 1 < nv) b += __ldg(brow + c0 + 2 * i + 1);
-            }
-            a = apply_act(a, p.act);
-            b = apply_act(b, p.act);
-            __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-            packed[i] = *reinterpret_cast<uint32_t*>(&h);
-          }
-          __nv_bfloat16* dst = yrow + c0;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            if (8 * i + 8 <= nv) {
-              reinterpret_cast<uint4*>(dst)[i] =
-                  make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-            } else if (8 * i < nv) {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                if (8 * i + e < nv) {
-                  const uint32_t w = packed[4 * i + e / 2];
-                  reinterpret_cast<uint16_t*>(dst)[8 * i + e] = (e & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xffffu);
-                }
-              }
-            }
-          }
-        }
-      }
+      uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
+      if (p.act == DSN_ACT_NONE) epilogue_tile<DSN_ACT_NONE>(taddr, ncols, brow, stage_w, rp, lane);
+      else if (p.act == DSN_ACT_RELU) epilogue_tile<DSN_ACT_RELU>(taddr, ncols, brow, stage_w, rp, lane);
+      else epilogue_tile<DSN_ACT_GELU>(taddr, ncols, brow, stage_w, rp, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
@@ -435,9 +484,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
 
 }  // namespace
 
-size_t dsn_gemm_smem_bytes(int BN, int stages) {
-  return 1024 /* alignment slack */ + kCtrlBytes + (size_t)stages * (kABytes + (size_t)BN * BK * 2) +
-         sizeof(int32_t) * (DSN_MAX_GROUPS + 1);
+size_t dsn_gemm_smem_bytes(int BN, int stages, int G) {
+  return 1024 /* alignment slack */ + kCtrlBytes + (size_t)stages * (kABytes + (size_t)BN * BK * 2) + kStageOutBytes +
+         sizeof(int32_t) * ((size_t)G + 1);
 }
 
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s) {

@@ -25,7 +25,7 @@ __device__ __forceinline__ void dsn_set_status(int32_t* status, int code, int de
 
 // ----------------------------------------------------------------------------------------------
 // Grouped GEMM parameters (bf16, tcgen05).  One launch covers every group whose slice has a
-// tensor map in this launch (map_id != 0xFF).
+// tensor-map pair in this launch (map_id != 0xFF); one pair per distinct (k_in, k_out).
 // ----------------------------------------------------------------------------------------------
 #define DSN_GEMM_MAX_MAPS 16
 #define DSN_GEMM_BM 128
@@ -65,7 +65,7 @@ struct GemmParams {
 
 // launchers implemented in the .cu files
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
-size_t dsn_gemm_smem_bytes(int BN, int stages);
+size_t dsn_gemm_smem_bytes(int BN, int stages, int G);
 
 cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_out, float* logits_out,
                             float* partial, int splits, int32_t* status, cudaStream_t s);
