@@ -162,6 +162,7 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     p.k_in[t] = (int16_t)c.k_in[t];
     p.k_out[t] = (int16_t)c.k_out[t];
   }
+  while (p.g.stages > 2 && dsn_gemm_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
   const size_t smem = dsn_gemm_smem_bytes(g.BN, g.stages, r->G);
 
   // one tensor-map pair per distinct slice (k_in, k_out), DSN_GEMM_MAX_MAPS pairs per launch
@@ -207,6 +208,11 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
       const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
       const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)g.BN};
       e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
+      if (e) return e;
+      const uint64_t yd[2] = {(uint64_t)map_n[m], (uint64_t)r->B * g.R};  // columns clipped at k_out
+      const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
+      const uint32_t yb[2] = {64, 32};
+      e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
       if (e) return e;
     }
     if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) return DSN_ERR_CUDA;

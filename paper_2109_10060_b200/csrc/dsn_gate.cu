@@ -20,6 +20,15 @@ constexpr int kJB = 16;            // hidden units per CTA in the hidden-layer k
 constexpr int kPoolThreads = 512;
 constexpr int kMlpThreads = 256;
 
+// 16-byte read-only load that the compiler keeps in program order, so that a run of them stays
+// in flight together instead of being interleaved with the arithmetic that consumes them
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
 __device__ __forceinline__ void add8(float (&acc)[8], const uint4& v) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -47,9 +56,16 @@ pool_bf16_vec_kernel(const __nv_bfloat16* __restrict__ x, int R, int64_t ldx, in
     if (v < nvec) {
       const uint4* col = reinterpret_cast<const uint4*>(xb) + v;
       int r = r0 + ty;
-      for (; r + 3 * RG < r1; r += 4 * RG) {  // four independent loads in flight per thread
-        const uint4 a0 = __ldg(col + (int64_t)r * stride), a1 = __ldg(col + (int64_t)(r + RG) * stride),
-                    a2 = __ldg(col + (int64_t)(r + 2 * RG) * stride), a3 = __ldg(col + (int64_t)(r + 3 * RG) * stride);
+      for (; r + 7 * RG < r1; r += 8 * RG) {  // eight independent loads in flight per thread
+        uint4 a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] = ld_stream16(col + (int64_t)(r + u * RG) * stride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) add8(acc, a[u]);
+      }
+      for (; r + 3 * RG < r1; r += 4 * RG) {
+        const uint4 a0 = ld_stream16(col + (int64_t)r * stride), a1 = ld_stream16(col + (int64_t)(r + RG) * stride),
+                    a2 = ld_stream16(col + (int64_t)(r + 2 * RG) * stride), a3 = ld_stream16(col + (int64_t)(r + 3 * RG) * stride);
         add8(acc, a0); add8(acc, a1); add8(acc, a2); add8(acc, a3);
       }
       for (; r < r1; r += RG) add8(acc, __ldg(col + (int64_t)r * stride));
@@ -97,14 +113,31 @@ gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, 
   const int b0 = blockIdx.x * kSB, j0 = blockIdx.y * kJB;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_r = 1.0f / (float)R;
-  for (int e = tid; e < kSB * c_valid; e += kMlpThreads) {
-    const int s = e / c_valid, c = e - s * c_valid;
-    float acc = 0.f;
-    if (b0 + s < B) {
-      const float* p = partial + ((int64_t)(b0 + s) * splits) * c_valid + c;
-      for (int sp = 0; sp < splits; ++sp) acc += p[(int64_t)sp * c_valid];
+  if (c_valid % 4 == 0) {  // partial rows are 16-byte aligned: fold with 16-byte loads, splits in flight together
+    const int n4 = c_valid >> 2;
+    for (int e = tid; e < kSB * n4; e += kMlpThreads) {
+      const int s = e / n4, c4 = e - s * n4;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (b0 + s < B) {
+        const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)(b0 + s) * splits) * c_valid) + c4;
+#pragma unroll 8
+        for (int sp = 0; sp < splits; ++sp) {
+          const float4 t = p[(int64_t)sp * n4];
+          acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+      }
+      reinterpret_cast<float4*>(pooled + s * c_valid)[c4] = make_float4(acc.x * inv_r, acc.y * inv_r, acc.z * inv_r, acc.w * inv_r);
     }
-    pooled[e] = acc * inv_r;
+  } else {
+    for (int e = tid; e < kSB * c_valid; e += kMlpThreads) {
+      const int s = e / c_valid, c = e - s * c_valid;
+      float acc = 0.f;
+      if (b0 + s < B) {
+        const float* p = partial + ((int64_t)(b0 + s) * splits) * c_valid + c;
+        for (int sp = 0; sp < splits; ++sp) acc += p[(int64_t)sp * c_valid];
+      }
+      pooled[e] = acc * inv_r;
+    }
   }
   __syncthreads();
   const bool vec = (c_valid % 4 == 0) && (C_full % 4 == 0) && ((reinterpret_cast<uintptr_t>(W1) & 15) == 0);
@@ -119,7 +152,7 @@ gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, 
     if (vec) {
       const float4* w4 = reinterpret_cast<const float4*>(w);
       const int n4 = c_valid >> 2;
-#pragma unroll 4
+#pragma unroll 8
       for (int c = lane; c < n4; c += 32) {
         const float4 wv = __ldg(w4 + c);
 #pragma unroll
@@ -151,17 +184,23 @@ gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, 
 __global__ void __launch_bounds__(kMlpThreads)
 gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const float* __restrict__ W2,
                   const float* __restrict__ b2, int32_t* __restrict__ idx_out, float* __restrict__ logits_out,
-                  int32_t* status) {
+                  int32_t* status, int w2_in_smem) {
+  extern __shared__ __align__(16) float w2s[];  // [T][C_mlp] when it fits
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (w2_in_smem) {  // one round of loads by the whole CTA instead of T dependent first touches per warp
+    for (int e = threadIdx.x; e < T * C_mlp; e += kMlpThreads) w2s[e] = __ldg(W2 + e);
+    __syncthreads();
+  }
   const int b = blockIdx.x * (kMlpThreads / 32) + warp;
   if (b >= B) return;
   const float* h = hid + (int64_t)b * C_mlp;
+  const float* wbase = w2_in_smem ? w2s : W2;
   int best = 0, nonfinite = 0;
   float best_v = 0.f;
   for (int t = 0; t < T; ++t) {
-    const float* w = W2 + (int64_t)t * C_mlp;
+    const float* w = wbase + (int64_t)t * C_mlp;
     float v = 0.f;
-    for (int j = lane; j < C_mlp; j += 32) v = fmaf(__ldg(w + j), h[j], v);
+    for (int j = lane; j < C_mlp; j += 32) v = fmaf(w[j], h[j], v);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     v += b2 ? b2[t] : 0.f;
@@ -186,8 +225,8 @@ gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const 
 }  // namespace
 
 int dsn_gate_splits(const dsn_gate_desc& g, int sm_count) {
-  // about four 512-thread CTAs per SM, at least 8 rows per CTA
-  int want = (4 * sm_count + g.B - 1) / g.B;
+  // at most four 512-thread CTAs per SM (one resident wave), at least 8 rows per CTA
+  int want = (4 * sm_count) / g.B;
   int max_by_rows = g.R / 8 > 0 ? g.R / 8 : 1;
   int s = want < max_by_rows ? want : max_by_rows;
   if (s < 1) s = 1;
@@ -228,8 +267,10 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int per_cta = kMlpThreads / 32;
-  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, 0, s>>>(hid, g.B, g.C_mlp, g.T, g.W2, g.b2, idx_out,
-                                                                         logits_out, status);
+  const size_t w2_bytes = sizeof(float) * (size_t)g.T * g.C_mlp;
+  const int w2_in_smem = w2_bytes <= 40 * 1024;
+  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, w2_in_smem ? w2_bytes : 0, s>>>(
+      hid, g.B, g.C_mlp, g.T, g.W2, g.b2, idx_out, logits_out, status, w2_in_smem);
   return cudaGetLastError();
 }
 

@@ -13,14 +13,16 @@
 // the full tensors, so everything beyond the slice arrives in shared memory as zeros: it is never
 // fetched from L2 and never multiplied.
 //
-// Structure of a CTA (persistent, one per SM, 192 threads):
+// Structure of a CTA (persistent, one per SM, 320 threads):
 //   warp 0      one lane issues the TMA loads into a ring of shared-memory stages
 //   warp 1      one lane issues tcgen05.mma (M = 128, N = 16..256, K = 16) into a TMEM accumulator;
 //               two accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
-//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), bias / activation, bf16
-//               rounding, a 32-row x 128-byte transpose through swizzled shared memory, then
-//               stores in which eight lanes write one contiguous 128-byte piece of an output row
-//               (grouped or input-order / scattered rows alike)
+//   warps 2..9  epilogue, two warps per TMEM lane quarter taking alternate 64-column chunks:
+//               tcgen05.ld (one accumulator row per thread), bias / activation, bf16 rounding into a
+//               32-row x 128-byte swizzled staging tile, then one TMA store of that tile when the
+//               warp's 32 rows are consecutive rows of the output (the tensor map clips the columns
+//               at k_out); otherwise stores in which eight lanes write one contiguous 128-byte
+//               piece of an output row (group tails, sample boundaries of scattered output)
 // Every mbarrier wait is bounded; on a timeout the CTA records DSN_ERR_TIMEOUT, stops issuing
 // work, lets its copies land, frees its TMEM and returns.
 #include "dsn_internal.cuh"
@@ -28,13 +30,14 @@
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
 constexpr int BM = DSN_GEMM_BM;
 constexpr int BK = DSN_GEMM_BK;
 constexpr uint32_t kABytes = BM * BK * 2;  // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr int kMaxStages = 8;
-constexpr uint32_t kStageOutBytes = 4 * 32 * 128;  // epilogue transpose: 4 warps x 32 rows x 128 bytes
+constexpr uint32_t kStageOutBytes = kEpiWarps * 32 * 128;  // epilogue staging: 32 rows x 128 bytes per warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -104,6 +107,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
       : "memory");
 }
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// make shared-memory writes of this thread visible to the async (TMA) proxy
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -186,11 +200,19 @@ __device__ __forceinline__ float apply_act(float v) {
 }
 
 // Epilogue of one tile for one warp: accumulator rows (one per lane) -> bias, activation, bf16 ->
-// 32 x 128-byte transpose in swizzled shared memory -> row-contiguous global stores.
+// 32 x 128-byte swizzled staging tile -> global memory.  The warp takes the 64-column chunks
+// `first`, `first + 2`, ...  With `contig` the 32 rows are consecutive output rows starting at
+// `base_row` and each chunk leaves as one TMA store (columns clipped by the map); otherwise eight
+// lanes store one 128-byte piece of a row each.
 template <int ACT>
-__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, const float* brow, uint8_t* stage_w,
-                                              __nv_bfloat16* const (&rp)[8], int lane) {
-  for (int c0 = 0; c0 < ncols; c0 += 64) {
+__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
+                                              uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
+                                              const CUtensorMap* mapY, int base_row) {
+  for (int c0 = 64 * first; c0 < ncols; c0 += 128) {
+    // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
+    // staging tile before it is overwritten; free when nothing is outstanding
+    if (lane == 0) bulk_wait_read0();
+    __syncwarp();
     // phase 1: this thread's row, 64 columns -> bf16 -> its 128-byte row of the staging tile
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
@@ -217,6 +239,15 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, const f
           *reinterpret_cast<uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
+    }
+    if (contig) {
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_2d(mapY, n0 + c0, base_row, smem_u32(stage_w));
+        bulk_commit();
+      }
+      continue;
     }
     __syncwarp();
     // phase 2: eight lanes per row, 16 bytes each: contiguous 128-byte pieces of output rows
@@ -313,7 +344,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 4);
+      mbar_init(bar_tempty + 8 * a, kEpiWarps);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -414,8 +445,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;          // TMEM lane quarter this warp may read
+    const int first = (warp - 2) >> 2;  // which alternate 64-column chunks this warp takes
     const int m = q * 32 + lane;     // accumulator row of this thread
     int it = 0;
     bool ok = true;
@@ -450,12 +482,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
-      // output rows this lane writes in the store phase: row 4*i + lane/8 of the warp's 32 rows
+      // output rows this lane writes in the direct-store phase: row 4*i + lane/8 of the warp's 32 rows
       __nv_bfloat16* rp[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i)
         rp[i] = reinterpret_cast<__nv_bfloat16*>(
             __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(yrow), 4 * i + (lane >> 3)));
+      // 32 consecutive output rows can leave through the TMA unit
+      const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
+      // (a slice width that is no multiple of 8 columns = 16 bytes keeps the element-wise path: the
+      // store was seen to clip the row at 16-byte granularity and would touch columns >= k_out)
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
 
       // every lane waits, then the warp takes one decision so that tcgen05.ld stays warp-wide
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 4));
@@ -463,13 +500,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
-      if (p.act == DSN_ACT_NONE) epilogue_tile<DSN_ACT_NONE>(taddr, ncols, brow, stage_w, rp, lane);
-      else if (p.act == DSN_ACT_RELU) epilogue_tile<DSN_ACT_RELU>(taddr, ncols, brow, stage_w, rp, lane);
-      else epilogue_tile<DSN_ACT_GELU>(taddr, ncols, brow, stage_w, rp, lane);
+      const CUtensorMap* mY = &p.mapY[t.map];
+      if (p.act == DSN_ACT_NONE)
+        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+      else if (p.act == DSN_ACT_RELU)
+        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+      else
+        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
     }
+    if (lane == 0) bulk_wait0();  // this warp's TMA stores are complete before the CTA retires
   }
 
   // ------------------------------------------------------------------ teardown
