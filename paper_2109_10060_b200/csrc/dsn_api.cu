@@ -162,8 +162,26 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     p.k_in[t] = (int16_t)c.k_in[t];
     p.k_out[t] = (int16_t)c.k_out[t];
   }
-  while (p.g.stages > 2 && dsn_gemm_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
-  const size_t smem = dsn_gemm_smem_bytes(g.BN, g.stages, r->G);
+  // CTA pairs (two SMs per 256-row tile) halve the weight traffic per SM; fall back to one CTA per
+  // tile when no pair can be resident
+  const int bn_slot = g.BN == 256 ? 2 : (g.BN == 128 ? 1 : 0);
+  int clusters = 0;
+  size_t smem = 0;
+  if (ctx->gemm_mode == 0) {
+    p.g.pair = 1;
+    p.g.stages = g.BN == 256 ? 6 : 8;
+    while (p.g.stages > 2 && dsn_gemm_pair_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
+    smem = dsn_gemm_pair_smem_bytes(g.BN, g.stages, r->G);
+    if (ctx->pair_clusters[bn_slot] < 0) ctx->pair_clusters[bn_slot] = dsn_gemm_pair_max_clusters(227 * 1024);
+    clusters = ctx->pair_clusters[bn_slot];
+    if (clusters > ctx->sm_count / 2) clusters = ctx->sm_count / 2;
+  }
+  if (clusters <= 0) {
+    p.g.pair = 0;
+    p.g.stages = g.BN == 256 ? 4 : (g.BN == 128 ? 6 : 8);
+    while (p.g.stages > 2 && dsn_gemm_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
+    smem = dsn_gemm_smem_bytes(g.BN, g.stages, r->G);
+  }
 
   // one tensor-map pair per distinct slice (k_in, k_out), DSN_GEMM_MAX_MAPS pairs per launch
   int done[DSN_MAX_SLICES];
@@ -206,7 +224,7 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
       if (e) return e;
       const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)map_n[m]};  // rows beyond k_out: zeros, not fetched
       const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
-      const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)g.BN};
+      const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)(g.pair ? g.BN / 2 : g.BN)};
       e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
       if (e) return e;
       const uint64_t yd[2] = {(uint64_t)map_n[m], (uint64_t)r->B * g.R};  // columns clipped at k_out
@@ -215,7 +233,11 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
       e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
       if (e) return e;
     }
-    if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
+    if (g.pair) {
+      if (dsn_launch_gemm_bf16_pair(p, clusters, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
+    } else if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) {
+      return DSN_ERR_CUDA;
+    }
   }
   return DSN_OK;
 }
@@ -278,7 +300,8 @@ int check_gate(const dsn_gate_desc* g) {
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * 4 * (size_t)g->c_valid > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 1) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
+    return DSN_ERR_UNSUPPORTED;  // score kernel stages W2 in shared memory
   return DSN_OK;
 }
 
@@ -370,6 +393,11 @@ int dsn_create(dsn_ctx** out, int device) {
   if (!c) return DSN_ERR_INVALID_ARG;
   c->device = device;
   c->sm_count = prop.multiProcessorCount;
+  c->pair_clusters[0] = c->pair_clusters[1] = c->pair_clusters[2] = -1;
+  {
+    const char* m = getenv("DSN_GEMM_MODE");  // "1cta" forces one CTA per tile (for comparisons)
+    c->gemm_mode = (m && strcmp(m, "1cta") == 0) ? 1 : 0;
+  }
   cudaDriverEntryPointQueryResult q;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
       q != cudaDriverEntryPointSuccess || !c->encode_tiled) {

@@ -6,16 +6,17 @@
 // different rows, four loads are in flight per thread; fp32 accumulation in registers, one
 // shared-memory reduction across the row groups, column sums to partial[b][split][c].  No atomics,
 // so sums are reproducible run to run.
-// Kernel 2 (L2-bound, plain FMA): grid (B/4, C_mlp/16).  A CTA folds the partial sums of 4 samples
-// (scaled by 1/R) into shared memory and computes 16 hidden units for them, one warp per two
-// units with 16-byte weight loads and a shuffle reduction; ReLU; hid[b][j] to scratch.
-// Kernel 3 (tiny): one warp per sample evaluates the T scores and takes the arg-max with a strict
-// '>' scan in ascending path order (ties keep the lowest index).
+// Kernel 2 (latency-bound, plain FMA): grid (B/4, C_mlp/16).  A CTA folds the partial sums of 4
+// samples (scaled by 1/R) into shared memory and computes 16 hidden units for them, one warp per
+// two units, all weight loads of a 1024-channel panel in flight at once; ReLU; hid[b][j] to scratch.
+// Kernel 3 (tiny): one warp per sample, lane t owns the score of path t; arg-max by a strict '>'
+// scan in ascending path order (ties keep the lowest index).
 #include "dsn_internal.cuh"
 
 namespace {
 
-constexpr int kSB = 4;             // samples per CTA in the hidden-layer kernel
+constexpr int kSBSmall = 4;        // samples per CTA in the hidden-layer kernel
+constexpr int kSBLarge = 8;        // ... for large batches, where re-reading W1 per CTA would bound the kernel
 constexpr int kJB = 16;            // hidden units per CTA in the hidden-layer kernel
 constexpr int kPoolThreads = 512;
 constexpr int kMlpThreads = 256;
@@ -106,114 +107,162 @@ pool_scalar_kernel(const Tin* __restrict__ x, int R, int64_t ldx, int c_valid, i
   }
 }
 
+// 16-byte load kept in program order (see ld_stream16) but allowed to stay in L1/L2
+__device__ __forceinline__ float4 ld_ordered16(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
+// Hidden layer for kSB samples x kJB units per CTA.  The loop over the input channels runs in
+// panels of 1024: a warp first issues the 16-byte loads of its two weight rows for the panel
+// (16 per lane, all in flight), then the CTA folds the pooling partial sums of the panel into
+// shared memory (their loads overlap the weight loads), then the FMAs run out of registers and
+// shared memory.  Every global load of a panel is therefore issued in one round.
+template <int kSB>
 __global__ void __launch_bounds__(kMlpThreads)
 gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, int C_full, int c_valid, int C_mlp,
                    const float* __restrict__ W1, const float* __restrict__ b1, float* __restrict__ hid) {
-  extern __shared__ __align__(16) float pooled[];  // [kSB][c_valid]
+  __shared__ __align__(16) float pooled[kSB][1024];
   const int b0 = blockIdx.x * kSB, j0 = blockIdx.y * kJB;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_r = 1.0f / (float)R;
-  if (c_valid % 4 == 0) {  // partial rows are 16-byte aligned: fold with 16-byte loads, splits in flight together
-    const int n4 = c_valid >> 2;
-    for (int e = tid; e < kSB * n4; e += kMlpThreads) {
-      const int s = e / n4, c4 = e - s * n4;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (b0 + s < B) {
-        const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)(b0 + s) * splits) * c_valid) + c4;
-#pragma unroll 8
-        for (int sp = 0; sp < splits; ++sp) {
-          const float4 t = p[(int64_t)sp * n4];
-          acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-        }
-      }
-      reinterpret_cast<float4*>(pooled + s * c_valid)[c4] = make_float4(acc.x * inv_r, acc.y * inv_r, acc.z * inv_r, acc.w * inv_r);
-    }
-  } else {
-    for (int e = tid; e < kSB * c_valid; e += kMlpThreads) {
-      const int s = e / c_valid, c = e - s * c_valid;
-      float acc = 0.f;
-      if (b0 + s < B) {
-        const float* p = partial + ((int64_t)(b0 + s) * splits) * c_valid + c;
-        for (int sp = 0; sp < splits; ++sp) acc += p[(int64_t)sp * c_valid];
-      }
-      pooled[e] = acc * inv_r;
-    }
-  }
-  __syncthreads();
   const bool vec = (c_valid % 4 == 0) && (C_full % 4 == 0) && ((reinterpret_cast<uintptr_t>(W1) & 15) == 0);
+  const int ja = j0 + 2 * warp, jb = ja + 1;
+  float acc[2][kSB];
 #pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    const int j = j0 + 2 * warp + u;
-    if (j >= C_mlp) break;  // warp-uniform
-    float acc[kSB];
+  for (int u = 0; u < 2; ++u)
 #pragma unroll
-    for (int s = 0; s < kSB; ++s) acc[s] = 0.f;
-    const float* w = W1 + (int64_t)j * C_full;
+    for (int s = 0; s < kSB; ++s) acc[u][s] = 0.f;
+
+  for (int cbase = 0; cbase < c_valid; cbase += 1024) {
+    const int cw = c_valid - cbase < 1024 ? c_valid - cbase : 1024;  // panel width
+    float4 wa[8], wb[8];
     if (vec) {
-      const float4* w4 = reinterpret_cast<const float4*>(w);
-      const int n4 = c_valid >> 2;
-#pragma unroll 8
-      for (int c = lane; c < n4; c += 32) {
-        const float4 wv = __ldg(w4 + c);
+      const float4* pa = reinterpret_cast<const float4*>(W1 + (int64_t)(ja < C_mlp ? ja : 0) * C_full + cbase);
+      const float4* pb = reinterpret_cast<const float4*>(W1 + (int64_t)(jb < C_mlp ? jb : 0) * C_full + cbase);
+      const int n4 = cw >> 2;
 #pragma unroll
-        for (int s = 0; s < kSB; ++s) {
-          const float4 pv = reinterpret_cast<const float4*>(pooled + s * c_valid)[c];
-          acc[s] = fmaf(wv.x, pv.x, acc[s]);
-          acc[s] = fmaf(wv.y, pv.y, acc[s]);
-          acc[s] = fmaf(wv.z, pv.z, acc[s]);
-          acc[s] = fmaf(wv.w, pv.w, acc[s]);
+      for (int i = 0; i < 8; ++i) {
+        const int c = lane + 32 * i;
+        wa[i] = c < n4 ? ld_ordered16(pa + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        wb[i] = c < n4 ? ld_ordered16(pb + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    // fold the partial sums of this panel
+    if (c_valid % 4 == 0) {
+      const int n4 = cw >> 2, row4 = c_valid >> 2;
+      for (int e = tid; e < kSB * n4; e += kMlpThreads) {
+        const int s = e / n4, c4 = e - s * n4;
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (b0 + s < B) {
+          const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)(b0 + s) * splits) * c_valid + cbase) + c4;
+#pragma unroll 4
+          for (int sp = 0; sp < splits; ++sp) {
+            const float4 t = __ldg(p + (int64_t)sp * row4);
+            sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+          }
+        }
+        reinterpret_cast<float4*>(pooled[s])[c4] = make_float4(sum.x * inv_r, sum.y * inv_r, sum.z * inv_r, sum.w * inv_r);
+      }
+    } else {
+      for (int e = tid; e < kSB * cw; e += kMlpThreads) {
+        const int s = e / cw, c = e - s * cw;
+        float sum = 0.f;
+        if (b0 + s < B) {
+          const float* p = partial + ((int64_t)(b0 + s) * splits) * c_valid + cbase + c;
+          for (int sp = 0; sp < splits; ++sp) sum += p[(int64_t)sp * c_valid];
+        }
+        pooled[s][c] = sum * inv_r;
+      }
+    }
+    __syncthreads();
+    if (vec) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = lane + 32 * i;
+        if (c < (cw >> 2)) {
+#pragma unroll
+          for (int s = 0; s < kSB; ++s) {
+            const float4 pv = reinterpret_cast<const float4*>(pooled[s])[c];
+            acc[0][s] = fmaf(wa[i].x, pv.x, acc[0][s]); acc[0][s] = fmaf(wa[i].y, pv.y, acc[0][s]);
+            acc[0][s] = fmaf(wa[i].z, pv.z, acc[0][s]); acc[0][s] = fmaf(wa[i].w, pv.w, acc[0][s]);
+            acc[1][s] = fmaf(wb[i].x, pv.x, acc[1][s]); acc[1][s] = fmaf(wb[i].y, pv.y, acc[1][s]);
+            acc[1][s] = fmaf(wb[i].z, pv.z, acc[1][s]); acc[1][s] = fmaf(wb[i].w, pv.w, acc[1][s]);
+          }
         }
       }
     } else {
-      for (int c = lane; c < c_valid; c += 32) {
-        const float wv = __ldg(w + c);
+      for (int c = lane; c < cw; c += 32) {
+        const float va = ja < C_mlp ? __ldg(W1 + (int64_t)ja * C_full + cbase + c) : 0.f;
+        const float vb = jb < C_mlp ? __ldg(W1 + (int64_t)jb * C_full + cbase + c) : 0.f;
 #pragma unroll
-        for (int s = 0; s < kSB; ++s) acc[s] = fmaf(wv, pooled[s * c_valid + c], acc[s]);
+        for (int s = 0; s < kSB; ++s) {
+          acc[0][s] = fmaf(va, pooled[s][c], acc[0][s]);
+          acc[1][s] = fmaf(vb, pooled[s][c], acc[1][s]);
+        }
       }
     }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int j = ja + u;
 #pragma unroll
     for (int s = 0; s < kSB; ++s) {
-      float v = acc[s];
+      float v = acc[u][s];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0 && b0 + s < B) hid[(int64_t)(b0 + s) * C_mlp + j] = fmaxf(v + (b1 ? b1[j] : 0.f), 0.f);
+      if (lane == 0 && j < C_mlp && b0 + s < B) hid[(int64_t)(b0 + s) * C_mlp + j] = fmaxf(v + (b1 ? b1[j] : 0.f), 0.f);
     }
   }
 }
 
+// Scores and arg-max: one warp per sample.  W2 ([T][C_mlp], row pitch padded by one float) and the
+// sample's hidden vector are staged in shared memory with one round of loads; lane t (and t + 32)
+// accumulates the whole dot product of path t; lane 0 then scans the T scores in ascending order
+// with a strict '>' so that ties keep the lowest index.
 __global__ void __launch_bounds__(kMlpThreads)
 gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const float* __restrict__ W2,
                   const float* __restrict__ b2, int32_t* __restrict__ idx_out, float* __restrict__ logits_out,
-                  int32_t* status, int w2_in_smem) {
-  extern __shared__ __align__(16) float w2s[];  // [T][C_mlp] when it fits
+                  int32_t* status) {
+  extern __shared__ __align__(16) float sm[];
+  const int pitch = C_mlp + 1;
+  float* w2s = sm;                                   // [T][pitch]
+  float* hs = w2s + (size_t)T * pitch;               // [warps][C_mlp]
+  float* sc = hs + (size_t)(kMlpThreads / 32) * C_mlp;  // [warps][DSN_MAX_SLICES]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (w2_in_smem) {  // one round of loads by the whole CTA instead of T dependent first touches per warp
-    for (int e = threadIdx.x; e < T * C_mlp; e += kMlpThreads) w2s[e] = __ldg(W2 + e);
-    __syncthreads();
-  }
   const int b = blockIdx.x * (kMlpThreads / 32) + warp;
-  if (b >= B) return;
-  const float* h = hid + (int64_t)b * C_mlp;
-  const float* wbase = w2_in_smem ? w2s : W2;
-  int best = 0, nonfinite = 0;
-  float best_v = 0.f;
-  for (int t = 0; t < T; ++t) {
-    const float* w = wbase + (int64_t)t * C_mlp;
-    float v = 0.f;
-    for (int j = lane; j < C_mlp; j += 32) v = fmaf(w[j], h[j], v);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    v += b2 ? b2[t] : 0.f;
-    if (!isfinite(v)) ++nonfinite;
-    if (t == 0) {
-      best_v = v;
-    } else if (v > best_v) {  // strict: ties keep the lower index
-      best = t;
-      best_v = v;
-    }
-    if (lane == 0 && logits_out) logits_out[(int64_t)b * T + t] = v;
+  for (int e = threadIdx.x; e < T * C_mlp; e += kMlpThreads) {
+    const int t = e / C_mlp, j = e - t * C_mlp;
+    w2s[t * pitch + j] = __ldg(W2 + e);
   }
+  if (b < B)
+    for (int j = lane; j < C_mlp; j += 32) hs[warp * C_mlp + j] = hid[(int64_t)b * C_mlp + j];
+  __syncthreads();
+  if (b >= B) return;
+  const float* h = hs + warp * C_mlp;
+  for (int t = lane; t < T; t += 32) {
+    const float* w = w2s + t * pitch;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    int j = 0;
+    for (; j + 4 <= C_mlp; j += 4) {
+      a0 = fmaf(w[j], h[j], a0); a1 = fmaf(w[j + 1], h[j + 1], a1);
+      a2 = fmaf(w[j + 2], h[j + 2], a2); a3 = fmaf(w[j + 3], h[j + 3], a3);
+    }
+    for (; j < C_mlp; ++j) a0 = fmaf(w[j], h[j], a0);
+    const float v = (a0 + a1) + (a2 + a3) + (b2 ? b2[t] : 0.f);
+    sc[warp * DSN_MAX_SLICES + t] = v;
+    if (logits_out) logits_out[(int64_t)b * T + t] = v;
+  }
+  __syncwarp();
   if (lane == 0) {
+    const float* l = sc + warp * DSN_MAX_SLICES;
+    int best = 0, nonfinite = 0;
+    for (int t = 0; t < T; ++t) {
+      if (!isfinite(l[t])) ++nonfinite;
+      if (t > 0 && l[t] > l[best]) best = t;
+    }
     idx_out[b] = best;
     if (nonfinite) {
       dsn_set_status(status, DSN_ERR_NONFINITE, b);
@@ -256,21 +305,26 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const size_t smem = sizeof(float) * (size_t)kSB * g.c_valid;
-  if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(gate_hidden_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+  if (g.B >= 512) {
+    dim3 hgrid((g.B + kSBLarge - 1) / kSBLarge, (g.C_mlp + kJB - 1) / kJB);
+    gate_hidden_kernel<kSBLarge><<<hgrid, kMlpThreads, 0, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp,
+                                                               g.W1, g.b1, hid);
+  } else {
+    dim3 hgrid((g.B + kSBSmall - 1) / kSBSmall, (g.C_mlp + kJB - 1) / kJB);
+    gate_hidden_kernel<kSBSmall><<<hgrid, kMlpThreads, 0, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp,
+                                                               g.W1, g.b1, hid);
   }
-  dim3 hgrid((g.B + kSB - 1) / kSB, (g.C_mlp + kJB - 1) / kJB);
-  gate_hidden_kernel<<<hgrid, kMlpThreads, smem, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp, g.W1,
-                                                      g.b1, hid);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int per_cta = kMlpThreads / 32;
-  const size_t w2_bytes = sizeof(float) * (size_t)g.T * g.C_mlp;
-  const int w2_in_smem = w2_bytes <= 40 * 1024;
-  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, w2_in_smem ? w2_bytes : 0, s>>>(
-      hid, g.B, g.C_mlp, g.T, g.W2, g.b2, idx_out, logits_out, status, w2_in_smem);
+  const size_t smem = sizeof(float) * ((size_t)g.T * (g.C_mlp + 1) + (size_t)per_cta * g.C_mlp +
+                                       (size_t)per_cta * DSN_MAX_SLICES);
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(gate_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, smem, s>>>(hid, g.B, g.C_mlp, g.T, g.W2, g.b2,
+                                                                            idx_out, logits_out, status);
   return cudaGetLastError();
 }
 
@@ -317,7 +371,8 @@ extern "C" int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void*
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * kSB * (size_t)g->c_valid > 200 * 1024) return DSN_ERR_UNSUPPORTED;
+  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 1) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
+    return DSN_ERR_UNSUPPORTED;
   if (g->B == 0) return DSN_OK;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
   const size_t need = (size_t)g->B * splits * g->c_valid + (size_t)g->B * g->C_mlp;

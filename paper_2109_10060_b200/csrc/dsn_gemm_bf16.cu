@@ -25,252 +25,11 @@
 //               piece of an output row (group tails, sample boundaries of scattered output)
 // Every mbarrier wait is bounded; on a timeout the CTA records DSN_ERR_TIMEOUT, stops issuing
 // work, lets its copies land, frees its TMEM and returns.
-#include "dsn_internal.cuh"
-#include "dsn_tiles.cuh"
+#include "dsn_gemm_device.cuh"
 
 namespace {
 
-constexpr int kThreads = 320;
-constexpr int kEpiWarps = 8;
-constexpr int BM = DSN_GEMM_BM;
-constexpr int BK = DSN_GEMM_BK;
-constexpr uint32_t kABytes = BM * BK * 2;  // 16 KB: 128 rows of 128 bytes
-constexpr uint32_t kCtrlBytes = 1024;
-constexpr int kMaxStages = 8;
-constexpr uint32_t kStageOutBytes = kEpiWarps * 32 * 128;  // epilogue staging: 32 rows x 128 bytes per warp
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
-
-// ---------------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-
-// Bounded wait.  Returns false when the CTA is aborting (this or another thread ran out of time).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                            int32_t* status, int where) {
-  const uint64_t t0 = globaltimer_ns();
-  uint32_t spins = 0;
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 31u) == 0) {
-      if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        dsn_set_status(status, DSN_ERR_TIMEOUT, where);
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          int32_t* status, int where) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, where);
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// make shared-memory writes of this thread visible to the async (TMA) proxy
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// the mbarrier receives one arrival once every tcgen05.mma issued so far by this thread is done
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, 8-row groups
-// 1024 bytes apart (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
-__device__ __forceinline__ uint32_t make_idesc(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-// erf by the rational approximation of Abramowitz & Stegun, formula 7.1.26 (|error| <= 1.5e-7,
-// far below bf16 resolution): erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1 / (1 + p x), x >= 0.
-__device__ __forceinline__ float erf_as(float x) {
-  const float ax = fabsf(x);
-  const float t = __fdividef(1.f, fmaf(0.3275911f, ax, 1.f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float r = 1.f - poly * t * __expf(-ax * ax);
-  return copysignf(r, x);
-}
-
-// The activation is a template parameter so that the per-element loop holds no trace of the others.
-template <int ACT>
-__device__ __forceinline__ float apply_act(float v) {
-  if (ACT == DSN_ACT_RELU) return fmaxf(v, 0.f);
-  if (ACT == DSN_ACT_GELU) return 0.5f * v * (1.f + erf_as(v * 0.70710678118654752f));
-  return v;
-}
-
-// Epilogue of one tile for one warp: accumulator rows (one per lane) -> bias, activation, bf16 ->
-// 32 x 128-byte swizzled staging tile -> global memory.  The warp takes the 64-column chunks
-// `first`, `first + 2`, ...  With `contig` the 32 rows are consecutive output rows starting at
-// `base_row` and each chunk leaves as one TMA store (columns clipped by the map); otherwise eight
-// lanes store one 128-byte piece of a row each.
-template <int ACT>
-__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
-                                              uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
-                                              const CUtensorMap* mapY, int base_row) {
-  for (int c0 = 64 * first; c0 < ncols; c0 += 128) {
-    // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
-    // staging tile before it is overwritten; free when nothing is outstanding
-    if (lane == 0) bulk_wait_read0();
-    __syncwarp();
-    // phase 1: this thread's row, 64 columns -> bf16 -> its 128-byte row of the staging tile
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      if (c0 + 32 * half < ncols) {  // warp-uniform
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + c0 + 32 * half, v);
-        tmem_ld_wait();
-        const int cb = c0 + 32 * half;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = 8 * jj + 2 * e;
-            float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
-            if (brow) {
-              if (cb + c < ncols) a += __ldg(brow + cb + c);
-              if (cb + c + 1 < ncols) b += __ldg(brow + cb + c + 1);
-            }
-            __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
-            w[e] = *reinterpret_cast<uint32_t*>(&h);
-          }
-          const int j = 4 * half + jj;
-          *reinterpret_cast<uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-    }
-    if (contig) {
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        tma_store_2d(mapY, n0 + c0, base_row, smem_u32(stage_w));
-        bulk_commit();
-      }
-      continue;
-    }
-    __syncwarp();
-    // phase 2: eight lanes per row, 16 bytes each: contiguous 128-byte pieces of output rows
-    const int j = lane & 7, col = c0 + 8 * j;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int row = 4 * i + (lane >> 3);
-      if (rp[i] != nullptr && col < ncols) {
-        const uint4 val = *reinterpret_cast<const uint4*>(stage_w + row * 128 + ((j ^ (row & 7)) << 4));
-        if (col + 8 <= ncols) {
-          *reinterpret_cast<uint4*>(rp[i] + col) = val;
-        } else {  // slice width not a multiple of 8: the last few columns one by one
-          const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (col + e < ncols)
-              reinterpret_cast<uint16_t*>(rp[i] + col)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
-        }
-      }
-    }
-    __syncwarp();
-  }
-}
+using namespace dsn_gemm;
 
 // ---------------------------------------------------------------------------------- tile decode
 struct TileInfo {

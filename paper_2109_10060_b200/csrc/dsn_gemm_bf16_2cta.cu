@@ -1,0 +1,377 @@
+// Ragged grouped sliced GEMM on CTA pairs (tcgen05 cta_group::2), bf16 operands, fp32 accumulation.
+//
+// Same contract as the one-CTA kernel, different tile ownership: a cluster of two CTAs (two SMs)
+// computes a 256-row x BN-column tile.  Each CTA loads its own 128 activation rows and HALF of the
+// weight tile (BN/2 rows), the even CTA's MMA thread issues tcgen05.mma.cta_group::2 with M = 256,
+// and the tensor cores of both SMs read both halves of the weight tile.  Per SM the operand traffic
+// from L2 into shared memory drops from 16 KB + 32 KB to 16 KB + 16 KB per 128x256x64 block of
+// work, which is what bounds the one-CTA kernel on wide layers.  No multicast loads are used: every
+// CTA fetches its own bytes.
+//
+// Barriers (every CTA has the same shared-memory layout):
+//   full[s]    even CTA only.  One arrival (its producer's expect_tx for the bytes of BOTH CTAs);
+//              the TMA loads of both CTAs complete their bytes on it.
+//   empty[s]   both CTAs.  The even CTA's tcgen05.commit (multicast to both) frees the stage.
+//   tfull[a]   both CTAs.  The same multicast commit tells both epilogues that accumulator a is done.
+//   tempty[a]  even CTA only, 2 x 8 arrivals: the epilogue warps of both CTAs (remote arrive).
+// Every wait is bounded; on a timeout the CTA flags DSN_ERR_TIMEOUT and leaves its loops.
+#include <cuda_runtime.h>
+
+#include "dsn_gemm_device.cuh"
+
+namespace {
+
+using namespace dsn_gemm;
+
+// shared-window address of the same location in the pair's even CTA (cluster rank 0)
+__device__ __forceinline__ uint32_t leader_addr(uint32_t local_addr) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(0));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// one arrival on the barrier at this offset in BOTH CTAs once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+
+struct PairTile {
+  int map, ki, ko, n0;
+  int p_end;
+  int row0, rows_end;
+  int b0, x0, y0;
+};
+
+// Tile `tile` of the pair schedule as seen by CTA `rank`: the pair owns m-tiles 2*mtp and 2*mtp+1 of
+// one (group, n-tile); an m-tile past the group's last one yields only invalid rows.
+__device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const int32_t* s_prefix, int tile, int rank) {
+  PairTile t;
+  const GemmGeom& g = p.g;
+  const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
+  const int grp = p.G - 1 - j;
+  const int sl = p.group_slice ? p.group_slice[grp] : grp;
+  t.map = p.map_id[sl];
+  t.ki = p.k_in[sl];
+  t.ko = p.k_out[sl];
+  const int p0 = p.offsets[grp];
+  t.p_end = p.offsets[grp + 1];
+  const int ntn = (t.ko + g.BN - 1) / g.BN;
+  const int local = tile - s_prefix[j];
+  const int nt = local % ntn, mt = 2 * (local / ntn) + rank;
+  t.n0 = nt * g.BN;
+  if (g.flat) {
+    t.row0 = p0 * g.R + mt * BM;
+    t.rows_end = t.p_end * g.R;
+    t.b0 = t.x0 = t.y0 = 0;
+  } else {
+    const int per_img = g.tiles_x * g.tiles_y;
+    const int ib = mt / per_img, rem = mt - ib * per_img;
+    const int ty = rem / g.tiles_x, tx = rem - ty * g.tiles_x;
+    t.b0 = p0 + ib * g.nb;
+    t.y0 = ty * g.bh;
+    t.x0 = tx * g.bw;
+    t.row0 = t.rows_end = 0;
+  }
+  return t;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const GemmGeom& g = p.g;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+
+  const uint32_t bar_full = base;
+  const uint32_t bar_empty = base + 8 * kMaxStages;
+  const uint32_t bar_tfull = base + 16 * kMaxStages;
+  const uint32_t bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16 * kMaxStages + 32);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxStages + 36);
+
+  const int stages = g.stages;
+  const uint32_t bh_bytes = (uint32_t)(g.BN / 2) * BK * 2;  // this CTA's half of the weight tile
+  const uint32_t stage_bytes = kABytes + bh_bytes;
+  const uint32_t tiles_base = base + kCtrlBytes;
+  uint8_t* out_stage = smem + kCtrlBytes + (size_t)stages * stage_bytes;
+  int32_t* s_prefix = reinterpret_cast<int32_t*>(out_stage + kStageOutBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const uint32_t tmem_cols = 2u * (uint32_t)g.BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, 2 * kEpiWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), tmem_cols);
+    tmem_relinquish_pair();
+  }
+
+  auto ntiles_of = [&](int grp) {
+    const int sl = p.group_slice ? p.group_slice[grp] : grp;
+    if (sl < 0 || sl >= p.T || p.map_id[sl] == 0xFF) return 0;
+    const int cnt = p.offsets[grp + 1] - p.offsets[grp];
+    if (cnt <= 0) return 0;
+    const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
+    return ((mt + 1) / 2) * ((p.k_out[sl] + g.BN - 1) / g.BN);
+  };
+  dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything can arrive on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = s_prefix[p.G];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total; tile += npairs) {
+        const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+        const CUtensorMap* mA = &p.mapA[t.map];
+        const CUtensorMap* mB = &p.mapB[t.map];
+        const int nkc = (t.ki + BK - 1) / BK;
+        int ncols = t.ko - t.n0;
+        ncols = ncols > g.BN ? g.BN : ncols;
+        const int n_inst = (ncols + 31) & ~31;
+        const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
+        int bsel = t.b0;
+        if (g.a_input_order) bsel = t.b0 < t.p_end ? p.perm[t.b0] : p.B;  // past the group: out of range, zeros
+        for (int tap = 0; ok && tap < g.taps; ++tap) {
+          const int r = tap / g.KW, s = tap - r * g.KW;
+          for (int kc = 0; kc < nkc; ++kc) {
+            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
+            const uint32_t full_lead = leader_addr(bar_full + 8 * stage);  // the even CTA's barrier
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * (a_box_bytes + bh_bytes));
+            const uint32_t sa = tiles_base + stage * stage_bytes;
+            if (g.flat) tma_load_4d_pair(sa, mA, kc * BK, t.row0, 0, 0, full_lead);
+            else tma_load_4d_pair(sa, mA, kc * BK, t.x0 + s - g.pad, t.y0 + r - g.pad, bsel, full_lead);
+            tma_load_3d_pair(sa + kABytes, mB, kc * BK, tap, brow0, full_lead);
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
+        const PairTile t = decode_pair_tile(p, s_prefix, tile, 0);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
+        tc_fence_after();
+        int ncols = t.ko - t.n0;
+        ncols = ncols > g.BN ? g.BN : ncols;
+        const int n_inst = (ncols + 31) & ~31;
+        const uint32_t idesc = make_idesc(2 * BM, n_inst);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
+        const int nkc = (t.ki + BK - 1) / BK;
+        uint32_t accumulate = 0;
+        for (int tap = 0; ok && tap < g.taps; ++tap) {
+          for (int kc = 0; kc < nkc; ++kc) {
+            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = tiles_base + stage * stage_bytes;
+            const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kABytes);
+            const int krem = t.ki - kc * BK;
+            const int nks = krem >= BK ? BK / 16 : (krem + 15) >> 4;
+            for (int ks = 0; ks < nks; ++ks) {
+              umma_bf16_pair(d_tmem, da + 2u * ks, db + 2u * ks, idesc, accumulate);
+              accumulate = 1;
+            }
+            umma_commit_pair(bar_empty + 8 * stage);
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+        if (ok) umma_commit_pair(bar_tfull + 8 * acc);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int q = warp & 3;
+    const int first = (warp - 2) >> 2;
+    const int m = q * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    const int box_rows = g.bw * g.bh * g.nb, img_rows = g.bw * g.bh;
+    for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+
+      bool valid;
+      int64_t out_row;
+      if (g.flat) {
+        const int gr = t.row0 + m;
+        valid = gr < t.rows_end;
+        out_row = gr;
+        if (valid && g.y_input_order) {
+          const int pp = gr / g.R;
+          out_row = (int64_t)p.perm[pp] * g.R + (gr - pp * g.R);
+        }
+      } else {
+        const int bi = m / img_rows, rem = m - bi * img_rows;
+        const int yy = t.y0 + rem / g.bw, xx = t.x0 + rem % g.bw;
+        const int pp = t.b0 + bi;
+        valid = m < box_rows && yy < g.H && xx < g.W && pp < t.p_end;
+        out_row = 0;
+        if (valid) {
+          const int smp = g.y_input_order ? p.perm[pp] : pp;
+          out_row = (int64_t)smp * g.R + yy * g.W + xx;
+        }
+      }
+      __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
+      const float* brow = p.bias ? p.bias + t.n0 : nullptr;
+      int ncols = t.ko - t.n0;
+      ncols = ncols > g.BN ? g.BN : ncols;
+      __nv_bfloat16* rp[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        rp[i] = reinterpret_cast<__nv_bfloat16*>(
+            __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(yrow), 4 * i + (lane >> 3)));
+      const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
+      uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
+      const CUtensorMap* mY = &p.mapY[t.map];
+      if (p.act == DSN_ACT_NONE)
+        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+      else if (p.act == DSN_ACT_RELU)
+        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+      else
+        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it
+    }
+    if (lane == 0) bulk_wait0();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA retires while its partner may still read its memory or signal its barriers
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, tmem_cols);
+  }
+}
+
+}  // namespace
+
+size_t dsn_gemm_pair_smem_bytes(int BN, int stages, int G) {
+  return 1024 + kCtrlBytes + (size_t)stages * (kABytes + (size_t)(BN / 2) * BK * 2) + kStageOutBytes +
+         sizeof(int32_t) * ((size_t)G + 1);
+}
+
+// Largest number of CTA pairs that can be resident at once for this shared-memory size (0: no pair fits).
+int dsn_gemm_pair_max_clusters(size_t smem_bytes) {
+  if (cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) !=
+      cudaSuccess)
+    return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_bf16_pair_kernel, &cfg) != cudaSuccess) return 0;
+  return n;
+}
+
+cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * clusters, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_bf16_pair_kernel, p);
+}

@@ -17,6 +17,8 @@ struct dsn_ctx {
   int sm_count;
   int32_t* d_status;   // DSN_STATUS_WORDS ints
   void* encode_tiled;  // cuTensorMapEncodeTiled entry point
+  int gemm_mode;       // 0 = CTA pairs where possible (default), 1 = one CTA per tile (DSN_GEMM_MODE=1cta)
+  int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
 };
 
 __device__ __forceinline__ void dsn_set_status(int32_t* status, int code, int detail) {
@@ -43,6 +45,7 @@ struct GemmGeom {
   int32_t y_input_order;   // rows scattered to sample perm[p]
   int32_t BN;              // n-tile (64, 128, 256) = rows of the weight box
   int32_t stages;
+  int32_t pair;            // 1: tiles are owned by CTA pairs (256 rows), weight box holds BN/2 rows
 };
 
 struct GemmParams {
@@ -67,6 +70,9 @@ struct GemmParams {
 // launchers implemented in the .cu files
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
 size_t dsn_gemm_smem_bytes(int BN, int stages, int G);
+cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s);
+size_t dsn_gemm_pair_smem_bytes(int BN, int stages, int G);
+int dsn_gemm_pair_max_clusters(size_t smem_bytes);
 
 cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_out, float* logits_out,
                             float* partial, int splits, int32_t* status, cudaStream_t s);
