@@ -97,12 +97,12 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const 
   const GemmGeom& g = p.g;
   const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
   const int grp = p.G - 1 - j;
-  const int sl = p.group_slice ? p.group_slice[grp] : grp;
+  const int sl = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
   t.map = p.map_id[sl];
   t.ki = p.k_in[sl];
   t.ko = p.k_out[sl];
-  const int p0 = p.offsets[grp];
-  t.p_end = p.offsets[grp + 1];
+  const int p0 = s_prefix[p.G + 1 + grp];      // group offsets, cached in shared memory
+  t.p_end = s_prefix[p.G + 2 + grp];
   const int ntn = (t.ko + g.BN - 1) / g.BN;
   const int local = tile - s_prefix[j];
   const int nt = local % ntn, mt = 2 * (local / ntn) + rank;
@@ -174,6 +174,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
     const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
     return ((mt + 1) / 2) * ((p.k_out[sl] + g.BN - 1) / g.BN);
   };
+  // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group
+  for (int j = threadIdx.x; j <= p.G; j += blockDim.x) s_prefix[p.G + 1 + j] = p.offsets[j];
+  for (int j = threadIdx.x; j < p.G; j += blockDim.x) {
+    const int sl = p.group_slice ? p.group_slice[j] : j;
+    s_prefix[2 * p.G + 2 + j] = (sl >= 0 && sl < p.T) ? sl : 0;
+  }
   dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);
   tc_fence_before();
   __syncthreads();
@@ -334,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
 
 size_t dsn_gemm_pair_smem_bytes(int BN, int stages, int G) {
   return 1024 + kCtrlBytes + (size_t)stages * (kABytes + (size_t)(BN / 2) * BK * 2) + kStageOutBytes +
-         sizeof(int32_t) * ((size_t)G + 1);
+         sizeof(int32_t) * (3 * (size_t)G + 3);
 }
 
 // Largest number of CTA pairs that can be resident at once for this shared-memory size (0: no pair fits).
