@@ -147,23 +147,29 @@ class Bottleneck:
         self.dsn.dsn_layer_forward(ctx, self.L, self.xs[k], None if self.gate_driven else self.idx_given, self.ys[k],
                                    self.ws, idx_out=self.idx_out)
 
-    def decomposed_step(self, ctx, i, mark):
-        """Same path as separate C calls; mark(name) records a CUDA event after each."""
-        d, k = self.dsn, i % self.copies
-        mark("start")
+    def _parts(self):
+        d = self.dsn
+        parts = []
         if self.gate_driven:
-            d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)
-            mark("gate")
-            d.dsn_route(ctx, self.idx_out, self.B, self.T, self.routing)
+            parts.append(("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)))
+            parts.append(("route", lambda ctx, k: d.dsn_route(ctx, self.idx_out, self.B, self.T, self.routing)))
         else:
-            d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)
-        mark("route")
-        d.dsn_sliced_conv(ctx, self.dec_layers[0], self.routing, self.xs[k], self.t1)
-        mark("gemm:conv1_1x1")
-        d.dsn_sliced_conv(ctx, self.dec_layers[1], self.routing, self.t1, self.t2)
-        mark("gemm:conv2_3x3")
-        d.dsn_sliced_conv(ctx, self.dec_layers[2], self.routing, self.t2, self.ys[k])
-        mark("gemm:conv3_1x1")
+            parts.append(("route", lambda ctx, k: d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)))
+        parts.append(("gemm:conv1_1x1", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[0], self.routing, self.xs[k], self.t1)))
+        parts.append(("gemm:conv2_3x3", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[1], self.routing, self.t1, self.t2)))
+        parts.append(("gemm:conv3_1x1", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[2], self.routing, self.t2, self.ys[k])))
+        return parts
+
+    def decomposed_step(self, ctx, i, mark):
+        """Same path as separate C calls; mark(name) is called after each."""
+        k = i % self.copies
+        mark("start")
+        for name, fn in self._parts():
+            fn(ctx, k)
+            mark(name)
+
+    def decomposed_part(self, ctx, i, part):
+        self._parts()[part][1](ctx, i % self.copies)
 
     def histogram(self):
         return np.bincount(self.idx_out.cpu().numpy() if self.gate_driven else self.cfg["idx"], minlength=self.T)
@@ -271,6 +277,7 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time direct API calls instead of a CUDA-graph replay (for profilers)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -313,32 +320,88 @@ def main():
         raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
     counts = wlk.histogram()
 
+    # The timed steps replay a CUDA graph that holds one step per rotating buffer set, so that the
+    # host's launch work stays out of the device timeline.  Falls back to direct calls if capture fails.
+    side = torch.cuda.Stream()
+    graph, graphed = None, False
+    try:
+        if args.no_graph:
+            raise RuntimeError("disabled by --no-graph")
+        with torch.cuda.stream(side):
+            wlk.step(ctx, 0)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(wlk.copies):
+                wlk.step(ctx, i)
+        graph.replay()
+        torch.cuda.synchronize()
+        graphed = True
+    except Exception as exc:  # noqa: BLE001
+        sys.stderr.write(f"graph capture unavailable ({exc}); timing direct calls\n")
+
+    def run_steps(n):
+        if graphed:
+            for _ in range(n // wlk.copies):
+                graph.replay()
+            for i in range(n % wlk.copies):
+                wlk.step(ctx, i)
+        else:
+            for i in range(n):
+                wlk.step(ctx, i)
+
+    run_steps(wlk.copies * 2)
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record(stream)
-    for i in range(args.steps):
-        wlk.step(ctx, i)
+    run_steps(args.steps)
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
 
-    # per-kernel durations: same kernels, one C call per step of the path, events between calls
-    names, acc = [], {}
-    dec_steps = min(args.steps, 50)
-    for i in range(3 + dec_steps):
-        evs = []
-        def mark(n):
-            ev = torch.cuda.Event(enable_timing=True)
-            ev.record(stream)
-            evs.append((n, ev))
-        wlk.decomposed_step(ctx, i, mark)
-        torch.cuda.synchronize()
-        if i >= 3:
-            for (n0, a), (n1, b) in zip(evs[:-1], evs[1:]):
-                acc.setdefault(n1, []).append(a.elapsed_time(b))
+    # per-kernel durations: each step of the path (same kernels, one C call each) captured as its own
+    # graph over the rotating buffers and replayed back to back
+    acc = {}
+    marks = []
+    wlk.decomposed_step(ctx, 0, lambda n: marks.append(n))
+    torch.cuda.synchronize()
+    part_names = marks[1:]
+    for pi, pname in enumerate(part_names):
+        try:
+            if args.no_graph:
+                raise RuntimeError("disabled by --no-graph")
+            gpart = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gpart, stream=side):
+                for i in range(wlk.copies):
+                    wlk.decomposed_part(ctx, i, pi)
+            gpart.replay()
+            torch.cuda.synchronize()
+            reps = 20
+            e0.record(stream)
+            for _ in range(reps):
+                gpart.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            acc[pname] = [e0.elapsed_time(e1) / (reps * wlk.copies)]
+        except Exception as exc:  # noqa: BLE001
+            sys.stderr.write(f"per-kernel graph for {pname} unavailable ({exc})\n")
+    if not acc:  # no graphs: direct calls with an event after each (includes launch gaps)
+        for i in range(13):
+            evs = []
+            def mark(n):
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(stream)
+                evs.append((n, ev))
+            wlk.decomposed_step(ctx, i, mark)
+            torch.cuda.synchronize()
+            if i >= 3:
+                for (n0, a), (n1, b) in zip(evs[:-1], evs[1:]):
+                    acc.setdefault(n1, []).append(a.elapsed_time(b))
+    wlk.decomposed_step(ctx, 0, lambda n: None)   # leave the routing arrays consistent
+    torch.cuda.synchronize()
     clocks = sampler.stop()
 
     # end to end: batch starts and ends in pinned host memory
@@ -389,6 +452,7 @@ def main():
                    else f"{wlk.name}: batch {wlk.B} per GPU, routing {wlk.cfg['routing']}",
                    "path": "gate -> route -> 1x1 -> 3x3 -> 1x1 -> input order (dsn_layer_forward)",
                    "l2": f"inputs and outputs rotate over {wlk.copies} buffers (> 126 MB L2)",
+                   "launch": "CUDA graph replay of the public-API step" if graphed else "direct calls",
                    "routing_histogram": counts.tolist(), "parallelism": f"batch shards x{world}, no collective"},
         "samples_per_s": world * wlk.B / (ms_step * 1e-3),
         "pct_bf16_peak_burst": 100 * value / world / peaks["bf16_tflops"],
@@ -401,10 +465,10 @@ def main():
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        n = 16
+        n = wlk.B
         f_cpu, dt = wlk.oracle_sample(n)
         out["cpu_baseline"] = {"value": f_cpu / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
-                               "sample": f"first {n} of {wlk.B} samples, gate + route + bottleneck, fp64 numpy, {dt:.1f} s"}
+                               "sample": f"{n} of {wlk.B} samples, gate + route + bottleneck chain, fp64 numpy (threaded BLAS), {dt:.1f} s wall"}
     print(json.dumps(out))
 
 
