@@ -267,6 +267,148 @@ def run_reference(args):
     }))
 
 
+
+# --------------------------------------------------------------------------------------------- per-layer table
+def run_table(args):
+    """Per-layer numbers for every configuration (markdown rows for the benchmark spec): CUDA-graph replay over
+    rotating buffers larger than L2, executed TFLOP/s, fraction of the shape's roofline bound."""
+    import torch
+    from paper_2109_10060_b200.build import build
+    build()
+    import paper_2109_10060_b200 as dsn
+    import dsn_workloads as wl
+    from oracle import dsn_oracle as O
+    dev = torch.device("cuda:0")
+    ctx = dsn.Context(0)
+    peaks = load_peaks()
+    PEAK, HBM = peaks["bf16_tflops"], peaks["hbm_gbs"]
+    ints = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    side = torch.cuda.Stream()
+
+    def graph_time(call, nbuf, reps=10):
+        with torch.cuda.stream(side):
+            call(0)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(nbuf):
+                call(i)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * nbuf) * 1e3  # us
+
+    print("| config | layer | routing | us | executed TFLOP/s | % measured BF16 peak | bound (TFLOP/s) | % of bound | GB/s | samples/s |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
+
+    def layer(cfgname, lname, rname, B, H, Cin, Cout, k_in, k_out, idx, K=1, act=0, orders=(1, 1), group_list=None):
+        T = len(k_in)
+        R = H * H if K == 3 else H
+        if group_list is None:
+            r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
+            dsn.dsn_route(ctx, ints(idx), B, T, r)
+        else:
+            r = group_list
+        per = B * R * (Cin + Cout) * 2
+        nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
+        xs = [torch.randn(B, R, Cin, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        ys = [torch.zeros(B, R, Cout, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        if K == 1:
+            W = (torch.randn(Cout, Cin, device=dev) * Cin ** -0.5).to(torch.bfloat16)
+            d = dsn.make_linear_desc(dsn.BF16, R, Cin, Cout, k_in, k_out, W, act=act, in_order=orders[0], out_order=orders[1])
+            call = lambda i: dsn.dsn_sliced_linear(ctx, d, r, xs[i % nbuf], ys[i % nbuf])
+        else:
+            W = (torch.randn(Cout, K, K, Cin, device=dev) * (Cin * K * K) ** -0.5).to(torch.bfloat16)
+            d = dsn.make_conv_desc(dsn.BF16, H, H, K, 1, Cin, Cout, k_in, k_out, W, act=act, in_order=orders[0],
+                                   out_order=orders[1])
+            call = lambda i: dsn.dsn_sliced_conv(ctx, d, r, xs[i % nbuf], ys[i % nbuf])
+        us = graph_time(call, nbuf)
+        code, _ = ctx.get_status()
+        assert code == 0, code
+        counts = np.bincount(idx, minlength=T)
+        flops = 2 * dsn.dsn_executed_macs(counts.tolist(), R, k_in, k_out, K)
+        byts = sum(2 * (int(n) * R * (k_in[t] + k_out[t]) + k_in[t] * k_out[t] * K * K) for t, n in enumerate(counts) if n)
+        tf = flops / us / 1e6
+        bound = min(PEAK, flops / byts * HBM / 1e3)
+        print(f"| {cfgname} | {lname} | {rname} | {us:.1f} | {tf:.0f} | {100 * tf / PEAK:.1f} | {bound:.0f} | "
+              f"{100 * tf / bound:.0f} | {byts / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
+        del xs, ys
+
+    def gate_route(cfgname, B, R, C, T):
+        per = B * R * C * 2
+        nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
+        xs = [torch.randn(B, R, C, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        W1 = torch.randn(128, C, device=dev) * C ** -0.5
+        W2 = torch.randn(T, 128, device=dev) * 128 ** -0.5
+        g = dsn.make_gate_desc(dsn.BF16, B, R, C, 128, T, W1, W2)
+        ws = torch.empty(dsn.dsn_gate_workspace_bytes(g), dtype=torch.uint8, device=dev)
+        idx = torch.zeros(B, dtype=torch.int32, device=dev)
+        r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
+        us = graph_time(lambda i: dsn.dsn_gate(ctx, g, xs[i % nbuf], idx, None, ws), nbuf)
+        print(f"| {cfgname} | gate (pool + FC-ReLU-FC + arg-max) | - | {us:.1f} | - | - | HBM {HBM:.0f} GB/s | "
+              f"{100 * per / us / 1e3 / HBM:.0f} | {per / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
+        us = graph_time(lambda i: dsn.dsn_route(ctx, idx, B, T, r), 8)
+        print(f"| {cfgname} | route | - | {us:.1f} | - | - | launch latency | - | - | {B / us * 1e6:.0f} |", flush=True)
+
+    # config 2 / 4: bottlenecks
+    for cfgname, B, stages in (("cfg2", 128, (3,)), ("cfg4", 256, (1, 2, 3, 4))):
+        for stage in stages:
+            hw, outer, inner = wl.RESNET_STAGES[stage]
+            widths = wl.WIDTHS_14[inner]
+            full = [outer] * 14
+            routings = [("uniform", wl.idx_quota_uniform(wl.rng(40 + stage, 6), B, 14))]
+            if cfgname == "cfg4":
+                routings.insert(0, ("skewed", wl.idx_skewed_bands(wl.rng(40 + stage, 6), B, 14)))
+            tag = f"{cfgname} {hw}x{hw}"
+            gate_route(tag, B, hw * hw, outer, 14)
+            for rname, idx in routings:
+                layer(tag, f"conv1 1x1 {outer}->w", rname, B, hw * hw, outer, inner, full, widths, idx, act=1)
+                layer(tag, "conv2 3x3 w->w", rname, B, hw, inner, inner, widths, widths, idx, K=3, act=1)
+                layer(tag, f"conv3 1x1 w->{outer}", rname, B, hw * hw, inner, outer, widths, full, idx)
+    # config 3: ViT-S style
+    B, paths = 256, wl.vit_small_paths()
+    idx = wl.idx_quota_uniform(wl.rng(3, 9), B, 48)
+    gate_route("cfg3", B, 197, 384, 48)
+    for lname, Cin, Cout, act in (("qkv", 384, 1152, 0), ("proj", 384, 384, 0), ("fc1", 384, 1536, 2), ("fc2", 1536, 384, 0)):
+        ki, ko = wl.vit_layer_slices(paths, 64, lname)
+        layer("cfg3", lname, "uniform", B, 197, Cin, Cout, ki, ko, idx, act=act)
+    # config 5: ViT-B width
+    B, paths = 1024, wl.vit_base_paths()
+    gate_route("cfg5", B, 197, 768, 8)
+    cases = [("all on path 7", wl.idx_all_one(B, 7)), ("all on path 0", wl.idx_all_one(B, 0)),
+             ("uniform", wl.idx_quota_uniform(wl.rng(5, 9), B, 8)), ("zipf(1.2)", wl.idx_zipf(wl.rng(5, 9), B, 8))]
+    for rname, idx in cases:
+        for lname, Cin, Cout, act in (("qkv", 768, 2304, 0), ("fc1", 768, 3072, 2), ("fc2", 3072, 768, 0)):
+            ki, ko = wl.vit_layer_slices(paths, 64, lname)
+            layer("cfg5", lname, rname, B, 197, Cin, Cout, ki, ko, idx, act=act)
+    # singleton groups: 1024 caller-built groups of one sample each
+    idx = (np.arange(B) % 8).astype(np.int32)
+    order = np.arange(B, dtype=np.int32)
+    gl = dsn.make_routing(B, B, ints(np.ones(B)), ints(np.arange(B + 1)), ints(order), ints(order), ints(idx))
+    for lname, Cin, Cout, act in (("qkv", 768, 2304, 0), ("fc1", 768, 3072, 2), ("fc2", 3072, 768, 0)):
+        ki, ko = wl.vit_layer_slices(paths, 64, lname)
+        layer("cfg5", lname, "1024 singleton groups", B, 197, Cin, Cout, ki, ko, idx, act=act, group_list=gl)
+    # MobileNet-shaped pointwise layers (supplement)
+    for hw, C in ((14, 640), (7, 1152)):
+        widths = wl.WIDTHS_14[C]
+        idx = wl.idx_quota_uniform(wl.rng(6, 6), 256, 14)
+        layer(f"M {hw}x{hw}", f"pointwise 1x1 c->c (full {C})", "uniform", 256, hw * hw, C, C, widths, widths, idx, act=1)
+    # config 1: fp32 single layer
+    c1 = wl.config1()
+    x, W = torch.from_numpy(c1["x"]).to(dev), torch.from_numpy(c1["W"]).to(dev)
+    y = torch.zeros(64, 1, 256, device=dev)
+    r = dsn.make_routing(64, 4, ints(np.zeros(4)), ints(np.zeros(5)), ints(np.zeros(64)), ints(np.zeros(64)))
+    dsn.dsn_route(ctx, ints(c1["idx"]), 64, 4, r)
+    d = dsn.make_linear_desc(dsn.F32, 1, 256, 256, c1["k_in"], c1["k_out"], W)
+    us = graph_time(lambda i: dsn.dsn_sliced_linear(ctx, d, r, x, y), 8)
+    fl = 2 * dsn.dsn_executed_macs(np.bincount(c1["idx"], minlength=4).tolist(), 1, c1["k_in"], c1["k_out"], 1)
+    print(f"| cfg1 | fp32 linear 256x256, B=64 | iid | {us:.1f} | {fl / us / 1e6:.3f} | - | launch latency | - | - | {64 / us * 1e6:.0f} |")
+
 # --------------------------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
@@ -277,12 +419,16 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", action="store_true", help="print per-layer markdown rows for every configuration")
     ap.add_argument("--no-graph", action="store_true", help="time direct API calls instead of a CUDA-graph replay (for profilers)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.table:
+        run_table(args)
         return
 
     import torch
