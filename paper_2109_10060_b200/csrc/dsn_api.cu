@@ -8,6 +8,15 @@
 
 #include "dsn_internal.cuh"
 
+int dsn_pdl_enabled() {
+  static int enabled = -1;
+  if (enabled < 0) {
+    const char* e = getenv("DSN_PDL");
+    enabled = (e && e[0] == '0') ? 0 : 1;
+  }
+  return enabled;
+}
+
 namespace {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -49,6 +49,8 @@ permute_rows_kernel(SliceTable st, int elem_bytes, int R, const char* __restrict
                     char* __restrict__ dst, int64_t ld_dst, int to_grouped, int G,
                     const int32_t* __restrict__ offsets, const int32_t* __restrict__ perm,
                     const int32_t* __restrict__ group_slice) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   const int p = blockIdx.x;
   const RowJob j = locate(p, G, offsets, perm, group_slice);
   if (!j.valid) return;
@@ -79,6 +81,8 @@ __global__ void __launch_bounds__(kThreads)
 zero_tail_kernel(SliceTable st, int elem_bytes, int R, int C_out, char* __restrict__ y, int64_t ldy,
                  int y_input_order, int G, const int32_t* __restrict__ offsets,
                  const int32_t* __restrict__ perm, const int32_t* __restrict__ group_slice) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   const int p = blockIdx.x;
   const RowJob j = locate(p, G, offsets, perm, group_slice);
   if (!j.valid) return;
@@ -99,17 +103,15 @@ cudaError_t dsn_launch_permute_rows(const SliceTable& st, int elem_bytes, int R,
                                     const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                     cudaStream_t s) {
   if (B == 0) return cudaSuccess;
-  permute_rows_kernel<<<B, kThreads, 0, s>>>(st, elem_bytes, R, static_cast<const char*>(src), ld_src,
-                                              static_cast<char*>(dst), ld_dst, to_grouped, G, offsets, perm,
-                                              group_slice);
-  return cudaGetLastError();
+  return dsn_launch(permute_rows_kernel, dim3(B), dim3(kThreads), 0, s, 1, st, elem_bytes, R,
+                    static_cast<const char*>(src), ld_src, static_cast<char*>(dst), ld_dst, to_grouped, G, offsets, perm,
+                    group_slice);
 }
 
 cudaError_t dsn_launch_zero_tail(const SliceTable& st, int elem_bytes, int R, int C_out, void* y, int64_t ldy,
                                  int y_input_order, int B, int G, const int32_t* offsets, const int32_t* perm,
                                  const int32_t* group_slice, cudaStream_t s) {
   if (B == 0) return cudaSuccess;
-  zero_tail_kernel<<<B, kThreads, 0, s>>>(st, elem_bytes, R, C_out, static_cast<char*>(y), ldy, y_input_order, G,
-                                           offsets, perm, group_slice);
-  return cudaGetLastError();
+  return dsn_launch(zero_tail_kernel, dim3(B), dim3(kThreads), 0, s, 1, st, elem_bytes, R, C_out, static_cast<char*>(y),
+                    ldy, y_input_order, G, offsets, perm, group_slice);
 }

@@ -44,6 +44,8 @@ __global__ void __launch_bounds__(kPoolThreads)
 pool_bf16_vec_kernel(const __nv_bfloat16* __restrict__ x, int R, int64_t ldx, int c_valid, int splits, int CT,
                      float* __restrict__ partial) {
   __shared__ float red[kPoolThreads * 8];
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   const int b = blockIdx.y, sp = blockIdx.x;
   const int r0 = (int)(((int64_t)R * sp) / splits), r1 = (int)(((int64_t)R * (sp + 1)) / splits);
   const int nvec = c_valid >> 3;
@@ -96,6 +98,8 @@ template <typename Tin>
 __global__ void __launch_bounds__(128)
 pool_scalar_kernel(const Tin* __restrict__ x, int R, int64_t ldx, int c_valid, int splits,
                    float* __restrict__ partial) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   const int b = blockIdx.y, sp = blockIdx.x;
   const int r0 = (int)(((int64_t)R * sp) / splits), r1 = (int)(((int64_t)R * (sp + 1)) / splits);
   const Tin* xb = x + (int64_t)b * R * ldx;
@@ -124,6 +128,8 @@ __global__ void __launch_bounds__(kMlpThreads)
 gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, int C_full, int c_valid, int C_mlp,
                    const float* __restrict__ W1, const float* __restrict__ b1, float* __restrict__ hid) {
   __shared__ __align__(16) float pooled[kSB][1024];
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   const int b0 = blockIdx.x * kSB, j0 = blockIdx.y * kJB;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_r = 1.0f / (float)R;
@@ -233,6 +239,8 @@ gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const 
   float* sc = hs + (size_t)(kMlpThreads / 32) * C_mlp;  // [warps][DSN_MAX_SLICES]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int b = blockIdx.x * (kMlpThreads / 32) + warp;
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   for (int e = threadIdx.x; e < T * C_mlp; e += kMlpThreads) {
     const int t = e / C_mlp, j = e - t * C_mlp;
     w2s[t * pitch + j] = __ldg(W2 + e);
@@ -294,25 +302,25 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
     const int nvec = g.c_valid / 8;
     int CT = 8;
     while (CT < nvec && CT < 128) CT <<= 1;
-    pool_bf16_vec_kernel<<<grid, kPoolThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), g.R, g.ldx,
-                                                        g.c_valid, splits, CT, partial);
+    dsn_launch(pool_bf16_vec_kernel, grid, dim3(kPoolThreads), 0, s, 1, static_cast<const __nv_bfloat16*>(x), g.R,
+               g.ldx, g.c_valid, splits, CT, partial);
   } else if (g.dtype == DSN_BF16) {
-    pool_scalar_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(static_cast<const __nv_bfloat16*>(x), g.R, g.ldx,
-                                                           g.c_valid, splits, partial);
+    dsn_launch(pool_scalar_kernel<__nv_bfloat16>, grid, dim3(128), 0, s, 1, static_cast<const __nv_bfloat16*>(x), g.R,
+               g.ldx, g.c_valid, splits, partial);
   } else {
-    pool_scalar_kernel<float><<<grid, 128, 0, s>>>(static_cast<const float*>(x), g.R, g.ldx, g.c_valid, splits,
-                                                   partial);
+    dsn_launch(pool_scalar_kernel<float>, grid, dim3(128), 0, s, 1, static_cast<const float*>(x), g.R, g.ldx, g.c_valid,
+               splits, partial);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (g.B >= 512) {
     dim3 hgrid((g.B + kSBLarge - 1) / kSBLarge, (g.C_mlp + kJB - 1) / kJB);
-    gate_hidden_kernel<kSBLarge><<<hgrid, kMlpThreads, 0, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp,
-                                                               g.W1, g.b1, hid);
+    dsn_launch(gate_hidden_kernel<kSBLarge>, hgrid, dim3(kMlpThreads), 0, s, 1, (const float*)partial, splits, g.B, g.R,
+               g.C_full, g.c_valid, g.C_mlp, g.W1, g.b1, hid);
   } else {
     dim3 hgrid((g.B + kSBSmall - 1) / kSBSmall, (g.C_mlp + kJB - 1) / kJB);
-    gate_hidden_kernel<kSBSmall><<<hgrid, kMlpThreads, 0, s>>>(partial, splits, g.B, g.R, g.C_full, g.c_valid, g.C_mlp,
-                                                               g.W1, g.b1, hid);
+    dsn_launch(gate_hidden_kernel<kSBSmall>, hgrid, dim3(kMlpThreads), 0, s, 1, (const float*)partial, splits, g.B, g.R,
+               g.C_full, g.c_valid, g.C_mlp, g.W1, g.b1, hid);
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -323,8 +331,8 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
     e = cudaFuncSetAttribute(gate_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  gate_score_kernel<<<(g.B + per_cta - 1) / per_cta, kMlpThreads, smem, s>>>(hid, g.B, g.C_mlp, g.T, g.W2, g.b2,
-                                                                            idx_out, logits_out, status);
+  dsn_launch(gate_score_kernel, dim3((g.B + per_cta - 1) / per_cta), dim3(kMlpThreads), smem, s, 1, (const float*)hid,
+             g.B, g.C_mlp, g.T, g.W2, g.b2, idx_out, logits_out, status);
   return cudaGetLastError();
 }
 

@@ -121,6 +121,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
     const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
     return mt * ((p.k_out[sl] + g.BN - 1) / g.BN);
   };
+  // barriers and TMEM are set up; everything below reads what earlier kernels wrote
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group
   for (int j = threadIdx.x; j <= p.G; j += blockDim.x) s_prefix[p.G + 1 + j] = p.offsets[j];
   for (int j = threadIdx.x; j < p.G; j += blockDim.x) {
@@ -303,6 +306,5 @@ cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_
     if (e != cudaSuccess) return e;
     configured = smem_bytes;
   }
-  gemm_bf16_kernel<<<sm_count, kThreads, smem_bytes, s>>>(p);
-  return cudaGetLastError();
+  return dsn_launch(gemm_bf16_kernel, dim3(sm_count), dim3(kThreads), smem_bytes, s, 1, p);
 }

@@ -174,6 +174,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
     const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
     return ((mt + 1) / 2) * ((p.k_out[sl] + g.BN - 1) / g.BN);
   };
+  // barriers and TMEM are set up; everything below reads what earlier kernels wrote
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group
   for (int j = threadIdx.x; j <= p.G; j += blockDim.x) s_prefix[p.G + 1 + j] = p.offsets[j];
   for (int j = threadIdx.x; j < p.G; j += blockDim.x) {
@@ -365,19 +368,11 @@ int dsn_gemm_pair_max_clusters(size_t smem_bytes) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-  if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * clusters, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem_bytes;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_bf16_pair_kernel, p);
+  static size_t configured = 0;
+  if (smem_bytes > configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) return e;
+    configured = smem_bytes;
+  }
+  return dsn_launch(gemm_bf16_pair_kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
 }

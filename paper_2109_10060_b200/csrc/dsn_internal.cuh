@@ -21,6 +21,44 @@ struct dsn_ctx {
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
 };
 
+// Programmatic dependent launch: a kernel may be scheduled while its predecessor in the stream is
+// still draining.  Every kernel of this library therefore calls dsn_grid_dependency_wait() before its
+// first access to global memory (it returns once the predecessor grid has completed and its writes
+// are visible; the predecessors of that grid completed before it passed its own wait), and
+// dsn_grid_launch_dependents() right after, which lets the next kernel's CTAs start their set-up on
+// SMs that this grid has already left.
+__device__ __forceinline__ void dsn_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dsn_grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+int dsn_pdl_enabled();  // 1 unless the environment says DSN_PDL=0
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t dsn_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              int cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (dsn_pdl_enabled()) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = (unsigned)n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ void dsn_set_status(int32_t* status, int code, int detail) {
   if (status && atomicCAS(status, 0, code) == 0) status[1] = detail;
 }

@@ -23,6 +23,8 @@ linear_f32_kernel(SliceTable st, int R, const float* __restrict__ x, int64_t ldx
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
 
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   auto ntiles_of = [&](int g) {
     const int rows = (offsets[g + 1] - offsets[g]) * R;
     const int sl = group_slice ? group_slice[g] : g;
@@ -120,7 +122,6 @@ cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const floa
   const int64_t bound = ((int64_t)B * R / BM + G) * ((max_ko + BN - 1) / BN);
   int64_t grid = bound < (int64_t)sm_count * 4 ? bound : (int64_t)sm_count * 4;
   if (grid < 1) grid = 1;
-  linear_f32_kernel<<<(unsigned)grid, kThreads, sizeof(int32_t) * (G + 1), s>>>(
-      st, R, x, ldx, W, ldw, y, ldy, bias, act, x_input_order, y_input_order, G, offsets, perm, group_slice);
-  return cudaGetLastError();
+  return dsn_launch(linear_f32_kernel, dim3((unsigned)grid), dim3(kThreads), sizeof(int32_t) * (G + 1), s, 1, st, R, x,
+                    ldx, W, ldw, y, ldy, bias, act, x_input_order, y_input_order, G, offsets, perm, group_slice);
 }

@@ -20,6 +20,8 @@ route_kernel(const int32_t* __restrict__ idx, int B, int T, int32_t* __restrict_
   __shared__ int32_t s_bad;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   if (tid < DSN_MAX_SLICES) s_run[tid] = 0;
   if (tid == 0) s_bad = 0;
   __syncthreads();
@@ -99,6 +101,5 @@ route_kernel(const int32_t* __restrict__ idx, int B, int T, int32_t* __restrict_
 
 cudaError_t dsn_launch_route(const int32_t* idx, int B, int T, int32_t* counts, int32_t* offsets,
                              int32_t* perm, int32_t* inv_perm, int32_t* status, cudaStream_t s) {
-  route_kernel<<<1, kThreads, 0, s>>>(idx, B, T, counts, offsets, perm, inv_perm, status);
-  return cudaGetLastError();
+  return dsn_launch(route_kernel, dim3(1), dim3(kThreads), 0, s, 1, idx, B, T, counts, offsets, perm, inv_perm, status);
 }
