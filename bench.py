@@ -566,11 +566,9 @@ def main():
     if code != 0:
         raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    t2 = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    from paper_2109_10060_b200.sharding import max_over_ranks
+    t = max_over_ranks(torch.tensor([ms_total], dtype=torch.float64, device=dev), dist if world > 1 else None)
+    t2 = max_over_ranks(torch.tensor([ms_e2e], dtype=torch.float64, device=dev), dist if world > 1 else None)
     ms_step = float(t.item()) / args.steps
     ms_e2e = float(t2.item())
     flops = wlk.exec_flops(counts)
