@@ -14,6 +14,8 @@ Passages followed (DS-Net++, "Dynamic Weight Slicing"):
   * slice-able convolution W[:c_O, :c_I] * X ........... Sec. 3.3, "Filter number"
   * ViT QKV / proj / MLP slicing ....................... Sec. 3.4, Eq. (slimmableMLP)
   * gate: average-pool encoder, two-layer MLP, one-hot . Sec. 3.5
+  * gate attention head X * (1 + tanh(W3 ReLU(W1 X_E))) . Sec. 3.5, "double-headed dynamic gate"
+  * split batch norm with re-calibration (Re-SBN) ...... Sec. 3.3
   * on-the-fly multiply-add count ...................... Sec. 4.3 "Complexity penalty"
 
 Readings where the paper is silent (each is listed in the design notes):
@@ -116,6 +118,32 @@ def gate(x, W1, W2, b1=None, b2=None, c_valid=None):
     return idx, scores, margin
 
 
+def gate_attention(x, W1, W3, b1=None, b3=None, c_valid=None):
+    """Channel-attention head of the double-headed gate (Sec. 3.5): it shares W1 with the routing head.
+
+    scale[i][c] = 1 + tanh(b3[c] + sum_j W3[c][j] * ReLU(b1[j] + sum_c' W1[j][c'] * pooled[i][c']))
+    x_hat[i][r][c] = x[i][r][c] * scale[i][c]          for c < c_valid
+    x [B][R][C], W1 [C_mlp][C], W3 [C][C_mlp].  Returns (scale [B][c_valid], x_hat [B][R][c_valid]).
+    """
+    x = np.asarray(x, dtype=F64)
+    W1 = np.asarray(W1, dtype=F64)
+    W3 = np.asarray(W3, dtype=F64)
+    B, R, C = x.shape
+    cv = C if c_valid is None else int(c_valid)
+    scale = np.zeros((B, cv), dtype=F64)
+    for i in range(B):
+        pooled = x[i, :, :cv].sum(axis=0) / R
+        hid = W1[:, :cv] @ pooled
+        if b1 is not None:
+            hid = hid + np.asarray(b1, dtype=F64)
+        hid = np.maximum(hid, 0.0)
+        a = W3[:cv] @ hid
+        if b3 is not None:
+            a = a + np.asarray(b3, dtype=F64)[:cv]
+        scale[i] = 1.0 + np.tanh(a)
+    return scale, x[:, :, :cv] * scale[:, None, :]
+
+
 # --------------------------------------------------------------------------- routing
 def route(idx, T):
     """Group samples by path index, defined by enumeration.
@@ -146,9 +174,20 @@ def route(idx, T):
 
 
 # --------------------------------------------------------------------------- sliced layers
-def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, samples=None):
+def split_bn(z, t, gamma, beta, mu, sigma):
+    """Re-SBN for an input of route t with c = z.shape[-1] channels (Sec. 3.3):
+    gamma[:c] * (z - mu_t[:c]) / sigma_t[:c] + beta[:c]; mu, sigma are [T][C] per-route statistics."""
+    c = z.shape[-1]
+    g, b = np.asarray(gamma, dtype=F64)[:c], np.asarray(beta, dtype=F64)[:c]
+    m, s = np.asarray(mu, dtype=F64)[t, :c], np.asarray(sigma, dtype=F64)[t, :c]
+    return g * ((z - m) / s) + b
+
+
+def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None):
     """y[i][r][o] = act(b[o] + sum_{c<k_in[t]} x[i][r][c] W[o][c]),  o < k_out[t],  t = idx[i].
 
+    bn = (gamma[C_out], beta[C_out], mu[T][C_out], sigma[T][C_out]) inserts Re-SBN between the
+    contraction (+ bias) and the activation.
     x [B][R][C_in], W [C_out][C_in] (stored [out][in]).  Entries with o >= k_out[t] are not part
     of the result and hold `fill`.  `samples` restricts evaluation to a subset of samples (others
     hold `fill`); the per-sample definition makes that exact.
@@ -165,11 +204,13 @@ def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, 
         z = x[i, :, :ki] @ W[:ko, :ki].T
         if bias is not None:
             z = z + np.asarray(bias, dtype=F64)[:ko]
+        if bn is not None:                          # layer -> Re-SBN -> activation
+            z = split_bn(z, t, *bn)
         y[i, :, :ko] = activation(z, act)
     return y
 
 
-def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.nan, samples=None):
+def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None):
     """Slice-able convolution, stride 1, zero padding, no kernel flip.
 
     x [B][H][W][C_in] (channels last), W [C_O][C_I][K][K] (the paper's indexing).
@@ -194,6 +235,8 @@ def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.na
                 z += xp[r:r + H, s:s + Wd, :] @ W[:ko, :ki, r, s].T
         if bias is not None:
             z = z + np.asarray(bias, dtype=F64)[:ko]
+        if bn is not None:
+            z = split_bn(z, t, *bn)
         y[i, :, :, :ko] = activation(z, act)
     return y
 

@@ -253,6 +253,64 @@ def test_gate_known_winner_permutation_ties_bias_cvalid():
     np.testing.assert_array_equal(s1, s2)
 
 
+def test_gate_attention_head_brute_force_library_and_identity():
+    B, R, C, M = 4, 5, 6, 3
+    x, W1, W3, b1, b3 = rand(B, R, C), rand(M, C), rand(C, M), rand(M), rand(C)
+    scale, xh = O.gate_attention(x, W1, W3, b1, b3)
+    for i in range(B):
+        pooled = [sum(float(x[i, r, c]) for r in range(R)) / R for c in range(C)]
+        hid = [max(0.0, float(b1[j]) + sum(float(W1[j, c]) * pooled[c] for c in range(C))) for j in range(M)]
+        for c in range(C):
+            a = float(b3[c]) + sum(float(W3[c, j]) * hid[j] for j in range(M))
+            assert abs(scale[i, c] - (1.0 + math.tanh(a))) < 1e-12
+            for r in range(R):
+                assert abs(xh[i, r, c] - x[i, r, c] * (1.0 + math.tanh(a))) < 1e-12
+    xt = torch.from_numpy(x)
+    h = torch.relu(torch.nn.functional.linear(xt.mean(dim=1), torch.from_numpy(W1), torch.from_numpy(b1)))
+    lib = 1 + torch.tanh(torch.nn.functional.linear(h, torch.from_numpy(W3), torch.from_numpy(b3)))
+    np.testing.assert_allclose(scale, lib.numpy(), rtol=1e-12, atol=1e-12)
+    s0, x0 = O.gate_attention(x, W1, np.zeros((C, M)))             # delta(0) = 1: the head is the identity
+    assert np.all(s0 == 1.0) and np.array_equal(x0, x)
+    assert np.all(scale > 0.0) and np.all(scale < 2.0)              # 1 + tanh lies in (0, 2)
+    s_cv, x_cv = O.gate_attention(x, W1, W3, c_valid=4)             # elastic input
+    assert s_cv.shape == (B, 4) and x_cv.shape == (B, R, 4)
+    x2 = x.copy(); x2[..., 4:] = 1e9
+    np.testing.assert_array_equal(O.gate_attention(x2, W1, W3, c_valid=4)[0], s_cv)
+
+
+def test_split_bn_library_brute_force_and_identity():
+    B, H, Wd, Ci, Co, T = 3, 4, 3, 5, 6, 2
+    x, W = rand(B, H, Wd, Ci), rand(Co, Ci, 3, 3)
+    gamma, beta = rand(Co), rand(Co)
+    mu, sigma = rand(T, Co), np.abs(rand(T, Co)) + 0.5
+    idx = np.array([1, 0, 1]); k_in, k_out = [3, 5], [4, 6]
+    got = O.sliced_conv(x, W, idx, k_in, k_out, 1, bn=(gamma, beta, mu, sigma), act=O.ACT_RELU)
+    plain = O.sliced_conv(x, W, idx, k_in, k_out, 1)
+    for i in range(B):
+        t, ko = idx[i], k_out[idx[i]]
+        z = torch.from_numpy(plain[i:i + 1, :, :, :ko].copy()).permute(0, 3, 1, 2)
+        ref = torch.nn.functional.batch_norm(z, torch.from_numpy(mu[t, :ko].copy()), torch.from_numpy(sigma[t, :ko] ** 2),
+                                             torch.from_numpy(gamma[:ko].copy()), torch.from_numpy(beta[:ko].copy()),
+                                             training=False, eps=1e-30)
+        np.testing.assert_allclose(got[i, :, :, :ko], torch.relu(ref)[0].permute(1, 2, 0).numpy(), rtol=1e-11, atol=1e-12)
+        # brute force on one element: per-route statistics, shared gamma / beta sliced to the width
+        o = ko - 1
+        want = max(0.0, gamma[o] * (plain[i, 1, 1, o] - mu[t, o]) / sigma[t, o] + beta[o])
+        assert abs(got[i, 1, 1, o] - want) < 1e-12
+    ident = O.sliced_linear(rand(2, 3, 4), rand(5, 4), [0, 0], [4], [5],
+                            bn=(np.ones(5), np.zeros(5), np.zeros((1, 5)), np.ones((1, 5))))
+    # identity statistics leave the layer unchanged; wrong-route statistics change it
+    xx, WW = rand(2, 3, 4), rand(5, 4)
+    a = O.sliced_linear(xx, WW, [0, 1], [4, 4], [5, 5])
+    b = O.sliced_linear(xx, WW, [0, 1], [4, 4], [5, 5], bn=(np.ones(5), np.zeros(5), np.zeros((2, 5)), np.ones((2, 5))))
+    np.testing.assert_array_equal(a, b)
+    mu2 = np.zeros((2, 5)); mu2[1] = 1.0
+    c = O.sliced_linear(xx, WW, [0, 1], [4, 4], [5, 5], bn=(np.ones(5), np.zeros(5), mu2, np.ones((2, 5))))
+    np.testing.assert_array_equal(c[0], a[0])
+    np.testing.assert_allclose(c[1], a[1] - 1.0, rtol=0, atol=1e-15)
+    assert ident.shape == (2, 3, 5)
+
+
 # ------------------------------------------------------------------ routing
 @pytest.mark.parametrize("B,T", [(1, 1), (7, 1), (1, 5), (33, 4), (100, 14), (64, 48)])
 def test_route_invariants(B, T):
