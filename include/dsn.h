@@ -98,7 +98,9 @@ typedef struct dsn_linear_desc {
   const int32_t* k_out; /* host [T], 1..C_out                                            */
   const void* W;        /* device [C_out][ldw]; bf16: 16-byte aligned                    */
   const float* bias;    /* device [C_out] fp32 or NULL                                   */
-  int32_t act;          /* dsn_act                                                       */
+  const float* bn_scale;/* device [T][C_out] fp32 or NULL: per-path affine a_t of Re-SBN (dsn_resbn_fold) */
+  const float* bn_shift;/* device [T][C_out] fp32 (required with bn_scale): b_t          */
+  int32_t act;          /* dsn_act; order of operations: contraction, + bias, * a_t + b_t, activation */
   int32_t in_order;     /* dsn_order of x: INPUT_ORDER [B][R][ldx] by sample, or GROUPED by position */
   int32_t out_order;    /* dsn_order of y                                                */
   int32_t tail;         /* dsn_tail: columns >= k_out[t] left untouched, or zero-filled up to C_out */
@@ -117,6 +119,8 @@ typedef struct dsn_conv_desc {
   const int32_t* k_out; /* host [T]                                                      */
   const void* W;        /* device [C_out][K][K][C_in] bf16, dense, 16-byte aligned, C_in % 8 == 0 */
   const float* bias;
+  const float* bn_scale;/* as in dsn_linear_desc                                         */
+  const float* bn_shift;
   int32_t act;
   int32_t in_order, out_order, tail;
 } dsn_conv_desc;
@@ -182,6 +186,29 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
  * Arguments and results are those of dsn_gate. */
 int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out,
                     float* logits_out, void* stream);
+
+/* Double-headed gate (Sec. 3.5): the routing head of dsn_gate plus the channel-attention head that
+ * shares W1: scale[i][c] = 1 + tanh(b3[c] + sum_j W3[c][j] * ReLU(W1 X_E + b1)[j]), c < c_valid.
+ * W3: device [C_full][C_mlp] fp32, b3: device [C_full] or NULL.  scale_out: device [B][c_valid] fp32.
+ * idx_out / logits_out as in dsn_gate (both heads always run).  Workspace as for dsn_gate. */
+int dsn_gate_attention(dsn_ctx* ctx, const dsn_gate_desc* g, const float* W3, const float* b3, const void* x,
+                       int32_t* idx_out, float* logits_out, float* scale_out, void* workspace, size_t ws_bytes,
+                       void* stream);
+
+/* Applies the attention head: y[p or i][r][c] = x[i][r][c] * scale[i][c] for c < c_valid (bf16 or fp32
+ * activations, fp32 scale).  With r != NULL and to_grouped = 1 the result is written in grouped
+ * order (position p holds sample perm[p]), i.e. the scaling is fused with the gather; otherwise y is
+ * in input order.  x and y may be the same buffer when the order does not change. */
+int dsn_scale_channels(dsn_ctx* ctx, const dsn_routing* r, int32_t to_grouped, int32_t dtype, int32_t B,
+                       int32_t R, int32_t c_valid, const void* x, int64_t ldx, const float* scale, void* y,
+                       int64_t ldy, void* stream);
+
+/* Split batch norm with re-calibration (Sec. 3.3): gamma[:c] * (X - mu_t) / sigma_t + beta[:c] with
+ * per-route statistics.  At inference it is the per-path per-channel affine a_t = gamma / sigma_t,
+ * b_t = beta - gamma * mu_t / sigma_t, which the sliced layers apply in their epilogue
+ * (bn_scale / bn_shift).  gamma, beta: device [C]; mu, sigma: device [T][C]; outputs device [T][C]. */
+int dsn_resbn_fold(dsn_ctx* ctx, int32_t T, int32_t C, const float* gamma, const float* beta, const float* mu,
+                   const float* sigma, float* scale_out, float* shift_out, void* stream);
 
 /* ---- routing (stable grouping by path index; one-hot routing of Sec. 3.1) -------------- */
 /* idx: device [B], values in [0, T).  Fills out->counts/offsets/perm/inv_perm (device arrays the

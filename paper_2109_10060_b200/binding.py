@@ -25,7 +25,7 @@ MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
 
 EXPORTS = [
     "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_widths_from_ratios",
-    "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_route", "dsn_permute_rows",
+    "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
     "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
 ]
@@ -52,16 +52,16 @@ class LinearDesc(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("R", C.c_int32), ("C_in", C.c_int32), ("C_out", C.c_int32),
                 ("ldx", C.c_int64), ("ldw", C.c_int64), ("ldy", C.c_int64), ("T", C.c_int32),
                 ("k_in", C.POINTER(C.c_int32)), ("k_out", C.POINTER(C.c_int32)), ("W", C.c_void_p),
-                ("bias", C.c_void_p), ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32),
-                ("tail", C.c_int32)]
+                ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p), ("act", C.c_int32),
+                ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
 
 
 class ConvDesc(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("H", C.c_int32), ("W_", C.c_int32), ("K", C.c_int32), ("pad", C.c_int32),
                 ("C_in", C.c_int32), ("C_out", C.c_int32), ("ldx", C.c_int64), ("ldy", C.c_int64),
                 ("T", C.c_int32), ("k_in", C.POINTER(C.c_int32)), ("k_out", C.POINTER(C.c_int32)),
-                ("W", C.c_void_p), ("bias", C.c_void_p), ("act", C.c_int32), ("in_order", C.c_int32),
-                ("out_order", C.c_int32), ("tail", C.c_int32)]
+                ("W", C.c_void_p), ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p),
+                ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
 
 
 class LayerDesc(C.Structure):
@@ -94,6 +94,9 @@ def load_library():
     lib.dsn_gate_workspace_bytes.restype = sz
     lib.dsn_gate.argtypes = [vp, C.POINTER(GateDesc), vp, vp, vp, vp, sz, vp]
     lib.dsn_gate_static.argtypes = [vp, C.POINTER(GateDesc), vp, vp, vp, vp]
+    lib.dsn_gate_attention.argtypes = [vp, C.POINTER(GateDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.dsn_scale_channels.argtypes = [vp, C.POINTER(Routing), i32, i32, i32, i32, i32, vp, i64, vp, vp, i64, vp]
+    lib.dsn_resbn_fold.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.dsn_route.argtypes = [vp, vp, i32, i32, C.POINTER(Routing), vp]
     lib.dsn_permute_rows.argtypes = [vp, C.POINTER(Routing), i32, i32, i32, C.POINTER(i32), vp, i64, vp, i64, i32, vp]
     lib.dsn_linear_workspace_bytes.argtypes = [C.POINTER(LinearDesc), i32]
@@ -190,20 +193,23 @@ def make_gate_desc(dtype, B, R, C_full, C_mlp, T, W1, W2, b1=None, b2=None, c_va
 
 
 def make_linear_desc(dtype, R, C_in, C_out, k_in, k_out, W, bias=None, act=ACT_NONE, in_order=INPUT_ORDER,
-                     out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldw=None, ldy=None) -> LinearDesc:
+                     out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldw=None, ldy=None, bn_scale=None,
+                     bn_shift=None) -> LinearDesc:
     ki, ko = _i32_array(k_in), _i32_array(k_out)
     d = LinearDesc(dtype, R, C_in, C_out, C_in if ldx is None else ldx, C_in if ldw is None else ldw,
-                   C_out if ldy is None else ldy, len(k_in), ki, ko, _ptr(W), _ptr(bias), act, in_order, out_order, tail)
-    d._keep = (ki, ko, W, bias)
+                   C_out if ldy is None else ldy, len(k_in), ki, ko, _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift),
+                   act, in_order, out_order, tail)
+    d._keep = (ki, ko, W, bias, bn_scale, bn_shift)
     return d
 
 
 def make_conv_desc(dtype, H, Wd, K, pad, C_in, C_out, k_in, k_out, W, bias=None, act=ACT_NONE,
-                   in_order=INPUT_ORDER, out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldy=None) -> ConvDesc:
+                   in_order=INPUT_ORDER, out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldy=None, bn_scale=None,
+                   bn_shift=None) -> ConvDesc:
     ki, ko = _i32_array(k_in), _i32_array(k_out)
     d = ConvDesc(dtype, H, Wd, K, pad, C_in, C_out, C_in if ldx is None else ldx, C_out if ldy is None else ldy,
-                 len(k_in), ki, ko, _ptr(W), _ptr(bias), act, in_order, out_order, tail)
-    d._keep = (ki, ko, W, bias)
+                 len(k_in), ki, ko, _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift), act, in_order, out_order, tail)
+    d._keep = (ki, ko, W, bias, bn_scale, bn_shift)
     return d
 
 
@@ -235,6 +241,25 @@ def dsn_gate_static(ctx: Context, g: GateDesc, x, idx_out, logits_out=None, stre
     overlap on the device, and problems beyond 1,048,576 scratch floats raise ERR_WORKSPACE."""
     _check(ctx.lib.dsn_gate_static(ctx.handle, C.byref(g), _ptr(x), _ptr(idx_out), _ptr(logits_out),
                                    _stream_handle(stream)), "dsn_gate_static")
+
+
+def dsn_gate_attention(ctx: Context, g: GateDesc, W3, b3, x, idx_out, scale_out, logits_out=None, workspace=None,
+                       stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(ctx.lib.dsn_gate_attention(ctx.handle, C.byref(g), _ptr(W3), _ptr(b3), _ptr(x), _ptr(idx_out),
+                                      _ptr(logits_out), _ptr(scale_out), _ptr(workspace), ws_bytes,
+                                      _stream_handle(stream)), "dsn_gate_attention")
+
+
+def dsn_scale_channels(ctx: Context, routing, to_grouped, dtype, B, R, c_valid, x, ldx, scale, y, ldy, stream=None):
+    _check(ctx.lib.dsn_scale_channels(ctx.handle, C.byref(routing) if routing is not None else None,
+                                      1 if to_grouped else 0, dtype, B, R, c_valid, _ptr(x), ldx, _ptr(scale), _ptr(y),
+                                      ldy, _stream_handle(stream)), "dsn_scale_channels")
+
+
+def dsn_resbn_fold(ctx: Context, T, Cn, gamma, beta, mu, sigma, scale_out, shift_out, stream=None):
+    _check(ctx.lib.dsn_resbn_fold(ctx.handle, T, Cn, _ptr(gamma), _ptr(beta), _ptr(mu), _ptr(sigma), _ptr(scale_out),
+                                  _ptr(shift_out), _stream_handle(stream)), "dsn_resbn_fold")
 
 
 def dsn_route(ctx: Context, idx, B: int, T: int, routing: Routing, stream=None):

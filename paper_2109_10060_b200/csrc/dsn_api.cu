@@ -60,6 +60,7 @@ struct LayerCall {
   const int32_t *k_in, *k_out;
   const void* Wt;
   const float* bias;
+  const float *bn_scale, *bn_shift;
   int act, in_order, out_order, tail;
 };
 
@@ -79,6 +80,7 @@ int check_routing(const dsn_routing* r, int T) {
 
 int validate_call(const LayerCall& c, const dsn_routing* r, const void* x, const void* y) {
   if (!x || !y || !c.Wt) return DSN_ERR_INVALID_ARG;
+  if ((c.bn_scale == nullptr) != (c.bn_shift == nullptr)) return DSN_ERR_INVALID_ARG;
   if (c.dtype != DSN_BF16 && c.dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
   if (c.H < 1 || c.W < 1 || c.C_in < 1 || c.C_out < 1 || c.C_in > 32767 || c.C_out > 32767) return DSN_ERR_INVALID_ARG;
   if (c.act < DSN_ACT_NONE || c.act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
@@ -165,6 +167,9 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
   p.y = static_cast<__nv_bfloat16*>(y);
   p.ldy = c.ldy;
   p.bias = c.bias;
+  p.bn_scale = c.bn_scale;
+  p.bn_shift = c.bn_shift;
+  p.bn_ld = c.C_out;
   p.act = c.act;
   p.status = ctx->d_status;
   for (int t = 0; t < c.T; ++t) {
@@ -263,7 +268,8 @@ int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void
     if (e) return e;
   } else {
     if (dsn_launch_linear_f32(st, c.T, c.H * c.W, static_cast<const float*>(x), c.ldx,
-                              static_cast<const float*>(c.Wt), c.w_row, static_cast<float*>(y), c.ldy, c.bias, c.act,
+                              static_cast<const float*>(c.Wt), c.w_row, static_cast<float*>(y), c.ldy, c.bias, c.bn_scale, c.bn_shift,
+                              c.C_out, c.act,
                               c.in_order == DSN_INPUT_ORDER, c.out_order == DSN_INPUT_ORDER, r->B, r->G, r->offsets,
                               r->perm, r->group_slice, ctx->sm_count, s) != cudaSuccess)
       return DSN_ERR_CUDA;
@@ -285,7 +291,7 @@ LayerCall from_linear(const dsn_linear_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = d->ldw; c.w_tap = d->ldw;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -298,7 +304,7 @@ LayerCall from_conv(const dsn_conv_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = (int64_t)d->K * d->K * d->C_in; c.w_tap = d->C_in;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -486,6 +492,47 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
   if (!aligned16(workspace)) return DSN_ERR_ALIGNMENT;
   if (dsn_launch_gate(*g, x, idx_out, logits_out, static_cast<float*>(workspace), splits, ctx->d_status,
                       as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_gate_attention(dsn_ctx* ctx, const dsn_gate_desc* g, const float* W3, const float* b3, const void* x,
+                       int32_t* idx_out, float* logits_out, float* scale_out, void* workspace, size_t ws_bytes,
+                       void* stream) {
+  if (!W3 || !scale_out) return DSN_ERR_INVALID_ARG;
+  int e = dsn_gate(ctx, g, x, idx_out, logits_out, workspace, ws_bytes, stream);
+  if (e) return e;
+  if (g->B == 0) return DSN_OK;
+  if ((size_t)4 * 4 * g->C_mlp > 48 * 1024) return DSN_ERR_UNSUPPORTED;
+  const int splits = dsn_gate_splits(*g, ctx->sm_count);
+  const float* hid = static_cast<const float*>(workspace) + (size_t)g->B * splits * g->c_valid;
+  if (dsn_launch_gate_attention(*g, hid, W3, b3, scale_out, as_stream(stream)) != cudaSuccess) return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_scale_channels(dsn_ctx* ctx, const dsn_routing* r, int32_t to_grouped, int32_t dtype, int32_t B, int32_t R,
+                       int32_t c_valid, const void* x, int64_t ldx, const float* scale, void* y, int64_t ldy,
+                       void* stream) {
+  if (!ctx || !x || !y || !scale || B < 0 || R < 1 || c_valid < 1 || ldx < c_valid || ldy < c_valid)
+    return DSN_ERR_INVALID_ARG;
+  if (dtype != DSN_BF16 && dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
+  const int32_t* perm = nullptr;
+  if (to_grouped) {
+    if (!r || !r->perm || r->B != B) return DSN_ERR_INVALID_ARG;
+    if (x == y) return DSN_ERR_INVALID_ARG;  // a permutation cannot run in place
+    perm = r->perm;
+  }
+  if (dsn_launch_scale_channels(dtype == DSN_BF16 ? 2 : 4, B, R, c_valid, x, ldx, scale, y, ldy, perm,
+                                as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_resbn_fold(dsn_ctx* ctx, int32_t T, int32_t C, const float* gamma, const float* beta, const float* mu,
+                   const float* sigma, float* scale_out, float* shift_out, void* stream) {
+  if (!ctx || T < 1 || T > DSN_MAX_SLICES || C < 1 || !gamma || !beta || !mu || !sigma || !scale_out || !shift_out)
+    return DSN_ERR_INVALID_ARG;
+  if (dsn_launch_resbn_fold(T * C, C, gamma, beta, mu, sigma, scale_out, shift_out, as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
   return DSN_OK;
 }

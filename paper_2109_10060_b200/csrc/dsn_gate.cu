@@ -279,6 +279,126 @@ gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const 
   }
 }
 
+// Attention head (Sec. 3.5): scale[b][c] = 1 + tanh(b3[c] + sum_j W3[c][j] * hid[b][j]).  A CTA owns
+// kSBSmall samples x 64 channels; their hidden vectors sit in shared memory, a warp walks 8 channels
+// with its lanes across the C_mlp products (16-byte loads of the W3 row when C_mlp % 4 == 0).
+__global__ void __launch_bounds__(kMlpThreads)
+gate_attention_kernel(const float* __restrict__ hid, int B, int C_mlp, int C_full, int c_valid,
+                      const float* __restrict__ W3, const float* __restrict__ b3, float* __restrict__ scale_out) {
+  extern __shared__ __align__(16) float hs[];  // [kSBSmall][C_mlp]
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  const int b0 = blockIdx.x * kSBSmall, c0 = blockIdx.y * 64;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int e = threadIdx.x; e < kSBSmall * C_mlp; e += kMlpThreads) {
+    const int s = e / C_mlp, j = e - s * C_mlp;
+    hs[e] = (b0 + s < B) ? hid[(int64_t)(b0 + s) * C_mlp + j] : 0.f;
+  }
+  __syncthreads();
+  const bool vec = (C_mlp % 4 == 0) && ((reinterpret_cast<uintptr_t>(W3) & 15) == 0);
+  for (int u = 0; u < 8; ++u) {
+    const int c = c0 + warp * 8 + u;
+    if (c >= c_valid) break;  // warp-uniform
+    float acc[kSBSmall];
+#pragma unroll
+    for (int s = 0; s < kSBSmall; ++s) acc[s] = 0.f;
+    const float* w = W3 + (int64_t)c * C_mlp;
+    if (vec) {
+      for (int j4 = lane; j4 < (C_mlp >> 2); j4 += 32) {
+        const float4 wv = __ldg(reinterpret_cast<const float4*>(w) + j4);
+#pragma unroll
+        for (int s = 0; s < kSBSmall; ++s) {
+          const float4 hv = reinterpret_cast<const float4*>(hs + s * C_mlp)[j4];
+          acc[s] = fmaf(wv.x, hv.x, acc[s]); acc[s] = fmaf(wv.y, hv.y, acc[s]);
+          acc[s] = fmaf(wv.z, hv.z, acc[s]); acc[s] = fmaf(wv.w, hv.w, acc[s]);
+        }
+      }
+    } else {
+      for (int j = lane; j < C_mlp; j += 32) {
+        const float wv = __ldg(w + j);
+#pragma unroll
+        for (int s = 0; s < kSBSmall; ++s) acc[s] = fmaf(wv, hs[s * C_mlp + j], acc[s]);
+      }
+    }
+#pragma unroll
+    for (int s = 0; s < kSBSmall; ++s) {
+      float v = acc[s];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0 && b0 + s < B) scale_out[(int64_t)(b0 + s) * c_valid + c] = 1.f + tanhf(v + (b3 ? b3[c] : 0.f));
+    }
+  }
+  (void)C_full;
+}
+
+// y = x * scale[sample][channel]; one CTA per (row band, sample); grouped output when perm is given.
+template <typename Tio>
+__global__ void __launch_bounds__(256)
+scale_channels_kernel(const Tio* __restrict__ x, int64_t ldx, const float* __restrict__ scale, Tio* __restrict__ y,
+                      int64_t ldy, int R, int c_valid, int bands, const int32_t* __restrict__ perm) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  const int pos = blockIdx.y, band = blockIdx.x;
+  const int smp = perm ? perm[pos] : pos;   // output position pos holds sample smp
+  if (smp < 0) return;
+  const int r0 = (int)(((int64_t)R * band) / bands), r1 = (int)(((int64_t)R * (band + 1)) / bands);
+  const Tio* xs = x + (int64_t)smp * R * ldx;
+  Tio* ys = y + (int64_t)pos * R * ldy;
+  const float* sc = scale + (int64_t)smp * c_valid;
+  const int64_t total = (int64_t)(r1 - r0) * c_valid;
+  for (int64_t e = threadIdx.x; e < total; e += 256) {
+    const int r = r0 + (int)(e / c_valid), c = (int)(e % c_valid);
+    ys[(int64_t)r * ldy + c] = (Tio)((float)xs[(int64_t)r * ldx + c] * __ldg(sc + c));
+  }
+}
+
+// bf16, c_valid % 8 == 0, 16-byte aligned rows: eight channels per thread
+__global__ void __launch_bounds__(256)
+scale_channels_bf16_vec_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const float* __restrict__ scale,
+                               __nv_bfloat16* __restrict__ y, int64_t ldy, int R, int c_valid, int bands,
+                               const int32_t* __restrict__ perm) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  const int pos = blockIdx.y, band = blockIdx.x;
+  const int smp = perm ? perm[pos] : pos;
+  if (smp < 0) return;
+  const int r0 = (int)(((int64_t)R * band) / bands), r1 = (int)(((int64_t)R * (band + 1)) / bands);
+  const int nvec = c_valid >> 3;
+  const uint4* xs = reinterpret_cast<const uint4*>(x + (int64_t)smp * R * ldx);
+  uint4* ys = reinterpret_cast<uint4*>(y + (int64_t)pos * R * ldy);
+  const float* sc = scale + (int64_t)smp * c_valid;
+  const int64_t total = (int64_t)(r1 - r0) * nvec, sx = ldx >> 3, sy = ldy >> 3;
+  for (int64_t e = threadIdx.x; e < total; e += 256) {
+    const int r = r0 + (int)(e / nvec), v = (int)(e % nvec);
+    const uint4 in = __ldg(xs + (int64_t)r * sx + v);
+    const float4 s0 = __ldg(reinterpret_cast<const float4*>(sc) + 2 * v), s1 = __ldg(reinterpret_cast<const float4*>(sc) + 2 * v + 1);
+    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = __uint_as_float(w[j] << 16) * sv[2 * j], b = __uint_as_float(w[j] & 0xffff0000u) * sv[2 * j + 1];
+      __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+      o[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    ys[(int64_t)r * sy + v] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// a_t = gamma / sigma_t, b_t = beta - gamma * mu_t / sigma_t
+__global__ void resbn_fold_kernel(int n, int C, const float* __restrict__ gamma, const float* __restrict__ beta,
+                                  const float* __restrict__ mu, const float* __restrict__ sigma,
+                                  float* __restrict__ scale_out, float* __restrict__ shift_out) {
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n) return;
+  const int c = e % C;
+  const float a = gamma[c] / sigma[e];
+  scale_out[e] = a;
+  shift_out[e] = fmaf(-a, mu[e], beta[c]);
+}
+
 }  // namespace
 
 int dsn_gate_splits(const dsn_gate_desc& g, int sm_count) {
@@ -394,4 +514,37 @@ extern "C" int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void*
                       static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
   return DSN_OK;
+}
+
+cudaError_t dsn_launch_gate_attention(const dsn_gate_desc& g, const float* hid, const float* W3, const float* b3,
+                                      float* scale_out, cudaStream_t s) {
+  dim3 grid((g.B + kSBSmall - 1) / kSBSmall, (g.c_valid + 63) / 64);
+  return dsn_launch(gate_attention_kernel, grid, dim3(kMlpThreads), sizeof(float) * kSBSmall * g.C_mlp, s, 1, hid, g.B,
+                    g.C_mlp, g.C_full, g.c_valid, W3, b3, scale_out);
+}
+
+cudaError_t dsn_launch_scale_channels(int elem_bytes, int B, int R, int c_valid, const void* x, int64_t ldx,
+                                      const float* scale, void* y, int64_t ldy, const int32_t* perm_or_null,
+                                      cudaStream_t s) {
+  if (B == 0) return cudaSuccess;
+  int bands = R / 16 > 0 ? R / 16 : 1;
+  if (bands > 16) bands = 16;
+  dim3 grid(bands, B);
+  const bool vec = elem_bytes == 2 && c_valid % 8 == 0 && ldx % 8 == 0 && ldy % 8 == 0 &&
+                   ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(scale)) & 15) == 0;
+  if (vec)
+    return dsn_launch(scale_channels_bf16_vec_kernel, grid, dim3(256), 0, s, 1, static_cast<const __nv_bfloat16*>(x), ldx,
+                      scale, static_cast<__nv_bfloat16*>(y), ldy, R, c_valid, bands, perm_or_null);
+  if (elem_bytes == 2)
+    return dsn_launch(scale_channels_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, 1, static_cast<const __nv_bfloat16*>(x),
+                      ldx, scale, static_cast<__nv_bfloat16*>(y), ldy, R, c_valid, bands, perm_or_null);
+  return dsn_launch(scale_channels_kernel<float>, grid, dim3(256), 0, s, 1, static_cast<const float*>(x), ldx, scale,
+                    static_cast<float*>(y), ldy, R, c_valid, bands, perm_or_null);
+}
+
+cudaError_t dsn_launch_resbn_fold(int n, int C, const float* gamma, const float* beta, const float* mu,
+                                  const float* sigma, float* scale_out, float* shift_out, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  return dsn_launch(resbn_fold_kernel, dim3((n + 255) / 256), dim3(256), 0, s, 1, n, C, gamma, beta, mu, sigma, scale_out,
+                    shift_out);
 }

@@ -33,7 +33,7 @@ using namespace dsn_gemm;
 
 // ---------------------------------------------------------------------------------- tile decode
 struct TileInfo {
-  int map, ki, ko, n0;
+  int map, ki, ko, n0, slice;
   int p_end;            // one past the group's last grouped position
   int row0, rows_end;   // flat: first grouped row of the tile, one past the group's last row
   int b0, x0, y0;       // per-image tiling: first position, pixel origin
@@ -45,6 +45,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int32
   const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
   const int grp = p.G - 1 - j;
   const int sl = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
+  t.slice = sl;
   t.map = p.map_id[sl];
   t.ki = p.k_in[sl];
   t.ko = p.k_out[sl];
@@ -248,6 +249,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       }
       __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
+      const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       // output rows this lane writes in the direct-store phase: row 4*i + lane/8 of the warp's 32 rows
@@ -270,11 +273,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
       const CUtensorMap* mY = &p.mapY[t.map];
       if (p.act == DSN_ACT_NONE)
-        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       else if (p.act == DSN_ACT_RELU)
-        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       else
-        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);

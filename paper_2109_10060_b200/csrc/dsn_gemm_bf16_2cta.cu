@@ -84,7 +84,7 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 
 struct PairTile {
-  int map, ki, ko, n0;
+  int map, ki, ko, n0, slice;
   int p_end;
   int row0, rows_end;
   int b0, x0, y0;
@@ -98,6 +98,7 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const 
   const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
   const int grp = p.G - 1 - j;
   const int sl = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
+  t.slice = sl;
   t.map = p.map_id[sl];
   t.ki = p.k_in[sl];
   t.ko = p.k_out[sl];
@@ -299,6 +300,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
       }
       __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
+      const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       __nv_bfloat16* rp[8];
@@ -316,11 +319,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
       const CUtensorMap* mY = &p.mapY[t.map];
       if (p.act == DSN_ACT_NONE)
-        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       else if (p.act == DSN_ACT_RELU)
-        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       else
-        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, stage_w, rp, lane, contig, mY, (int)base_row);
+        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it

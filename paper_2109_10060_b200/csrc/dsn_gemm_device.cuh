@@ -184,7 +184,7 @@ __device__ __forceinline__ float apply_act(float v) {
 // lanes store one 128-byte piece of a row each.
 template <int ACT>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
-                                              uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
+                                              const float* sc_row, const float* sh_row, uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
                                               const CUtensorMap* mapY, int base_row) {
   for (int c0 = 64 * first; c0 < ncols; c0 += 128) {
     // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
@@ -209,6 +209,10 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
             if (brow) {
               if (cb + c < ncols) a += __ldg(brow + cb + c);
               if (cb + c + 1 < ncols) b += __ldg(brow + cb + c + 1);
+            }
+            if (sc_row) {  // Re-SBN of this tile's path: per-channel scale and shift
+              if (cb + c < ncols) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
+              if (cb + c + 1 < ncols) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
             }
             __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
             w[e] = *reinterpret_cast<uint32_t*>(&h);

@@ -101,6 +101,9 @@ struct GemmParams {
   __nv_bfloat16* y;
   int64_t ldy;
   const float* bias;
+  const float* bn_scale;  // [T][bn_ld] per-path affine of Re-SBN, or nullptr
+  const float* bn_shift;
+  int32_t bn_ld;
   int32_t act;
   int32_t* status;
 };
@@ -115,6 +118,14 @@ int dsn_gemm_pair_max_clusters(size_t smem_bytes);
 cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_out, float* logits_out,
                             float* partial, int splits, int32_t* status, cudaStream_t s);
 int dsn_gate_splits(const dsn_gate_desc& g, int sm_count);
+// attention head: hid = partial + B*splits*c_valid (written by dsn_launch_gate on the same stream)
+cudaError_t dsn_launch_gate_attention(const dsn_gate_desc& g, const float* hid, const float* W3, const float* b3,
+                                      float* scale_out, cudaStream_t s);
+cudaError_t dsn_launch_scale_channels(int elem_bytes, int B, int R, int c_valid, const void* x, int64_t ldx,
+                                      const float* scale, void* y, int64_t ldy, const int32_t* perm_or_null,
+                                      cudaStream_t s);
+cudaError_t dsn_launch_resbn_fold(int n, int C, const float* gamma, const float* beta, const float* mu,
+                                  const float* sigma, float* scale_out, float* shift_out, cudaStream_t s);
 
 cudaError_t dsn_launch_route(const int32_t* idx, int B, int T, int32_t* counts, int32_t* offsets,
                              int32_t* perm, int32_t* inv_perm, int32_t* status, cudaStream_t s);
@@ -126,7 +137,7 @@ struct SliceTable {
 
 cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const float* x, int64_t ldx,
                                   const float* W, int64_t ldw, float* y, int64_t ldy, const float* bias,
-                                  int act, int x_input_order, int y_input_order, int B, int G,
+                                  const float* bn_scale, const float* bn_shift, int bn_ld, int act, int x_input_order, int y_input_order, int B, int G,
                                   const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                   int sm_count, cudaStream_t s);
 
