@@ -12,7 +12,7 @@ Passages followed (DS-Net++, "Dynamic Weight Slicing"):
   * dynamic network = route picked per input .......... Eq. (dyn_net), Sec. 3.1
   * weight slicing  psi(x) = W[:k] x ................... Eq. (weight_slicing), Sec. 3.2
   * slice-able convolution W[:c_O, :c_I] * X ........... Sec. 3.3, "Filter number"
-  * ViT QKV / proj / MLP slicing ....................... Sec. 3.4, Eq. (slimmableMLP)
+  * ViT QKV / proj / MLP slicing, self-attention ....... Sec. 3.4, Eq. (slimmableMLP)
   * gate: average-pool encoder, two-layer MLP, one-hot . Sec. 3.5
   * gate attention head X * (1 + tanh(W3 ReLU(W1 X_E))) . Sec. 3.5, "double-headed dynamic gate"
   * split batch norm with re-calibration (Re-SBN) ...... Sec. 3.3
@@ -264,6 +264,29 @@ def vit_qkv(x, Wq, Wk, Wv, idx, paths, D_h, samples=None):
     k_in = [p[0] for p in paths]
     k_out = [p[1] * D_h for p in paths]
     return tuple(sliced_linear(x, Wm, idx, k_in, k_out, samples=samples) for Wm in (Wq, Wk, Wv))
+
+
+def attention(q, k, v, idx, heads, D_h, samples=None, fill=np.nan):
+    """Slimmable self-attention (Sec. 3.4): for every sample with h = heads[idx] heads,
+    A_a = Softmax(Q_a K_a^T / sqrt(D_h)) V_a for a < h, output = Concat(A_0 .. A_{h-1}).
+
+    q, k, v [B][N][H*D_h] (head a occupies columns a*D_h .. (a+1)*D_h - 1).  Returns [B][N][H*D_h] with
+    the columns of heads >= h holding `fill`.
+    """
+    q, k, v = (np.asarray(a, dtype=F64) for a in (q, k, v))
+    B, N, HD = q.shape
+    out = np.full((B, N, HD), fill, dtype=F64)
+    todo = range(B) if samples is None else samples
+    for i in todo:
+        h = int(heads[int(idx[i])])
+        for a in range(h):
+            sl = slice(a * D_h, (a + 1) * D_h)
+            s = q[i, :, sl] @ k[i, :, sl].T / np.sqrt(D_h)
+            s = s - s.max(axis=1, keepdims=True)          # softmax over the keys, row by row
+            p = np.exp(s)
+            p = p / p.sum(axis=1, keepdims=True)
+            out[i, :, sl] = p @ v[i, :, sl]
+    return out
 
 
 def vit_mlp(x, Wfc1, Wfc2, idx, paths, mirror_bf16=True, samples=None):

@@ -402,6 +402,32 @@ def test_vit_pieces_against_library():
         np.testing.assert_allclose(out[i, :, :de], orf.numpy(), rtol=1e-11, atol=1e-12)
 
 
+def test_attention_library_brute_force_and_closed_forms():
+    B, N, H, Dh = 3, 7, 4, 5
+    q, k, v = rand(B, N, H * Dh), rand(B, N, H * Dh), rand(B, N, H * Dh)
+    heads, idx = [2, 4, 1], np.array([1, 0, 2])
+    out = O.attention(q, k, v, idx, heads, Dh)
+    for i in range(B):
+        h = heads[idx[i]]
+        qt, kt, vt = (torch.from_numpy(a[i].reshape(N, H, Dh)[:, :h].transpose(1, 0, 2).copy()) for a in (q, k, v))
+        ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt)       # [h][N][Dh], scale 1/sqrt(Dh)
+        np.testing.assert_allclose(out[i, :, :h * Dh], ref.permute(1, 0, 2).reshape(N, h * Dh).numpy(), rtol=1e-11, atol=1e-12)
+        assert np.all(np.isnan(out[i, :, h * Dh:]))
+    # brute force for one (sample, head, query)
+    i, a, n = 1, 3, 2
+    s = [sum(q[i, n, a * Dh + d] * k[i, m, a * Dh + d] for d in range(Dh)) / math.sqrt(Dh) for m in range(N)]
+    e = [math.exp(x - max(s)) for x in s]
+    for d in range(Dh):
+        want = sum(e[m] / sum(e) * v[i, m, a * Dh + d] for m in range(N))
+        assert abs(out[i, n, a * Dh + d] - want) < 1e-12
+    # zero queries give uniform attention: the mean of the values; one dominant key copies its value
+    o0 = O.attention(np.zeros_like(q), k, v, np.zeros(B, int), [H], Dh)
+    np.testing.assert_allclose(o0, np.broadcast_to(v.mean(axis=1, keepdims=True), v.shape), rtol=1e-12, atol=1e-12)
+    kk = np.zeros((1, N, Dh)); kk[0, 3] = 50.0
+    o1 = O.attention(np.ones((1, N, Dh)), kk, v[:1, :, :Dh], [0], [1], Dh)
+    np.testing.assert_allclose(o1[0], np.broadcast_to(v[0, 3, :Dh], (N, Dh)), rtol=1e-9, atol=1e-9)
+
+
 def test_executed_macs_closed_form():
     idx = np.array([0, 2, 2, 1, 0, 2])
     k_in, k_out, R = [4, 8, 16], [3, 6, 9], 7
