@@ -414,7 +414,7 @@ def test_attention_library_brute_force_and_closed_forms():
         np.testing.assert_allclose(out[i, :, :h * Dh], ref.permute(1, 0, 2).reshape(N, h * Dh).numpy(), rtol=1e-11, atol=1e-12)
         assert np.all(np.isnan(out[i, :, h * Dh:]))
     # brute force for one (sample, head, query)
-    i, a, n = 1, 3, 2
+    i, a, n = 0, 3, 2
     s = [sum(q[i, n, a * Dh + d] * k[i, m, a * Dh + d] for d in range(Dh)) / math.sqrt(Dh) for m in range(N)]
     e = [math.exp(x - max(s)) for x in s]
     for d in range(Dh):
