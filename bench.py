@@ -377,6 +377,27 @@ def run_table(args):
     for lname, Cin, Cout, act in (("qkv", 384, 1152, 0), ("proj", 384, 384, 0), ("fc1", 384, 1536, 2), ("fc2", 1536, 384, 0)):
         ki, ko = wl.vit_layer_slices(paths, 64, lname)
         layer("cfg3", lname, "uniform", B, 197, Cin, Cout, ki, ko, idx, act=act)
+    def attention(cfgname, B, N, H, heads, idx, rname):
+        T = len(heads)
+        r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
+        dsn.dsn_route(ctx, ints(idx), B, T, r)
+        per = B * N * 4 * H * 64 * 2
+        nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
+        qs = [torch.randn(B, N, 3 * H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        os_ = [torch.zeros(B, N, H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        d = dsn.make_attention_desc(N, H, 64, heads, order=dsn.GROUPED)
+        us = graph_time(lambda i: dsn.dsn_sliced_attention(ctx, d, r, qs[i % nbuf], os_[i % nbuf]), nbuf)
+        assert ctx.get_status()[0] == 0
+        hsum = sum(heads[t] for t in idx)
+        flops = 4.0 * N * N * 64 * hsum
+        byts = 2.0 * N * 4 * 64 * hsum
+        tf = flops / us / 1e6
+        bound = min(PEAK, flops / byts * HBM / 1e3)
+        print(f"| {cfgname} | attention core (N={N}) | {rname} | {us:.1f} | {tf:.0f} | {100 * tf / PEAK:.1f} | {bound:.0f} | "
+              f"{100 * tf / bound:.0f} | {byts / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
+
+    attention("cfg3", 256, 197, 6, [p_[1] for p_ in wl.vit_small_paths()], wl.idx_quota_uniform(wl.rng(3, 9), 256, 48), "uniform")
+    attention("cfg5", 1024, 197, 12, [p_[1] for p_ in wl.vit_base_paths()], wl.idx_quota_uniform(wl.rng(5, 9), 1024, 8), "uniform")
     # config 5: ViT-B width
     B, paths = 1024, wl.vit_base_paths()
     gate_route("cfg5", B, 197, 768, 8)

@@ -125,6 +125,21 @@ typedef struct dsn_conv_desc {
   int32_t in_order, out_order, tail;
 } dsn_conv_desc;
 
+/* Slimmable self-attention core (Sec. 3.4): A_a = Softmax(Q_a K_a^T / sqrt(D_h)) V_a for the h heads of
+ * the sample's path, concatenated.  qkv rows are laid out [head][q|k|v][D_h] (the output of the sliced
+ * QKV layer with the head-major fused weight), out rows [head][D_h]; heads >= h are neither read nor
+ * written.  qkv and out are both in `order` (all rows of a sample are contiguous either way). */
+typedef struct dsn_attention_desc {
+  int32_t dtype;        /* DSN_BF16                                                      */
+  int32_t N;            /* tokens per sample, 1..256                                     */
+  int32_t H, D_h;       /* full head count; head dimension (64)                          */
+  int64_t ld_qkv;       /* elements between rows of qkv, >= 3*H*D_h, multiple of 8       */
+  int64_t ld_out;       /* elements between rows of out, >= H*D_h, multiple of 8         */
+  int32_t T;
+  const int32_t* heads; /* host [T]: head count of each path, 1..H                       */
+  int32_t order;        /* dsn_order of qkv and out                                      */
+} dsn_attention_desc;
+
 /* One dynamic block: optional gate, routing, then up to DSN_MAX_CHAIN layers that all inherit
  * the block's routing (Sec. 5, "inherit the control signal").  Layer j reads layer j-1's output;
  * layer 0 reads x in input order, the last layer writes y in input order; intermediate
@@ -233,6 +248,11 @@ int dsn_sliced_linear(dsn_ctx* ctx, const dsn_linear_desc* d, const dsn_routing*
                       void* y, void* workspace, size_t ws_bytes, void* stream);
 int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, const void* x,
                     void* y, void* workspace, size_t ws_bytes, void* stream);
+
+/* qkv, out: device bf16, 16-byte aligned.  fp32 scores and softmax, bf16 probabilities for the
+ * second contraction, bf16 output. */
+int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_routing* r, const void* qkv,
+                         void* out, void* stream);
 
 /* ---- whole dynamic block (Eq. (dyn_net)) ------------------------------------------------ */
 size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L);

@@ -26,7 +26,7 @@ MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
 EXPORTS = [
     "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_widths_from_ratios",
     "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
-    "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
+    "dsn_sliced_attention", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
 ]
 
@@ -62,6 +62,11 @@ class ConvDesc(C.Structure):
                 ("T", C.c_int32), ("k_in", C.POINTER(C.c_int32)), ("k_out", C.POINTER(C.c_int32)),
                 ("W", C.c_void_p), ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p),
                 ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
+
+
+class AttentionDesc(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D_h", C.c_int32), ("ld_qkv", C.c_int64),
+                ("ld_out", C.c_int64), ("T", C.c_int32), ("heads", C.POINTER(C.c_int32)), ("order", C.c_int32)]
 
 
 class LayerDesc(C.Structure):
@@ -105,6 +110,7 @@ def load_library():
     lib.dsn_conv_workspace_bytes.restype = sz
     lib.dsn_sliced_linear.argtypes = [vp, C.POINTER(LinearDesc), C.POINTER(Routing), vp, vp, vp, sz, vp]
     lib.dsn_sliced_conv.argtypes = [vp, C.POINTER(ConvDesc), C.POINTER(Routing), vp, vp, vp, sz, vp]
+    lib.dsn_sliced_attention.argtypes = [vp, C.POINTER(AttentionDesc), C.POINTER(Routing), vp, vp, vp]
     lib.dsn_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
     lib.dsn_layer_workspace_bytes.restype = sz
     lib.dsn_layer_forward.argtypes = [vp, C.POINTER(LayerDesc), vp, vp, vp, C.POINTER(Routing), vp, vp, sz, vp]
@@ -282,6 +288,19 @@ def dsn_sliced_conv(ctx: Context, d: ConvDesc, routing: Routing, x, y, workspace
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(ctx.lib.dsn_sliced_conv(ctx.handle, C.byref(d), C.byref(routing), _ptr(x), _ptr(y), _ptr(workspace),
                                    ws_bytes, _stream_handle(stream)), "dsn_sliced_conv")
+
+
+def make_attention_desc(N, H, D_h, heads, order=INPUT_ORDER, ld_qkv=None, ld_out=None) -> AttentionDesc:
+    hs = _i32_array(heads)
+    d = AttentionDesc(BF16, N, H, D_h, 3 * H * D_h if ld_qkv is None else ld_qkv, H * D_h if ld_out is None else ld_out,
+                      len(heads), hs, order)
+    d._keep = (hs,)
+    return d
+
+
+def dsn_sliced_attention(ctx: Context, d: AttentionDesc, routing: Routing, qkv, out, stream=None):
+    _check(ctx.lib.dsn_sliced_attention(ctx.handle, C.byref(d), C.byref(routing), _ptr(qkv), _ptr(out),
+                                        _stream_handle(stream)), "dsn_sliced_attention")
 
 
 def dsn_layer_workspace_bytes(L: LayerDesc) -> int:

@@ -591,6 +591,33 @@ int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, 
   return run_layer(ctx, from_conv(d), r, x, y, as_stream(stream));
 }
 
+int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_routing* r, const void* qkv, void* out,
+                         void* stream) {
+  if (!ctx || !d || !qkv || !out || !d->heads) return DSN_ERR_INVALID_ARG;
+  if (d->dtype != DSN_BF16 || d->D_h != 64 || d->N > 256) return DSN_ERR_UNSUPPORTED;
+  if (d->N < 1 || d->H < 1 || d->H > 64 || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (d->ld_qkv < (int64_t)3 * d->H * d->D_h || d->ld_out < (int64_t)d->H * d->D_h) return DSN_ERR_INVALID_ARG;
+  if (d->order != DSN_INPUT_ORDER && d->order != DSN_GROUPED) return DSN_ERR_INVALID_ARG;
+  for (int t = 0; t < d->T; ++t)
+    if (d->heads[t] < 1 || d->heads[t] > d->H) return DSN_ERR_INVALID_ARG;
+  int e = check_routing(r, d->T);
+  if (e) return e;
+  if (!aligned16(qkv) || !aligned16(out) || d->ld_qkv % 8 || d->ld_out % 8) return DSN_ERR_ALIGNMENT;
+  if (r->B == 0) return DSN_OK;
+  if ((int64_t)r->B * d->N > 0x7fffffffLL) return DSN_ERR_INVALID_ARG;
+  CUtensorMap map;
+  const uint64_t dims[3] = {64, (uint64_t)3 * d->H, (uint64_t)r->B * d->N};
+  const uint64_t str[2] = {128, (uint64_t)d->ld_qkv * 2};
+  const uint32_t box[3] = {64, 1, 128};
+  e = encode_map(ctx, &map, qkv, 3, dims, str, box);
+  if (e) return e;
+  if (dsn_launch_attention(map, d->heads, d->T, d->N, d->H, r->B, r->G, d->order == DSN_GROUPED, r->offsets, r->perm,
+                           r->group_slice, qkv, d->ld_qkv, out, d->ld_out, ctx->d_status, as_stream(stream)) !=
+      cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
 size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L) {
   LayerPlan pl;
   if (plan_layer(L, pl)) return 0;

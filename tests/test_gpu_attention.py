@@ -1,0 +1,107 @@
+"""GPU parity of the slimmable self-attention core against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import dsn_workloads as wl
+from oracle import dsn_oracle as O
+from gpu_util import DEV, SENTINEL, check_status, down, route_on_gpu, up_bf16
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3   # max|err| / max|ref| per sample; probabilities are rounded to bf16 before the second product
+
+
+@pytest.fixture(scope="module")
+def ctx(dsn):
+    return dsn.Context(0)
+
+
+def head_major(q, k, v, H, Dh):
+    """[B][N][H*Dh] x3 -> [B][N][H][3][Dh] flattened: the fused QKV layer's output layout."""
+    B, N, _ = q.shape
+    st = np.stack([q.reshape(B, N, H, Dh), k.reshape(B, N, H, Dh), v.reshape(B, N, H, Dh)], axis=3)
+    return np.ascontiguousarray(st.reshape(B, N, 3 * H * Dh))
+
+
+@pytest.mark.parametrize("B,N,H,heads,order", [(24, 197, 6, [3, 4, 5, 6], 0), (24, 197, 6, [3, 4, 5, 6], 1),
+                                               (10, 197, 12, [5, 6, 7, 8, 9, 10, 11, 12], 1), (6, 64, 4, [1, 4], 0),
+                                               (5, 256, 2, [2, 1], 1), (7, 130, 3, [3], 0), (4, 16, 2, [2, 1], 0)])
+def test_attention_matches_oracle(dsn, ctx, B, N, H, heads, order):
+    g = np.random.default_rng(B * 1000 + N + H)
+    Dh, T = 64, len(heads)
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    q, k, v = (wl.normal(g, (B, N, H * Dh)) for _ in range(3))
+    q = wl.to_bf16_values(q * 1.5)                      # sharper softmax than unit-variance scores
+    qkv = head_major(q, k, v, H, Dh)
+    r = route_on_gpu(dsn, ctx, idx, T)
+    perm = O.route(idx, T)[2]
+    src = qkv[perm] if order else qkv
+    out = torch.full((B, N, H * Dh), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    d = dsn.make_attention_desc(N, H, Dh, heads, order=order)
+    dsn.dsn_sliced_attention(ctx, d, r, up_bf16(src), out)
+    check_status(ctx, dsn)
+    got = down(out)
+    if order:
+        tmp = np.empty_like(got)
+        tmp[perm] = got
+        got = tmp
+    ref = O.attention(q, k, v, idx, heads, Dh)
+    for i in range(B):
+        w = heads[idx[i]] * Dh
+        err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
+        assert err <= TOL, (i, int(idx[i]), err)
+        assert np.all(got[i, :, w:] == SENTINEL)          # heads the path does not have stay untouched
+
+
+def test_attention_closed_forms_on_device(dsn, ctx):
+    """Zero queries -> every output row is the mean of the values; a dominant key copies its value."""
+    B, N, H, Dh = 2, 197, 2, 64
+    g = np.random.default_rng(3)
+    v = wl.normal(g, (B, N, H * Dh))
+    k = wl.normal(g, (B, N, H * Dh))
+    q = np.zeros((B, N, H * Dh), np.float32)
+    k[1] = 0.0
+    k[1, 100] = 8.0                                       # with q = 8: score 64*64/8 = 512 above all others
+    q[1] = 8.0
+    r = route_on_gpu(dsn, ctx, np.zeros(B, np.int32), 1)
+    out = torch.zeros((B, N, H * Dh), dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(N, H, Dh, [H]), r, up_bf16(head_major(q, k, v, H, Dh)), out)
+    check_status(ctx, dsn)
+    got = down(out)
+    mean = v[0].astype(np.float64).mean(axis=0)
+    assert np.max(np.abs(got[0] - mean)) <= 5e-3
+    np.testing.assert_array_equal(got[1], np.broadcast_to(v[1, 100].astype(np.float64), (N, H * Dh)))
+
+
+def test_vit_block_qkv_attention_proj_chain(dsn, ctx):
+    """QKV layer -> attention -> projection in grouped order with one routing: the path through a ViT
+    block's attention half, against the oracle evaluated on the device's own QKV output."""
+    cfg = wl.config3(B=32, routing="iid")
+    B, R, De, H, Dh, T, paths = cfg["B"], cfg["R"], cfg["D_e"], cfg["H"], cfg["D_h"], cfg["T"], cfg["paths"]
+    heads = [p[1] for p in paths]
+    r = route_on_gpu(dsn, ctx, cfg["idx"], T)
+    kq, koq = wl.vit_layer_slices(paths, Dh, "qkv")
+    kp, kop = wl.vit_layer_slices(paths, Dh, "proj")
+    Wf = up_bf16(wl.pack_qkv_head_major(cfg["Wq"], cfg["Wk"], cfg["Wv"], Dh))
+    qkv = torch.zeros((B, R, 3 * H * Dh), dtype=torch.bfloat16, device=DEV)
+    att = torch.zeros((B, R, H * Dh), dtype=torch.bfloat16, device=DEV)
+    y = torch.full((B, R, De), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(dsn.BF16, R, De, 3 * H * Dh, kq, koq, Wf, out_order=dsn.GROUPED), r,
+                          up_bf16(cfg["x"]), qkv)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(R, H, Dh, heads, order=dsn.GROUPED), r, qkv, att)
+    dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(dsn.BF16, R, H * Dh, De, kp, kop, up_bf16(cfg["Wproj"]),
+                                                    in_order=dsn.GROUPED), r, att, y)
+    check_status(ctx, dsn)
+    perm = O.route(cfg["idx"], T)[2]
+    qkv_in = np.empty((B, R, 3 * H * Dh))
+    qkv_in[perm] = down(qkv)                                    # device QKV, back in input order
+    five = qkv_in.reshape(B, R, H, 3, Dh)
+    q, k, v = (np.nan_to_num(five[:, :, :, w].reshape(B, R, H * Dh)) for w in range(3))
+    a_ref = O.round_bf16(O.attention(q, k, v, cfg["idx"], heads, Dh, fill=0.0))
+    ref = O.round_bf16(O.sliced_linear(a_ref, cfg["Wproj"], cfg["idx"], kp, kop))
+    got = down(y)
+    for i in range(B):
+        w = kop[cfg["idx"][i]]
+        err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
+        assert err <= 1e-2, (i, err)                            # two chained bf16 stages after the QKV layer
+        assert np.all(got[i, :, w:] == SENTINEL)
