@@ -48,7 +48,7 @@ enum dsn_dtype { DSN_F32 = 0, DSN_BF16 = 1 };
 enum dsn_act { DSN_ACT_NONE = 0, DSN_ACT_RELU = 1, DSN_ACT_GELU = 2 /* exact erf form */ };
 enum dsn_order { DSN_INPUT_ORDER = 0, DSN_GROUPED = 1 };
 enum dsn_tail { DSN_TAIL_UNTOUCHED = 0, DSN_TAIL_ZERO = 1 };
-enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1 };
+enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1, DSN_LAYER_ATTENTION = 2 };
 
 #define DSN_MAX_SLICES 64   /* largest T                                               */
 #define DSN_MAX_GROUPS 4096 /* largest G of a caller-built group list                  */
@@ -150,7 +150,8 @@ typedef struct dsn_layer_desc {
   int32_t T;
   int32_t n_layers;                 /* 1..DSN_MAX_CHAIN                                  */
   int32_t kind[DSN_MAX_CHAIN];      /* dsn_layer_kind                                    */
-  const void* layer[DSN_MAX_CHAIN]; /* dsn_linear_desc* or dsn_conv_desc* (order fields are ignored) */
+  const void* layer[DSN_MAX_CHAIN]; /* dsn_linear_desc*, dsn_conv_desc* or (between two layers) dsn_attention_desc*;
+                                       order and leading-dimension fields of chained elements are ignored */
 } dsn_layer_desc;
 
 /* ---- context ------------------------------------------------------------------------- */

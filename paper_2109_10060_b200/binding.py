@@ -20,7 +20,7 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
 INPUT_ORDER, GROUPED = 0, 1
 TAIL_UNTOUCHED, TAIL_ZERO = 0, 1
-LAYER_LINEAR, LAYER_CONV = 0, 1
+LAYER_LINEAR, LAYER_CONV, LAYER_ATTENTION = 0, 1, 2
 MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
 
 EXPORTS = [
@@ -224,7 +224,7 @@ def make_layer_desc(B, T, layers, gate: Optional[GateDesc] = None) -> LayerDesc:
     L.gate = C.pointer(gate) if gate is not None else None
     L.B, L.T, L.n_layers = B, T, len(layers)
     for j, d in enumerate(layers):
-        L.kind[j] = LAYER_CONV if isinstance(d, ConvDesc) else LAYER_LINEAR
+        L.kind[j] = LAYER_CONV if isinstance(d, ConvDesc) else (LAYER_ATTENTION if isinstance(d, AttentionDesc) else LAYER_LINEAR)
         L.layer[j] = C.cast(C.pointer(d), C.c_void_p)
     L._keep = (gate, list(layers))
     return L

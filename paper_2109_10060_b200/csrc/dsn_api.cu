@@ -62,6 +62,7 @@ struct LayerCall {
   const float* bias;
   const float *bn_scale, *bn_shift;
   int act, in_order, out_order, tail;
+  const dsn_attention_desc* att;  // non-null: this chain element is the attention core, not a sliced layer
 };
 
 int check_slices(int T, const int32_t* k_in, const int32_t* k_out, int C_in, int C_out) {
@@ -291,7 +292,7 @@ LayerCall from_linear(const dsn_linear_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = d->ldw; c.w_tap = d->ldw;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.att = nullptr;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -304,7 +305,7 @@ LayerCall from_conv(const dsn_conv_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = (int64_t)d->K * d->K * d->C_in; c.w_tap = d->C_in;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.att = nullptr;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -331,7 +332,18 @@ int layer_call_of(const dsn_layer_desc* L, int j, LayerCall& c) {
   if (!L->layer[j]) return DSN_ERR_INVALID_ARG;
   if (L->kind[j] == DSN_LAYER_LINEAR) c = from_linear(static_cast<const dsn_linear_desc*>(L->layer[j]));
   else if (L->kind[j] == DSN_LAYER_CONV) c = from_conv(static_cast<const dsn_conv_desc*>(L->layer[j]));
-  else return DSN_ERR_INVALID_ARG;
+  else if (L->kind[j] == DSN_LAYER_ATTENTION) {
+    // between two sliced layers only: it reads and writes grouped intermediates
+    if (j == 0 || j + 1 == L->n_layers) return DSN_ERR_INVALID_ARG;
+    const dsn_attention_desc* a = static_cast<const dsn_attention_desc*>(L->layer[j]);
+    memset(&c, 0, sizeof(c));
+    c.att = a;
+    c.dtype = a->dtype;
+    c.H = 1; c.W = a->N; c.K = 1;
+    c.C_in = 3 * a->H * a->D_h;
+    c.C_out = a->H * a->D_h;
+    c.T = a->T;
+  } else return DSN_ERR_INVALID_ARG;
   return DSN_OK;
 }
 
@@ -659,8 +671,10 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
                            : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
     void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
-    e = validate_call(c, &r, in, out);
-    if (e) return e;
+    if (!c.att) {
+      e = validate_call(c, &r, in, out);
+      if (e) return e;
+    }
   }
 
   const int32_t* idx = idx_in;
@@ -690,7 +704,15 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
                            : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
     void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
-    e = run_layer(ctx, calls[j], &r, in, out, s);
+    if (calls[j].att) {
+      dsn_attention_desc a = *calls[j].att;
+      a.ld_qkv = calls[j].C_in;   // dense grouped intermediates
+      a.ld_out = calls[j].C_out;
+      a.order = DSN_GROUPED;
+      e = dsn_sliced_attention(ctx, &a, &r, in, out, stream);
+    } else {
+      e = run_layer(ctx, calls[j], &r, in, out, s);
+    }
     if (e) return e;
   }
   return DSN_OK;

@@ -105,3 +105,49 @@ def test_vit_block_qkv_attention_proj_chain(dsn, ctx):
         err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
         assert err <= 1e-2, (i, err)                            # two chained bf16 stages after the QKV layer
         assert np.all(got[i, :, w:] == SENTINEL)
+
+
+def test_layer_forward_gate_qkv_attention_proj(dsn, ctx):
+    """The attention half of a ViT block as one dsn_layer_forward call: gate -> route -> QKV -> attention ->
+    proj -> input order, against the same chain made of separate calls."""
+    from gpu_util import up_f32
+    cfg = wl.config3(B=40, routing="iid")
+    B, R, De, H, Dh, T, paths = cfg["B"], cfg["R"], cfg["D_e"], cfg["H"], cfg["D_h"], cfg["T"], cfg["paths"]
+    heads = [p[1] for p in paths]
+    kq, koq = wl.vit_layer_slices(paths, Dh, "qkv")
+    kp, kop = wl.vit_layer_slices(paths, Dh, "proj")
+    Wf = up_bf16(wl.pack_qkv_head_major(cfg["Wq"], cfg["Wk"], cfg["Wv"], Dh))
+    Wp = up_bf16(cfg["Wproj"])
+    x = up_bf16(cfg["x"])
+    gW1, gW2 = up_f32(cfg["gate_W1"]), up_f32(cfg["gate_W2"])
+    gate = dsn.make_gate_desc(dsn.BF16, B, R, De, gW1.shape[0], T, gW1, gW2)
+    layers = [dsn.make_linear_desc(dsn.BF16, R, De, 3 * H * Dh, kq, koq, Wf),
+              dsn.make_attention_desc(R, H, Dh, heads),
+              dsn.make_linear_desc(dsn.BF16, R, H * Dh, De, kp, kop, Wp)]
+    L = dsn.make_layer_desc(B, T, layers, gate)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, R, De), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    idx_out = torch.zeros(B, dtype=torch.int32, device=DEV)
+    dsn.dsn_layer_forward(ctx, L, x, None, y, ws, idx_out=idx_out)
+    check_status(ctx, dsn)
+    idx = idx_out.cpu().numpy()
+    # separate calls with the same routing
+    r = route_on_gpu(dsn, ctx, idx, T)
+    qkv = torch.zeros((B, R, 3 * H * Dh), dtype=torch.bfloat16, device=DEV)
+    att = torch.zeros((B, R, H * Dh), dtype=torch.bfloat16, device=DEV)
+    y2 = torch.full((B, R, De), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(dsn.BF16, R, De, 3 * H * Dh, kq, koq, Wf, out_order=dsn.GROUPED), r, x, qkv)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(R, H, Dh, heads, order=dsn.GROUPED), r, qkv, att)
+    dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(dsn.BF16, R, H * Dh, De, kp, kop, Wp, in_order=dsn.GROUPED), r, att, y2)
+    check_status(ctx, dsn)
+    assert torch.equal(y, y2)
+    # and against the oracle end to end (three bf16 stages: chain tolerance)
+    q, k, v = O.vit_qkv(cfg["x"], cfg["Wq"], cfg["Wk"], cfg["Wv"], idx, paths, Dh)
+    q, k, v = (O.round_bf16(np.nan_to_num(a)) for a in (q, k, v))
+    a_ref = O.round_bf16(O.attention(q, k, v, idx, heads, Dh, fill=0.0))
+    ref = O.round_bf16(O.sliced_linear(a_ref, cfg["Wproj"], idx, kp, kop))
+    got = down(y)
+    for i in range(B):
+        w = kop[idx[i]]
+        err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
+        assert err <= 1e-2, (i, err)
