@@ -12,6 +12,7 @@ Passages followed (DS-Net++, "Dynamic Weight Slicing"):
   * dynamic network = route picked per input .......... Eq. (dyn_net), Sec. 3.1
   * weight slicing  psi(x) = W[:k] x ................... Eq. (weight_slicing), Sec. 3.2
   * slice-able convolution W[:c_O, :c_I] * X ........... Sec. 3.3, "Filter number"
+  * slice-able depthwise conv, kernel-size slicing ..... Sec. 3.3, "Group number ...", "Kernel size"
   * ViT QKV / proj / MLP slicing, self-attention ....... Sec. 3.4, Eq. (slimmableMLP)
   * gate: average-pool encoder, two-layer MLP, one-hot . Sec. 3.5
   * gate attention head X * (1 + tanh(W3 ReLU(W1 X_E))) . Sec. 3.5, "double-headed dynamic gate"
@@ -238,6 +239,43 @@ def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.na
         if bn is not None:
             z = split_bn(z, t, *bn)
         y[i, :, :, :ko] = activation(z, act)
+    return y
+
+
+def sliced_depthwise(x, W, idx, c, ksize, stride=1, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None):
+    """Slice-able depthwise convolution: group convolution with one filter per group (Sec. 3.3, "Group number
+    and filter number per group", first scheme: the output width follows the input width c), with kernel-size
+    slicing (the centred k x k part of the K x K filter) and the matching padding (k - 1) / 2, so that every
+    kernel size yields the same output size ("Kernel size", "Padding").
+
+    x [B][H][W][C] channels last, W [C][K][K].  For a sample of path t: channels < c[t], kernel ksize[t].
+    y[i][yy][xx][ch] = act(b[ch] + sum_{r,s<k} xpad[i][yy*stride + r - p][xx*stride + s - p][ch] * W[ch][k0+r][k0+s]),
+    k0 = (K - k) / 2, p = (k - 1) / 2, zero outside the image.  Output [B][Ho][Wo][C], Ho = (H - 1) // stride + 1.
+    """
+    x = np.asarray(x, dtype=F64)
+    W = np.asarray(W, dtype=F64)
+    B, H, Wd, C = x.shape
+    K = W.shape[1]
+    Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
+    y = np.full((B, Ho, Wo, C), fill, dtype=F64)
+    todo = range(B) if samples is None else samples
+    for i in todo:
+        t = int(idx[i])
+        ct, k = int(c[t]), int(ksize[t])
+        assert k % 2 == 1 and k <= K
+        k0, p = (K - k) // 2, (k - 1) // 2
+        xp = np.zeros((H + 2 * p, Wd + 2 * p, ct), dtype=F64)
+        xp[p:p + H, p:p + Wd, :] = x[i, :, :, :ct]
+        z = np.zeros((Ho, Wo, ct), dtype=F64)
+        for r in range(k):
+            for s in range(k):
+                win = xp[r:r + (Ho - 1) * stride + 1:stride, s:s + (Wo - 1) * stride + 1:stride, :]
+                z += win * W[:ct, k0 + r, k0 + s]
+        if bias is not None:
+            z = z + np.asarray(bias, dtype=F64)[:ct]
+        if bn is not None:
+            z = split_bn(z, t, *bn)
+        y[i, :, :, :ct] = activation(z, act)
     return y
 
 

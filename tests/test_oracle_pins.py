@@ -197,6 +197,44 @@ def test_conv_zero_padding_counts():
         assert y[i, 0, 0, 0] == 4 * k[i] and y[i, H - 1, Wd - 1, 1] == 4 * k[i]
 
 
+def test_depthwise_library_brute_force_and_kernel_slicing():
+    B, H, Wd, C, K = 3, 7, 6, 5, 7
+    x, W, b = rand(B, H, Wd, C), rand(C, K, K), rand(C)
+    idx = np.array([2, 0, 1]); c = [2, 5, 4]; ks = [3, 7, 5]
+    for stride in (1, 2):
+        got = O.sliced_depthwise(x, W, idx, c, ks, stride=stride, bias=b, act=O.ACT_RELU)
+        Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
+        assert got.shape == (B, Ho, Wo, C)
+        for i in range(B):
+            ct, k = c[idx[i]], ks[idx[i]]
+            k0 = (K - k) // 2
+            xt = torch.from_numpy(x[i:i + 1, :, :, :ct].copy()).permute(0, 3, 1, 2)
+            wt = torch.from_numpy(W[:ct, k0:k0 + k, k0:k0 + k].copy()).unsqueeze(1)
+            ref = torch.relu(torch.nn.functional.conv2d(xt, wt, torch.from_numpy(b[:ct].copy()), stride=stride,
+                                                         padding=(k - 1) // 2, groups=ct))
+            np.testing.assert_allclose(got[i, :, :, :ct], ref[0].permute(1, 2, 0).numpy(), rtol=1e-12, atol=1e-12)
+            assert np.all(np.isnan(got[i, :, :, ct:]))
+    # brute force, one output element (stride 2, 5x5 slice of the 7x7 filter)
+    got = O.sliced_depthwise(x, W, idx, c, ks, stride=2)
+    i, yy, xx, ch = 0, 1, 2, 3
+    acc = 0.0
+    for r in range(5):
+        for s_ in range(5):
+            iy, ix = yy * 2 + r - 2, xx * 2 + s_ - 2
+            if 0 <= iy < H and 0 <= ix < Wd:
+                acc += x[i, iy, ix, ch] * W[ch, 1 + r, 1 + s_]
+    assert abs(got[i, yy, xx, ch] - acc) < 1e-12
+    # a filter that is zero outside its centre 3x3 gives the same result for every kernel size
+    Wc = np.zeros((C, K, K)); Wc[:, 2:5, 2:5] = rand(C, 3, 3)
+    a3 = O.sliced_depthwise(x, Wc, np.zeros(B, int), [C], [3])
+    a7 = O.sliced_depthwise(x, Wc, np.zeros(B, int), [C], [7])
+    np.testing.assert_allclose(a3, a7, rtol=1e-12, atol=1e-12)
+    # channels are independent: channel ch of the output depends on channel ch of the input only
+    x2 = x.copy(); x2[..., 1] += 1.0
+    d = O.sliced_depthwise(x2, W, np.ones(B, int), c, ks) - O.sliced_depthwise(x, W, np.ones(B, int), c, ks)
+    assert np.all(d[..., [0, 2, 3, 4]] == 0) and np.any(d[..., 1] != 0)
+
+
 # ------------------------------------------------------------------ gate
 def brute_gate(x, W1, W2):
     B, R, C = x.shape
