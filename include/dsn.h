@@ -125,6 +125,29 @@ typedef struct dsn_conv_desc {
   int32_t in_order, out_order, tail;
 } dsn_conv_desc;
 
+/* Slice-able depthwise convolution (Sec. 3.3: group convolution whose group count follows the elastic
+ * input width; kernel-size slicing = the centred k x k part of the K x K filter; the padding follows
+ * the kernel size so that every k gives the same output size).  x [B][H][W][ldx], y [B][Ho][Wo][ldy]
+ * channels last with Ho = (H-1)/stride + 1; filter [K][K][C] bf16 (channels last), K odd <= 7.
+ * A sample of path t uses channels < c[t] and kernel size ksize[t]. */
+typedef struct dsn_depthwise_desc {
+  int32_t dtype;         /* DSN_BF16                                                     */
+  int32_t H, W_;         /* input size                                                   */
+  int32_t K;             /* stored kernel size (odd, <= 7)                               */
+  int32_t stride;        /* 1 or 2                                                       */
+  int32_t C;             /* full channel count                                           */
+  int64_t ldx, ldy;      /* elements between pixels of x, y (>= C)                       */
+  int32_t T;
+  const int32_t* c;      /* host [T] channels of each path, 1..C                         */
+  const int32_t* ksize;  /* host [T] kernel size of each path, odd, <= K                 */
+  const void* W;         /* device [K][K][C] bf16                                        */
+  const float* bias;     /* device [C] or NULL                                           */
+  const float* bn_scale; /* device [T][C] or NULL (dsn_resbn_fold)                       */
+  const float* bn_shift;
+  int32_t act;
+  int32_t in_order, out_order;
+} dsn_depthwise_desc;
+
 /* Slimmable self-attention core (Sec. 3.4): A_a = Softmax(Q_a K_a^T / sqrt(D_h)) V_a for the h heads of
  * the sample's path, concatenated.  qkv rows are laid out [head][q|k|v][D_h] (the output of the sliced
  * QKV layer with the head-major fused weight), out rows [head][D_h]; heads >= h are neither read nor
@@ -249,6 +272,9 @@ int dsn_sliced_linear(dsn_ctx* ctx, const dsn_linear_desc* d, const dsn_routing*
                       void* y, void* workspace, size_t ws_bytes, void* stream);
 int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, const void* x,
                     void* y, void* workspace, size_t ws_bytes, void* stream);
+
+int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_routing* r, const void* x, void* y,
+                         void* stream);
 
 /* qkv, out: device bf16, 16-byte aligned.  fp32 scores and softmax, bf16 probabilities for the
  * second contraction, bf16 output. */

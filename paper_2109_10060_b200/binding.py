@@ -26,7 +26,7 @@ MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
 EXPORTS = [
     "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_widths_from_ratios",
     "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
-    "dsn_sliced_attention", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
+    "dsn_sliced_attention", "dsn_sliced_depthwise", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
 ]
 
@@ -67,6 +67,14 @@ class ConvDesc(C.Structure):
 class AttentionDesc(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D_h", C.c_int32), ("ld_qkv", C.c_int64),
                 ("ld_out", C.c_int64), ("T", C.c_int32), ("heads", C.POINTER(C.c_int32)), ("order", C.c_int32)]
+
+
+class DepthwiseDesc(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("H", C.c_int32), ("W_", C.c_int32), ("K", C.c_int32), ("stride", C.c_int32),
+                ("C", C.c_int32), ("ldx", C.c_int64), ("ldy", C.c_int64), ("T", C.c_int32),
+                ("c", C.POINTER(C.c_int32)), ("ksize", C.POINTER(C.c_int32)), ("W", C.c_void_p), ("bias", C.c_void_p),
+                ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p), ("act", C.c_int32), ("in_order", C.c_int32),
+                ("out_order", C.c_int32)]
 
 
 class LayerDesc(C.Structure):
@@ -111,6 +119,7 @@ def load_library():
     lib.dsn_sliced_linear.argtypes = [vp, C.POINTER(LinearDesc), C.POINTER(Routing), vp, vp, vp, sz, vp]
     lib.dsn_sliced_conv.argtypes = [vp, C.POINTER(ConvDesc), C.POINTER(Routing), vp, vp, vp, sz, vp]
     lib.dsn_sliced_attention.argtypes = [vp, C.POINTER(AttentionDesc), C.POINTER(Routing), vp, vp, vp]
+    lib.dsn_sliced_depthwise.argtypes = [vp, C.POINTER(DepthwiseDesc), C.POINTER(Routing), vp, vp, vp]
     lib.dsn_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
     lib.dsn_layer_workspace_bytes.restype = sz
     lib.dsn_layer_forward.argtypes = [vp, C.POINTER(LayerDesc), vp, vp, vp, C.POINTER(Routing), vp, vp, sz, vp]
@@ -301,6 +310,20 @@ def make_attention_desc(N, H, D_h, heads, order=INPUT_ORDER, ld_qkv=None, ld_out
 def dsn_sliced_attention(ctx: Context, d: AttentionDesc, routing: Routing, qkv, out, stream=None):
     _check(ctx.lib.dsn_sliced_attention(ctx.handle, C.byref(d), C.byref(routing), _ptr(qkv), _ptr(out),
                                         _stream_handle(stream)), "dsn_sliced_attention")
+
+
+def make_depthwise_desc(H, Wd, K, stride, Cn, c, ksize, W, bias=None, act=ACT_NONE, in_order=INPUT_ORDER,
+                        out_order=INPUT_ORDER, ldx=None, ldy=None, bn_scale=None, bn_shift=None) -> DepthwiseDesc:
+    ca, ka = _i32_array(c), _i32_array(ksize)
+    d = DepthwiseDesc(BF16, H, Wd, K, stride, Cn, Cn if ldx is None else ldx, Cn if ldy is None else ldy, len(c), ca, ka,
+                      _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift), act, in_order, out_order)
+    d._keep = (ca, ka, W, bias, bn_scale, bn_shift)
+    return d
+
+
+def dsn_sliced_depthwise(ctx: Context, d: DepthwiseDesc, routing: Routing, x, y, stream=None):
+    _check(ctx.lib.dsn_sliced_depthwise(ctx.handle, C.byref(d), C.byref(routing), _ptr(x), _ptr(y),
+                                        _stream_handle(stream)), "dsn_sliced_depthwise")
 
 
 def dsn_layer_workspace_bytes(L: LayerDesc) -> int:

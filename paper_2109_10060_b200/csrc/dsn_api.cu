@@ -603,6 +603,27 @@ int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, 
   return run_layer(ctx, from_conv(d), r, x, y, as_stream(stream));
 }
 
+int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_routing* r, const void* x, void* y,
+                         void* stream) {
+  if (!ctx || !d || !x || !y || !d->W || !d->c || !d->ksize) return DSN_ERR_INVALID_ARG;
+  if (d->dtype != DSN_BF16) return DSN_ERR_UNSUPPORTED;
+  if (d->H < 1 || d->W_ < 1 || d->C < 1 || d->C > 32767 || d->K < 1 || d->K > 7 || d->K % 2 == 0) return DSN_ERR_INVALID_ARG;
+  if (d->stride != 1 && d->stride != 2) return DSN_ERR_UNSUPPORTED;
+  if (d->ldx < d->C || d->ldy < d->C || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (d->act < DSN_ACT_NONE || d->act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
+  if ((d->bn_scale == nullptr) != (d->bn_shift == nullptr)) return DSN_ERR_INVALID_ARG;
+  for (int t = 0; t < d->T; ++t)
+    if (d->c[t] < 1 || d->c[t] > d->C || d->ksize[t] < 1 || d->ksize[t] > d->K || d->ksize[t] % 2 == 0)
+      return DSN_ERR_INVALID_ARG;
+  int e = check_routing(r, d->T);
+  if (e) return e;
+  if (dsn_launch_depthwise(d->c, d->ksize, d->T, d->H, d->W_, d->K, d->stride, d->C, r->B, r->G, r->offsets, r->perm,
+                           r->group_slice, d->in_order == DSN_INPUT_ORDER, d->out_order == DSN_INPUT_ORDER, x, d->ldx,
+                           d->W, d->bias, d->bn_scale, d->bn_shift, d->act, y, d->ldy, as_stream(stream)) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
 int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_routing* r, const void* qkv, void* out,
                          void* stream) {
   if (!ctx || !d || !qkv || !out || !d->heads) return DSN_ERR_INVALID_ARG;

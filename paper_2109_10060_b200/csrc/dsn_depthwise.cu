@@ -1,0 +1,142 @@
+// Slice-able depthwise convolution (MobileNet DSConv's first half), channels last, bf16 storage with
+// fp32 arithmetic.  HBM-bound: a thread owns 8 consecutive channels (16 bytes) of one output pixel and
+// walks the k x k taps of its sample's kernel size (the centred part of the K x K filter); neighbouring
+// threads read neighbouring 16-byte pieces of a pixel, so every load and store is coalesced, and the
+// re-reads of overlapping windows are served by L1/L2.  Filter layout [K][K][C] (channels last).
+// A sample of path t uses channels < c[t] and kernel size ksize[t]; the rest is neither read nor written.
+#include "dsn_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct DwParams {
+  int16_t c[DSN_MAX_SLICES];
+  int8_t ksize[DSN_MAX_SLICES];
+  int32_t H, W, Ho, Wo, K, stride, C, T, G, bands;
+  int32_t x_input_order, y_input_order, act;
+  const int32_t* offsets;
+  const int32_t* perm;
+  const int32_t* group_slice;
+  const __nv_bfloat16* x;
+  int64_t ldx;
+  const __nv_bfloat16* w;
+  const float* bias;
+  const float* bn_scale;
+  const float* bn_shift;
+  __nv_bfloat16* y;
+  int64_t ldy;
+};
+
+__device__ __forceinline__ float act_apply(float v, int act) {
+  if (act == DSN_ACT_RELU) return fmaxf(v, 0.f);
+  if (act == DSN_ACT_GELU) return 0.5f * v * (1.f + erff(v * 0.70710678118654752f));
+  return v;
+}
+
+__global__ void __launch_bounds__(kThreads) depthwise_kernel(const __grid_constant__ DwParams p) {
+  __shared__ int s_info[3];  // slice, sample, valid
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  const int pos = blockIdx.y, band = blockIdx.x;
+  if (threadIdx.x == 0) {
+    int valid = pos < p.offsets[p.G], sl = 0, smp = 0;
+    if (valid) {
+      int lo = 0, hi = p.G;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.offsets[mid] <= pos) lo = mid; else hi = mid;
+      }
+      sl = p.group_slice ? p.group_slice[lo] : lo;
+      smp = p.perm[pos];
+      if (smp < 0 || sl < 0 || sl >= p.T) valid = 0;
+    }
+    s_info[0] = sl; s_info[1] = smp; s_info[2] = valid;
+  }
+  __syncthreads();
+  if (!s_info[2]) return;
+  const int sl = s_info[0], smp = s_info[1];
+  const int ct = p.c[sl], k = p.ksize[sl];
+  const int k0 = (p.K - k) >> 1, pad = (k - 1) >> 1;
+  const __nv_bfloat16* xs = p.x + (int64_t)(p.x_input_order ? smp : pos) * p.H * p.W * p.ldx;
+  __nv_bfloat16* ys = p.y + (int64_t)(p.y_input_order ? smp : pos) * p.Ho * p.Wo * p.ldy;
+  const float* sc = p.bn_scale ? p.bn_scale + (int64_t)sl * p.C : nullptr;
+  const float* sh = p.bn_scale ? p.bn_shift + (int64_t)sl * p.C : nullptr;
+  const int nvec = (ct + 7) >> 3;
+  const int pix0 = (int)(((int64_t)p.Ho * p.Wo * band) / p.bands), pix1 = (int)(((int64_t)p.Ho * p.Wo * (band + 1)) / p.bands);
+  const bool vec_ok = (p.ldx % 8 == 0) && (p.ldy % 8 == 0) && (p.C % 8 == 0) &&
+                      ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.w)) & 15) == 0;
+  for (int64_t e = threadIdx.x; e < (int64_t)(pix1 - pix0) * nvec; e += kThreads) {
+    const int pix = pix0 + (int)(e / nvec), v = (int)(e % nvec);
+    const int yy = pix / p.Wo, xx = pix - yy * p.Wo;
+    const int c0 = v * 8;
+    const int nch = ct - c0 < 8 ? ct - c0 : 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int r = 0; r < k; ++r) {
+      const int iy = yy * p.stride + r - pad;
+      if (iy < 0 || iy >= p.H) continue;
+      for (int s = 0; s < k; ++s) {
+        const int ix = xx * p.stride + s - pad;
+        if (ix < 0 || ix >= p.W) continue;
+        const __nv_bfloat16* xp = xs + ((int64_t)iy * p.W + ix) * p.ldx + c0;
+        const __nv_bfloat16* wp = p.w + ((int64_t)(k0 + r) * p.K + (k0 + s)) * p.C + c0;
+        if (vec_ok && nch == 8) {
+          const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xp)), wv = __ldg(reinterpret_cast<const uint4*>(wp));
+          const uint32_t xa[4] = {xv.x, xv.y, xv.z, xv.w}, wa[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            acc[2 * j] = fmaf(__uint_as_float(xa[j] << 16), __uint_as_float(wa[j] << 16), acc[2 * j]);
+            acc[2 * j + 1] = fmaf(__uint_as_float(xa[j] & 0xffff0000u), __uint_as_float(wa[j] & 0xffff0000u), acc[2 * j + 1]);
+          }
+        } else {
+          for (int j = 0; j < nch; ++j) acc[j] = fmaf(__bfloat162float(xp[j]), __bfloat162float(wp[j]), acc[j]);
+        }
+      }
+    }
+    __nv_bfloat16* yp = ys + (int64_t)pix * p.ldy + c0;
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float a = acc[2 * j], b = acc[2 * j + 1];
+      const int ca = c0 + 2 * j, cb = ca + 1;
+      if (p.bias) { if (ca < ct) a += p.bias[ca]; if (cb < ct) b += p.bias[cb]; }
+      if (sc) { if (ca < ct) a = fmaf(a, sc[ca], sh[ca]); if (cb < ct) b = fmaf(b, sc[cb], sh[cb]); }
+      __nv_bfloat162 h = __floats2bfloat162_rn(act_apply(a, p.act), act_apply(b, p.act));
+      o[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    if (vec_ok && nch == 8) {
+      *reinterpret_cast<uint4*>(yp) = make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      for (int j = 0; j < nch; ++j)
+        reinterpret_cast<uint16_t*>(yp)[j] = (j & 1) ? (uint16_t)(o[j >> 1] >> 16) : (uint16_t)(o[j >> 1] & 0xffffu);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t dsn_launch_depthwise(const int32_t* c, const int32_t* ksize, int T, int H, int W, int K, int stride, int C,
+                                 int B, int G, const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
+                                 int x_input_order, int y_input_order, const void* x, int64_t ldx, const void* w,
+                                 const float* bias, const float* bn_scale, const float* bn_shift, int act, void* y,
+                                 int64_t ldy, cudaStream_t s) {
+  if (B == 0) return cudaSuccess;
+  DwParams p;
+  memset(&p, 0, sizeof(p));
+  for (int t = 0; t < T; ++t) {
+    p.c[t] = (int16_t)c[t];
+    p.ksize[t] = (int8_t)ksize[t];
+  }
+  p.H = H; p.W = W; p.K = K; p.stride = stride; p.C = C; p.T = T; p.G = G;
+  p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
+  int bands = (p.Ho * p.Wo) / 64 > 0 ? (p.Ho * p.Wo) / 64 : 1;
+  if (bands > 32) bands = 32;
+  p.bands = bands;
+  p.x_input_order = x_input_order; p.y_input_order = y_input_order; p.act = act;
+  p.offsets = offsets; p.perm = perm; p.group_slice = group_slice;
+  p.x = static_cast<const __nv_bfloat16*>(x); p.ldx = ldx;
+  p.w = static_cast<const __nv_bfloat16*>(w);
+  p.bias = bias; p.bn_scale = bn_scale; p.bn_shift = bn_shift;
+  p.y = static_cast<__nv_bfloat16*>(y); p.ldy = ldy;
+  return dsn_launch(depthwise_kernel, dim3(bands, B), dim3(kThreads), 0, s, 1, p);
+}

@@ -135,6 +135,12 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
                                  const void* qkv, int64_t ld_qkv, void* out, int64_t ld_out, int32_t* status,
                                  cudaStream_t s);
 
+cudaError_t dsn_launch_depthwise(const int32_t* c, const int32_t* ksize, int T, int H, int W, int K, int stride, int C,
+                                 int B, int G, const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
+                                 int x_input_order, int y_input_order, const void* x, int64_t ldx, const void* w,
+                                 const float* bias, const float* bn_scale, const float* bn_shift, int act, void* y,
+                                 int64_t ldy, cudaStream_t s);
+
 struct SliceTable {
   int32_t k_in[DSN_MAX_SLICES];
   int32_t k_out[DSN_MAX_SLICES];
