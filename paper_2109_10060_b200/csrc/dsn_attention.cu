@@ -5,27 +5,30 @@
 // the output row holds [head][64] and feeds the sliced projection (k_in = h * 64).  Heads >= h of a
 // sample are neither read nor written.
 //
-// One CTA (128 threads) per (sample, head), N <= 256 tokens, D_h = 64:
-//   K [256 keys][64] and Q [128 queries][64] arrive by TMA (K-major, 128-byte swizzle);
-//   V is transposed by the threads into V^T [64][256 keys] in the same swizzled K-major layout
-//   (keys >= N are written as zeros);
-//   S = Q K^T: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
-//   every thread owns one query row: two passes over its S row in TMEM (row maximum; exponentials,
-//   row sum, P as bf16 into a swizzled K-major shared-memory tile, keys >= N as zeros);
+// One CTA (256 threads) per (sample, head), N <= 256 tokens, D_h = 64:
+//   Q [2 x 128 queries][64], K [256 keys][64] and V [256 keys][64] arrive by TMA (128-byte rows,
+//   128-byte swizzle).  K is the K-major B operand of S = Q K^T; V, whose rows are keys and whose
+//   64 contiguous elements are the head dimension, is the MN-major B operand of O = P V, so it is
+//   used as loaded (its rows >= N are cleared: they belong to the next sample);
+//   S = Q K^T for both 128-query halves: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
+//   two threads share one query row (warps w and w + 4 own the same TMEM lanes and half of the keys
+//   each): one pass over their part of the S row held in registers gives the row maximum, the
+//   exponentials, the row sum and P as bf16 in a swizzled K-major shared-memory tile (keys >= N: zeros);
 //   O = P V: tcgen05.mma M = 128, N = 64, K = keys rounded to 16; the row is scaled by 1 / sum,
-//   rounded to bf16 and stored as one 128-byte line.
-// The two 128-query halves of the sample run one after the other.  Waits are bounded as in the GEMM.
+//   rounded to bf16 and stored (each of the two threads writes 64 bytes of the 128-byte line).
+// Waits are bounded as in the GEMM.
 #include "dsn_gemm_device.cuh"
 
 namespace {
 
 using namespace dsn_gemm;
 
-constexpr int kAttThreads = 128;
-constexpr uint32_t kQBytes = 128 * 128;       // 128 queries x 64 bf16
+constexpr int kAttThreads = 256;
+constexpr uint32_t kQBytes = 2 * 128 * 128;   // two halves of 128 queries x 64 bf16
 constexpr uint32_t kKBytes = 256 * 128;       // 256 keys x 64 bf16
-constexpr uint32_t kVtBytes = 4 * 64 * 128;   // 4 key chunks x 64 (d) rows x 64 keys bf16
+constexpr uint32_t kVBytes = 256 * 128;       // 256 keys x 64 bf16
 constexpr uint32_t kPBytes = 4 * 128 * 128;   // 4 key chunks x 128 queries x 64 keys bf16
+constexpr uint32_t kSCols = 224;              // TMEM columns per S accumulator (two of them), O at 448
 
 struct AttParams {
   CUtensorMap map;        // qkv seen as [rows][3H][64], box 128 rows x 1 x 64
@@ -51,19 +54,32 @@ __device__ __forceinline__ int find_group_of(const int32_t* __restrict__ offsets
   return lo;
 }
 
+// MN-major operand descriptor: rows of the tile are K indices (128 bytes = 64 contiguous M/N elements
+// each), 8-row groups 1024 bytes apart, 128-byte swizzle; one K = 16 step is 16 rows = 2048 bytes.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_constant__ AttParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  // layout: control 1 KB | Q 16 KB | K 32 KB | V^T 32 KB | P 64 KB
+  // layout: control 1 KB (barriers, row maxima and sums) | Q 32 KB | K 32 KB | V 32 KB | P 64 KB
   const uint32_t bar_load = base, bar_mma = base + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 20);
-  int32_t* s_info = reinterpret_cast<int32_t*>(smem + 24);  // [0] heads of this sample, [1] row block
-  const uint32_t q_s = base + 1024, k_s = q_s + kQBytes, vt_s = k_s + kKBytes, p_s = vt_s + kVtBytes;
-  uint8_t* vt_ptr = smem + 1024 + kQBytes + kKBytes;
-  uint8_t* p_ptr = vt_ptr + kVtBytes;
+  int32_t* s_info = reinterpret_cast<int32_t*>(smem + 24);
+  float* s_red = reinterpret_cast<float*>(smem + 64);  // [2 parts][128 rows]: maxima, then sums
+  const uint32_t q_s = base + 2048, k_s = q_s + kQBytes, v_s = k_s + kKBytes, p_s = v_s + kVBytes;
+  uint8_t* v_ptr = smem + 2048 + kQBytes + kKBytes;
+  uint8_t* p_ptr = v_ptr + kVBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head = blockIdx.x, pos = blockIdx.y;
@@ -90,117 +106,129 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
   if (head >= s_info[0]) return;  // this sample's path has fewer heads (uniform over the CTA)
   const int N = p.N;
   const int64_t row0 = (int64_t)s_info[1] * N;
-  const int npad = (N + 15) & ~15;  // keys rounded to the MMA's K step / N granule
+  const int npad = (N + 15) & ~15;
+  const int nhalves = N > 128 ? 2 : 1;
 
   if (warp == 0) {
     tmem_alloc(smem_u32(tmem_slot), 512);
     tmem_relinquish();
   }
-  if (tid == 0) {  // K (two boxes of 128 keys) and the first 128 queries
-    mbar_expect_tx(bar_load, kKBytes + kQBytes);
-    tma_load_3d(k_s, &p.map, 0, head * 3 + 1, (int)row0, bar_load);
-    tma_load_3d(k_s + 128 * 128, &p.map, 0, head * 3 + 1, (int)row0 + 128, bar_load);
-    tma_load_3d(q_s, &p.map, 0, head * 3 + 0, (int)row0, bar_load);
-  }
-  // V^T: element (d, key) -> chunk key/64, row d, 16-byte piece (key%64)/8 XOR (d & 7), slot key % 8
-  {
-    const __nv_bfloat16* vsrc = p.qkv + row0 * p.ld_qkv + (int64_t)(head * 3 + 2) * 64;
-    for (int e = tid; e < 256 * 8; e += kAttThreads) {  // (key, group of 8 d)
-      const int key = e >> 3, d8 = e & 7;
-      uint4 val = make_uint4(0u, 0u, 0u, 0u);
-      if (key < N) val = __ldg(reinterpret_cast<const uint4*>(vsrc + (int64_t)key * p.ld_qkv) + d8);
-      const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-      const int kc = key >> 6, kk = key & 63;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int d = d8 * 8 + i;
-        const uint16_t bits = (i & 1) ? (uint16_t)(w[i >> 1] >> 16) : (uint16_t)(w[i >> 1] & 0xffffu);
-        *reinterpret_cast<uint16_t*>(vt_ptr + kc * 8192 + d * 128 + (((kk >> 3) ^ (d & 7)) << 4) + (kk & 7) * 2) = bits;
-      }
+  if (tid == 0) {
+    mbar_expect_tx(bar_load, kKBytes + kVBytes + kQBytes);
+    for (int b2 = 0; b2 < 2; ++b2) {
+      tma_load_3d(k_s + b2 * 16384, &p.map, 0, head * 3 + 1, (int)row0 + 128 * b2, bar_load);
+      tma_load_3d(v_s + b2 * 16384, &p.map, 0, head * 3 + 2, (int)row0 + 128 * b2, bar_load);
+      tma_load_3d(q_s + b2 * 16384, &p.map, 0, head * 3 + 0, (int)row0 + 128 * b2, bar_load);
     }
   }
-  fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 256;
-  const uint32_t idesc_s = make_idesc(128, npad), idesc_o = make_idesc(128, 64);
-  const float sl2 = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
-  bool ok = true;
-  uint32_t load_phase = 0, mma_phase = 0;
+  // up to 224 keys: both halves' S accumulators (224 columns each) and O fit in the 512 columns and both
+  // S products are issued at once; above that one S accumulator (256 columns) is reused by the halves
+  const bool two_s = npad <= (int)kSCols;
+  const uint32_t tmem_O = tmem_base + (two_s ? 2 * kSCols : 256);
+  const uint32_t idesc_s = make_idesc(128, npad);
+  const uint32_t idesc_o = make_idesc(128, 64) | (1u << 16);  // B operand MN-major
+  const float sl2 = 0.125f * 1.4426950408889634f;             // 1/sqrt(64) * log2(e)
 
-  for (int half = 0; half < 2 && ok; ++half) {
-    if (half * 128 >= N) break;
-    if (half == 1) {  // second 128 queries into the same buffer (the S MMA that read it has completed)
-      if (tid == 0) {
-        mbar_expect_tx(bar_load, kQBytes);
-        tma_load_3d(q_s, &p.map, 0, head * 3 + 0, (int)row0 + 128, bar_load);
-      }
-    }
-    // ---- S = Q K^T
-    if (tid == 0) {
-      if (mbar_wait(bar_load, load_phase, abort_flag, p.status, 21)) {
-        tc_fence_after();
-        const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
+  bool ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag, p.status, 21) ? 1 : 0) != 0;
+  uint32_t mma_phase = 0;
+  if (ok) {
+    // V rows >= N belong to the next sample (or to nobody): clear them so that 0 * garbage cannot appear
+    for (int e = tid; e < (npad - N) * 8; e += kAttThreads)
+      *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+    __syncthreads();
+    if (tid == 0) {  // S for both halves of the queries
+      tc_fence_after();
+      for (int half = 0; half < (two_s ? nhalves : 1); ++half) {
+        const uint64_t dq = make_smem_desc(q_s + half * 16384), dk = make_smem_desc(k_s);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_S, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-        umma_commit(bar_mma);
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tmem_base + half * kSCols, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
       }
+      umma_commit(bar_mma);
     }
-    load_phase ^= 1u;
     ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, abort_flag, p.status, 22) ? 1 : 0) != 0;
     mma_phase ^= 1u;
-    if (!ok) break;
-    tc_fence_after();
+  }
 
-    // ---- softmax of this thread's query row; P (bf16) into the swizzled K-major tile
-    const int m = warp * 32 + lane;  // accumulator row = TMEM lane
-    const uint32_t trow = tmem_S + ((uint32_t)(warp * 32) << 16);
-    float mx = -INFINITY;
-    for (int c0 = 0; c0 < npad; c0 += 32) {
-      uint32_t v[32];
-      tmem_ld_32x32(trow + c0, v);
-      tmem_ld_wait();
+  const int part = warp >> 2;                 // which half of the keys this thread owns
+  const int m = (warp & 3) * 32 + lane;       // query row within the half = TMEM lane
+  const int cols_per = npad >> 1;             // keys per part, a multiple of 8
+  const int cbeg = part * cols_per;
+
+  for (int half = 0; half < nhalves && ok; ++half) {
+    if (!two_s && half == 1) {  // second S product into the accumulator the first half has finished reading
+      if (tid == 0) {
+        tc_fence_after();
+        const uint64_t dq = make_smem_desc(q_s + 16384), dk = make_smem_desc(k_s);
 #pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (c0 + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
+        for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_base, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
+        umma_commit(bar_mma);
+      }
+      ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, abort_flag, p.status, 24) ? 1 : 0) != 0;
+      mma_phase ^= 1u;
+      if (!ok) break;
     }
+    tc_fence_after();
+    const uint32_t trow = tmem_base + (two_s ? half * kSCols : 0) + ((uint32_t)((warp & 3) * 32) << 16);
+    // ---- this thread's part of the S row, in registers
+    uint32_t v[4][32];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (32 * c < cols_per) tmem_ld_32x32(trow + cbeg + 32 * c, v[c]);  // uniform over the CTA
+    tmem_ld_wait();
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int j = 32 * c + i;
+        if (j < cols_per && cbeg + j < N) mx = fmaxf(mx, __uint_as_float(v[c][i]));
+      }
+    s_red[part * 128 + m] = mx;
+    __syncthreads();
+    mx = fmaxf(s_red[m], s_red[128 + m]);
+    __syncthreads();
     float sum = 0.f;
-    for (int c0 = 0; c0 < npad; c0 += 32) {
-      uint32_t v[32];
-      tmem_ld_32x32(trow + c0, v);
-      tmem_ld_wait();
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        uint32_t w[4];
+    for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int c = 8 * j + 2 * e;
-          float a = 0.f, b = 0.f;
-          if (c0 + c < N) a = exp2f((__uint_as_float(v[c]) - mx) * sl2);
-          if (c0 + c + 1 < N) b = exp2f((__uint_as_float(v[c + 1]) - mx) * sl2);
-          __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
-          // the row sum uses the rounded probabilities, the values the second MMA multiplies
-          sum += __low2float(hb) + __high2float(hb);
-          w[e] = *reinterpret_cast<uint32_t*>(&hb);
-        }
-        const int key = c0 + 8 * j;
-        if (key < npad)
+      for (int jv = 0; jv < 4; ++jv) {
+        const int j0 = 32 * c + 8 * jv;       // first of 8 keys, relative to the part
+        if (j0 < cols_per) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j = j0 + 2 * e;
+            float a = 0.f, b = 0.f;
+            if (cbeg + j < N) a = exp2f((__uint_as_float(v[c][8 * jv + 2 * e]) - mx) * sl2);
+            if (cbeg + j + 1 < N) b = exp2f((__uint_as_float(v[c][8 * jv + 2 * e + 1]) - mx) * sl2);
+            __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
+            sum += __low2float(hb) + __high2float(hb);  // the rounded probabilities are what the MMA multiplies
+            w[e] = *reinterpret_cast<uint32_t*>(&hb);
+          }
+          const int key = cbeg + j0;
           *reinterpret_cast<uint4*>(p_ptr + (key >> 6) * 16384 + m * 128 + ((((key & 63) >> 3) ^ (m & 7)) << 4)) =
               make_uint4(w[0], w[1], w[2], w[3]);
+        }
       }
     }
+    s_red[part * 128 + m] = sum;
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
+    sum = s_red[m] + s_red[128 + m];
 
     // ---- O = P V
     if (tid == 0) {
       tc_fence_after();
       for (int ks = 0; ks < npad / 16; ++ks) {
         const uint64_t dp = make_smem_desc(p_s + (ks >> 2) * 16384) + 2u * (ks & 3);
-        const uint64_t dv = make_smem_desc(vt_s + (ks >> 2) * 8192) + 2u * (ks & 3);
+        const uint64_t dv = make_smem_desc_mn(v_s + ks * 2048);
         umma_bf16(tmem_O, dp, dv, idesc_o, ks > 0 ? 1u : 0u);
       }
       umma_commit(bar_mma);
@@ -210,32 +238,29 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
     if (!ok) break;
     tc_fence_after();
     {
-      const uint32_t orow = tmem_O + ((uint32_t)(warp * 32) << 16);
+      const uint32_t orow = tmem_O + ((uint32_t)((warp & 3) * 32) << 16) + 32 * part;
       const int q = half * 128 + m;
       const float inv = 1.f / sum;
-      __nv_bfloat16* dst = p.out + (row0 + q) * p.ld_out + (int64_t)head * 64;
+      __nv_bfloat16* dst = p.out + (row0 + q) * p.ld_out + (int64_t)head * 64 + 32 * part;
+      uint32_t o[32];
+      tmem_ld_32x32(orow, o);
+      tmem_ld_wait();
+      if (q < N) {
 #pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32(orow + c0, v);
-        tmem_ld_wait();
-        if (q < N) {
+        for (int j = 0; j < 4; ++j) {
+          uint32_t w[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t w[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              __nv_bfloat162 hb = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]) * inv,
-                                                        __uint_as_float(v[8 * j + 2 * e + 1]) * inv);
-              w[e] = *reinterpret_cast<uint32_t*>(&hb);
-            }
-            *reinterpret_cast<uint4*>(dst + c0 + 8 * j) = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 hb = __floats2bfloat162_rn(__uint_as_float(o[8 * j + 2 * e]) * inv,
+                                                      __uint_as_float(o[8 * j + 2 * e + 1]) * inv);
+            w[e] = *reinterpret_cast<uint32_t*>(&hb);
           }
+          *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }
     tc_fence_before();
-    __syncthreads();  // TMEM rows and the P tile are free for the next half
+    __syncthreads();  // O, the P tile and the reduction scratch are free for the next half
   }
 
   tc_fence_before();
@@ -267,7 +292,7 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   p.qkv = static_cast<const __nv_bfloat16*>(qkv); p.ld_qkv = ld_qkv;
   p.out = static_cast<__nv_bfloat16*>(out); p.ld_out = ld_out;
   p.status = status;
-  const size_t smem = 1024 + 1024 + kQBytes + kKBytes + kVtBytes + kPBytes;
+  const size_t smem = 1024 + 2048 + kQBytes + kKBytes + kVBytes + kPBytes;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
