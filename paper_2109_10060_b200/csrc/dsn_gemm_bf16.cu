@@ -272,12 +272,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
       const CUtensorMap* mY = &p.mapY[t.map];
-      if (p.act == DSN_ACT_NONE)
-        epilogue_tile<DSN_ACT_NONE>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
-      else if (p.act == DSN_ACT_RELU)
-        epilogue_tile<DSN_ACT_RELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
-      else
-        epilogue_tile<DSN_ACT_GELU>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row);
+      const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
+      switch (variant) {
+        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);

@@ -169,7 +169,9 @@ __device__ __forceinline__ float erf_fast(float z) {
   return t;
 }
 
-// The activation is a template parameter so that the per-element loop holds no trace of the others.
+// The activation (and whether any per-column affine term exists) is a template parameter so that the
+// per-element loop holds no trace of the other variants: an if-converted erf or a few unused loads per
+// element are enough to put the epilogue behind the main loop.
 template <int ACT>
 __device__ __forceinline__ float apply_act(float v) {
   if (ACT == DSN_ACT_RELU) return fmaxf(v, 0.f);
@@ -182,7 +184,7 @@ __device__ __forceinline__ float apply_act(float v) {
 // `first`, `first + 2`, ...  With `contig` the 32 rows are consecutive output rows starting at
 // `base_row` and each chunk leaves as one TMA store (columns clipped by the map); otherwise eight
 // lanes store one 128-byte piece of a row each.
-template <int ACT>
+template <int ACT, bool AFF>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
                                               const float* sc_row, const float* sh_row, uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
                                               const CUtensorMap* mapY, int base_row) {
@@ -206,13 +208,15 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
           for (int e = 0; e < 4; ++e) {
             const int c = 8 * jj + 2 * e;
             float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
-            if (brow) {
-              if (cb + c < ncols) a += __ldg(brow + cb + c);
-              if (cb + c + 1 < ncols) b += __ldg(brow + cb + c + 1);
-            }
-            if (sc_row) {  // Re-SBN of this tile's path: per-channel scale and shift
-              if (cb + c < ncols) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
-              if (cb + c + 1 < ncols) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
+            if (AFF) {  // bias and / or the per-path Re-SBN scale and shift of this tile's columns
+              if (cb + c < ncols) {
+                if (brow) a += __ldg(brow + cb + c);
+                if (sc_row) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
+              }
+              if (cb + c + 1 < ncols) {
+                if (brow) b += __ldg(brow + cb + c + 1);
+                if (sc_row) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
+              }
             }
             __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
             w[e] = *reinterpret_cast<uint32_t*>(&h);
