@@ -253,13 +253,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
-      // output rows this lane writes in the direct-store phase: row 4*i + lane/8 of the warp's 32 rows
-      __nv_bfloat16* rp[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        rp[i] = reinterpret_cast<__nv_bfloat16*>(
-            __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(yrow), 4 * i + (lane >> 3)));
-      // 32 consecutive output rows can leave through the TMA unit
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
       // (a slice width that is no multiple of 8 columns = 16 bytes keeps the element-wise path: the
       // store was seen to clip the row at 16-byte granularity and would touch columns >= k_out)
@@ -274,12 +267,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const CUtensorMap* mY = &p.mapY[t.map];
       const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
       switch (variant) {
-        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
-        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
-        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
-        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
-        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
-        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, rp, lane, contig, mY, (int)base_row); break;
+        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
       }
       tc_fence_before();
       __syncwarp();

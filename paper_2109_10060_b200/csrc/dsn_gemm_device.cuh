@@ -181,12 +181,13 @@ __device__ __forceinline__ float apply_act(float v) {
 
 // Epilogue of one tile for one warp: accumulator rows (one per lane) -> bias, activation, bf16 ->
 // 32 x 128-byte swizzled staging tile -> global memory.  The warp takes the 64-column chunks
-// `first`, `first + 2`, ...  With `contig` the 32 rows are consecutive output rows starting at
+// `first`, `first + 2`, ...  `yrow` is this lane's output row (nullptr when the row is not part of the
+// result).  With `contig` the 32 rows are consecutive output rows starting at
 // `base_row` and each chunk leaves as one TMA store (columns clipped by the map); otherwise eight
 // lanes store one 128-byte piece of a row each.
 template <int ACT, bool AFF>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
-                                              const float* sc_row, const float* sh_row, uint8_t* stage_w, __nv_bfloat16* const (&rp)[8], int lane, bool contig,
+                                              const float* sc_row, const float* sh_row, uint8_t* stage_w, __nv_bfloat16* yrow, int lane, bool contig,
                                               const CUtensorMap* mapY, int base_row) {
   for (int c0 = 64 * first; c0 < ncols; c0 += 128) {
     // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
@@ -236,7 +237,13 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
       continue;
     }
     __syncwarp();
-    // phase 2: eight lanes per row, 16 bytes each: contiguous 128-byte pieces of output rows
+    // phase 2: eight lanes per row, 16 bytes each: contiguous 128-byte pieces of output rows.  Lane l
+    // stores row 4*i + l/8 of the warp's 32 rows in step i; the row pointers come from their owners.
+    __nv_bfloat16* rp[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      rp[i] = reinterpret_cast<__nv_bfloat16*>(
+          __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(yrow), 4 * i + (lane >> 3)));
     const int j = lane & 7, col = c0 + 8 * j;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
