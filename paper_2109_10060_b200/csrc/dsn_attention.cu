@@ -5,17 +5,21 @@
 // the output row holds [head][64] and feeds the sliced projection (k_in = h * 64).  Heads >= h of a
 // sample are neither read nor written.
 //
-// One CTA (256 threads) per (sample, head), N <= 256 tokens, D_h = 64:
-//   Q [2 x 128 queries][64], K [256 keys][64] and V [256 keys][64] arrive by TMA (128-byte rows,
+// One CTA (256 threads) per (sample, head, half of the queries), N <= 256 tokens, D_h = 64; two CTAs
+// fit on an SM (about 99 KB of shared memory and 256 TMEM columns each), so one CTA's loads and
+// barriers hide behind the other's arithmetic:
+//   Q [128 queries][64], K [256 keys][64] and V [256 keys][64] arrive by TMA (128-byte rows,
 //   128-byte swizzle).  K is the K-major B operand of S = Q K^T; V, whose rows are keys and whose
 //   64 contiguous elements are the head dimension, is the MN-major B operand of O = P V, so it is
 //   used as loaded (its rows >= N are cleared: they belong to the next sample);
-//   S = Q K^T for both 128-query halves: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
+//   S = Q K^T: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
 //   two threads share one query row (warps w and w + 4 own the same TMEM lanes and half of the keys
 //   each): one pass over their part of the S row held in registers gives the row maximum, the
-//   exponentials, the row sum and P as bf16 in a swizzled K-major shared-memory tile (keys >= N: zeros);
-//   O = P V: tcgen05.mma M = 128, N = 64, K = keys rounded to 16; the row is scaled by 1 / sum,
-//   rounded to bf16 and stored (each of the two threads writes 64 bytes of the 128-byte line).
+//   exponentials, the row sum and P as bf16 in a swizzled K-major shared-memory tile that reuses the
+//   space of K and Q (keys >= N: zeros);
+//   O = P V: tcgen05.mma M = 128, N = 64, K = keys rounded to 16, into the TMEM columns S has left;
+//   the row is scaled by 1 / sum, rounded to bf16 and stored (each of the two threads writes 64 bytes
+//   of the 128-byte line).
 // Waits are bounded as in the GEMM.
 #include "dsn_gemm_device.cuh"
 
@@ -24,11 +28,11 @@ namespace {
 using namespace dsn_gemm;
 
 constexpr int kAttThreads = 256;
-constexpr uint32_t kQBytes = 2 * 128 * 128;   // two halves of 128 queries x 64 bf16
+constexpr uint32_t kQBytes = 128 * 128;       // 128 queries x 64 bf16
 constexpr uint32_t kKBytes = 256 * 128;       // 256 keys x 64 bf16
 constexpr uint32_t kVBytes = 256 * 128;       // 256 keys x 64 bf16
-constexpr uint32_t kPBytes = 4 * 128 * 128;   // 4 key chunks x 128 queries x 64 keys bf16
-constexpr uint32_t kSCols = 224;              // TMEM columns per S accumulator (two of them), O at 448
+constexpr uint32_t kPBytes = 4 * 128 * 128;   // 4 key chunks x 128 queries x 64 keys bf16 (over K, Q and 16 KB more)
+constexpr uint32_t kAttTmemCols = 256;
 
 struct AttParams {
   CUtensorMap map;        // qkv seen as [rows][3H][64], box 128 rows x 1 x 64
@@ -66,37 +70,47 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
   return d;
 }
 
-__global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_constant__ AttParams p) {
+__global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_constant__ AttParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  // layout: control 1 KB (barriers, row maxima and sums) | Q 32 KB | K 32 KB | V 32 KB | P 64 KB
+  // layout: control 2 KB (barriers, row maxima and sums) | V 32 KB | K 32 KB | Q 16 KB | 16 KB;
+  // P (64 KB) overlays K, Q and the last 16 KB once S has been computed
   const uint32_t bar_load = base, bar_mma = base + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 20);
   int32_t* s_info = reinterpret_cast<int32_t*>(smem + 24);
   float* s_red = reinterpret_cast<float*>(smem + 64);  // [2 parts][128 rows]: maxima, then sums
-  const uint32_t q_s = base + 2048, k_s = q_s + kQBytes, v_s = k_s + kKBytes, p_s = v_s + kVBytes;
-  uint8_t* v_ptr = smem + 2048 + kQBytes + kKBytes;
+  const uint32_t v_s = base + 2048, k_s = v_s + kVBytes, q_s = k_s + kKBytes, p_s = k_s;
+  uint8_t* v_ptr = smem + 2048;
   uint8_t* p_ptr = v_ptr + kVBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int head = blockIdx.x, pos = blockIdx.y;
+  const int head = blockIdx.x, pos = blockIdx.y, half = blockIdx.z;
 
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
+  if (half * 128 >= p.N) return;
+  // Group of this position = (number of groups whose first position is <= pos) - 1, counted by the whole
+  // CTA in one round of loads instead of a chain of dependent ones; perm[pos] travels at the same time.
+  int blk_reg = 0;
+  if (tid == 0) blk_reg = p.grouped ? pos : p.perm[pos];
+  int n_le = 0;
+  for (int g0 = 0; g0 < p.G; g0 += kAttThreads) {
+    const int g = g0 + tid;
+    n_le += __syncthreads_count(g < p.G && p.offsets[g] <= pos);
+  }
   if (tid == 0) {
-    int h = 0, blk = 0;
-    if (pos < p.offsets[p.G]) {
-      const int g = find_group_of(p.offsets, p.G, pos);
+    int h = 0;
+    const int g = n_le - 1;
+    if (g >= 0 && pos < p.offsets[p.G]) {
       const int sl = p.group_slice ? p.group_slice[g] : g;
       if (sl >= 0 && sl < p.T) h = p.heads[sl];
-      blk = p.grouped ? pos : p.perm[pos];
-      if (blk < 0) h = 0;
+      if (blk_reg < 0) h = 0;
     }
     s_info[0] = h;
-    s_info[1] = blk;
+    s_info[1] = blk_reg;
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
     *abort_flag = 0;
@@ -107,52 +121,43 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
   const int N = p.N;
   const int64_t row0 = (int64_t)s_info[1] * N;
   const int npad = (N + 15) & ~15;
-  const int nhalves = N > 128 ? 2 : 1;
+  const int kboxes = npad > 128 ? 2 : 1;
 
   if (warp == 0) {
-    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_alloc(smem_u32(tmem_slot), kAttTmemCols);
     tmem_relinquish();
   }
   if (tid == 0) {
-    mbar_expect_tx(bar_load, kKBytes + kVBytes + kQBytes);
-    for (int b2 = 0; b2 < 2; ++b2) {
+    mbar_expect_tx(bar_load, (uint32_t)kboxes * 2u * 16384u + kQBytes);
+    for (int b2 = 0; b2 < kboxes; ++b2) {
       tma_load_3d(k_s + b2 * 16384, &p.map, 0, head * 3 + 1, (int)row0 + 128 * b2, bar_load);
       tma_load_3d(v_s + b2 * 16384, &p.map, 0, head * 3 + 2, (int)row0 + 128 * b2, bar_load);
-      tma_load_3d(q_s + b2 * 16384, &p.map, 0, head * 3 + 0, (int)row0 + 128 * b2, bar_load);
     }
+    tma_load_3d(q_s, &p.map, 0, head * 3 + 0, (int)row0 + 128 * half, bar_load);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // up to 224 keys: both halves' S accumulators (224 columns each) and O fit in the 512 columns and both
-  // S products are issued at once; above that one S accumulator (256 columns) is reused by the halves
-  const bool two_s = npad <= (int)kSCols;
-  const uint32_t tmem_O = tmem_base + (two_s ? 2 * kSCols : 256);
   const uint32_t idesc_s = make_idesc(128, npad);
   const uint32_t idesc_o = make_idesc(128, 64) | (1u << 16);  // B operand MN-major
   const float sl2 = 0.125f * 1.4426950408889634f;             // 1/sqrt(64) * log2(e)
 
   bool ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag, p.status, 21) ? 1 : 0) != 0;
-  uint32_t mma_phase = 0;
   if (ok) {
     // V rows >= N belong to the next sample (or to nobody): clear them so that 0 * garbage cannot appear
     for (int e = tid; e < (npad - N) * 8; e += kAttThreads)
       *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
     fence_async_smem();
     __syncthreads();
-    if (tid == 0) {  // S for both halves of the queries
+    if (tid == 0) {
       tc_fence_after();
-      for (int half = 0; half < (two_s ? nhalves : 1); ++half) {
-        const uint64_t dq = make_smem_desc(q_s + half * 16384), dk = make_smem_desc(k_s);
+      const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tmem_base + half * kSCols, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-      }
+      for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_base, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
       umma_commit(bar_mma);
     }
-    ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, abort_flag, p.status, 22) ? 1 : 0) != 0;
-    mma_phase ^= 1u;
+    ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag, p.status, 22) ? 1 : 0) != 0;
   }
 
   const int part = warp >> 2;                 // which half of the keys this thread owns
@@ -160,39 +165,42 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
   const int cols_per = npad >> 1;             // keys per part, a multiple of 8
   const int cbeg = part * cols_per;
 
-  for (int half = 0; half < nhalves && ok; ++half) {
-    if (!two_s && half == 1) {  // second S product into the accumulator the first half has finished reading
-      if (tid == 0) {
-        tc_fence_after();
-        const uint64_t dq = make_smem_desc(q_s + 16384), dk = make_smem_desc(k_s);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_base, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-        umma_commit(bar_mma);
-      }
-      ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, abort_flag, p.status, 24) ? 1 : 0) != 0;
-      mma_phase ^= 1u;
-      if (!ok) break;
-    }
+  if (ok) {
     tc_fence_after();
-    const uint32_t trow = tmem_base + (two_s ? half * kSCols : 0) + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     // ---- this thread's part of the S row, in registers
     uint32_t v[4][32];
 #pragma unroll
     for (int c = 0; c < 4; ++c)
       if (32 * c < cols_per) tmem_ld_32x32(trow + cbeg + 32 * c, v[c]);  // uniform over the CTA
     tmem_ld_wait();
+    // Keys >= N (next sample's rows, or padding) are masked once, by overwriting their scores with -inf
+    // in the one 32-key block of this thread that straddles N; everything after that is free of
+    // per-element bounds checks (the inner loops are instruction-issue bound).
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int kb = cbeg + 32 * c;  // first key of the block
+      if (32 * c < cols_per && kb + 32 > N) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (kb + i >= N) v[c][i] = 0xff800000u;  // -inf
+      }
+    }
     float mx = -INFINITY;
 #pragma unroll
     for (int c = 0; c < 4; ++c)
+      if (32 * c < cols_per) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int j = 32 * c + i;
-        if (j < cols_per && cbeg + j < N) mx = fmaxf(mx, __uint_as_float(v[c][i]));
+        for (int i = 0; i < 32; i += 2)
+          if (32 * c + i < cols_per)  // whole blocks except the last one of the part; multiple of 8, compile-time stride
+            mx = fmaxf(mx, fmaxf(__uint_as_float(v[c][i]), __uint_as_float(v[c][i + 1])));
       }
     s_red[part * 128 + m] = mx;
-    __syncthreads();
+    tc_fence_before();
+    __syncthreads();  // also: every thread has its S values, and K and Q are no longer needed
     mx = fmaxf(s_red[m], s_red[128 + m]);
     __syncthreads();
+    const float mxs = mx * sl2;
     float sum = 0.f;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -203,12 +211,12 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const int j = j0 + 2 * e;
-            float a = 0.f, b = 0.f;
-            if (cbeg + j < N) a = exp2f((__uint_as_float(v[c][8 * jv + 2 * e]) - mx) * sl2);
-            if (cbeg + j + 1 < N) b = exp2f((__uint_as_float(v[c][8 * jv + 2 * e + 1]) - mx) * sl2);
+            // exp2(s * c - max * c): one FMA and one special-function instruction per key; -inf gives 0
+            float a, b;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[c][8 * jv + 2 * e]), sl2, -mxs)));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[c][8 * jv + 2 * e + 1]), sl2, -mxs)));
+            sum += a + b;
             __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
-            sum += __low2float(hb) + __high2float(hb);  // the rounded probabilities are what the MMA multiplies
             w[e] = *reinterpret_cast<uint32_t*>(&hb);
           }
           const int key = cbeg + j0;
@@ -223,22 +231,20 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
     __syncthreads();
     sum = s_red[m] + s_red[128 + m];
 
-    // ---- O = P V
+    // ---- O = P V, into the columns S occupied
     if (tid == 0) {
       tc_fence_after();
       for (int ks = 0; ks < npad / 16; ++ks) {
         const uint64_t dp = make_smem_desc(p_s + (ks >> 2) * 16384) + 2u * (ks & 3);
         const uint64_t dv = make_smem_desc_mn(v_s + ks * 2048);
-        umma_bf16(tmem_O, dp, dv, idesc_o, ks > 0 ? 1u : 0u);
+        umma_bf16(tmem_base, dp, dv, idesc_o, ks > 0 ? 1u : 0u);
       }
       umma_commit(bar_mma);
     }
-    ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, abort_flag, p.status, 23) ? 1 : 0) != 0;
-    mma_phase ^= 1u;
-    if (!ok) break;
-    tc_fence_after();
-    {
-      const uint32_t orow = tmem_O + ((uint32_t)((warp & 3) * 32) << 16) + 32 * part;
+    ok = __syncthreads_and(mbar_wait(bar_mma, 1, abort_flag, p.status, 23) ? 1 : 0) != 0;
+    if (ok) {
+      tc_fence_after();
+      const uint32_t orow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + 32 * part;
       const int q = half * 128 + m;
       const float inv = 1.f / sum;
       __nv_bfloat16* dst = p.out + (row0 + q) * p.ld_out + (int64_t)head * 64 + 32 * part;
@@ -259,8 +265,6 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
         }
       }
     }
-    tc_fence_before();
-    __syncthreads();  // O, the P tile and the reduction scratch are free for the next half
   }
 
   tc_fence_before();
@@ -268,7 +272,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) attention_kernel(const __grid_
   if (warp == 0) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, kAttTmemCols);
   }
 }
 
@@ -292,12 +296,12 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   p.qkv = static_cast<const __nv_bfloat16*>(qkv); p.ld_qkv = ld_qkv;
   p.out = static_cast<__nv_bfloat16*>(out); p.ld_out = ld_out;
   p.status = status;
-  const size_t smem = 1024 + 2048 + kQBytes + kKBytes + kVBytes + kPBytes;
+  const size_t smem = 1024 + 2048 + kVBytes + kPBytes;  // P overlays K, Q and 16 KB more
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return dsn_launch(attention_kernel, dim3(H, B), dim3(kAttThreads), smem, s, 1, p);
+  return dsn_launch(attention_kernel, dim3(H, B, N > 128 ? 2 : 1), dim3(kAttThreads), smem, s, 1, p);
 }
