@@ -184,11 +184,13 @@ def split_bn(z, t, gamma, beta, mu, sigma):
     return g * ((z - m) / s) + b
 
 
-def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None):
+def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None, residual=None):
     """y[i][r][o] = act(b[o] + sum_{c<k_in[t]} x[i][r][c] W[o][c]),  o < k_out[t],  t = idx[i].
 
     bn = (gamma[C_out], beta[C_out], mu[T][C_out], sigma[T][C_out]) inserts Re-SBN between the
-    contraction (+ bias) and the activation.
+    contraction (+ bias) and the activation; residual [B][R][C_out] (the skip features of a residual block,
+    Sec. 5 "DS-ResNet": shortcut and residual output have the same sliced width) is added just before the
+    activation.
     x [B][R][C_in], W [C_out][C_in] (stored [out][in]).  Entries with o >= k_out[t] are not part
     of the result and hold `fill`.  `samples` restricts evaluation to a subset of samples (others
     hold `fill`); the per-sample definition makes that exact.
@@ -205,13 +207,15 @@ def sliced_linear(x, W, idx, k_in, k_out, bias=None, act=ACT_NONE, fill=np.nan, 
         z = x[i, :, :ki] @ W[:ko, :ki].T
         if bias is not None:
             z = z + np.asarray(bias, dtype=F64)[:ko]
-        if bn is not None:                          # layer -> Re-SBN -> activation
+        if bn is not None:                          # layer -> Re-SBN -> (+ shortcut) -> activation
             z = split_bn(z, t, *bn)
+        if residual is not None:                    # residual block: the skip features are added before the activation
+            z = z + np.asarray(residual, dtype=F64)[i, :, :ko]
         y[i, :, :ko] = activation(z, act)
     return y
 
 
-def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None):
+def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.nan, samples=None, bn=None, residual=None):
     """Slice-able convolution, stride 1, zero padding, no kernel flip.
 
     x [B][H][W][C_in] (channels last), W [C_O][C_I][K][K] (the paper's indexing).
@@ -238,6 +242,8 @@ def sliced_conv(x, W, idx, k_in, k_out, pad, bias=None, act=ACT_NONE, fill=np.na
             z = z + np.asarray(bias, dtype=F64)[:ko]
         if bn is not None:
             z = split_bn(z, t, *bn)
+        if residual is not None:
+            z = z + np.asarray(residual, dtype=F64)[i, :, :, :ko]
         y[i, :, :, :ko] = activation(z, act)
     return y
 

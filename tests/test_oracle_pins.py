@@ -349,6 +349,25 @@ def test_split_bn_library_brute_force_and_identity():
     assert ident.shape == (2, 3, 5)
 
 
+def test_residual_add_before_activation():
+    B, H, Wd, C = 2, 3, 3, 6
+    x, W, res = rand(B, H, Wd, C), rand(C, C, 1, 1), rand(B, H, Wd, C)
+    idx = np.array([0, 1]); k = [4, 6]
+    plain = O.sliced_conv(x, W, idx, k, k, 0)
+    got = O.sliced_conv(x, W, idx, k, k, 0, act=O.ACT_RELU, residual=res)
+    for i in range(B):
+        w = k[idx[i]]
+        np.testing.assert_allclose(got[i, ..., :w], np.maximum(plain[i, ..., :w] + res[i, ..., :w], 0.0), rtol=0, atol=1e-15)
+        assert np.all(np.isnan(got[i, ..., w:]))
+    # library form of a residual block tail: relu(conv(x) + shortcut)
+    xt = torch.from_numpy(x[:1, ..., :4].copy()).permute(0, 3, 1, 2)
+    ref = torch.relu(torch.nn.functional.conv2d(xt, torch.from_numpy(W[:4, :4].copy())) +
+                     torch.from_numpy(res[:1, ..., :4].copy()).permute(0, 3, 1, 2))
+    np.testing.assert_allclose(got[0, ..., :4], ref[0].permute(1, 2, 0).numpy(), rtol=1e-12, atol=1e-12)
+    lin = O.sliced_linear(x.reshape(B, 9, C), W[:, :, 0, 0], idx, k, k, residual=res.reshape(B, 9, C))
+    np.testing.assert_allclose(lin[0, :, :4], (plain[0] + res[0]).reshape(9, C)[:, :4], rtol=0, atol=1e-15)
+
+
 # ------------------------------------------------------------------ routing
 @pytest.mark.parametrize("B,T", [(1, 1), (7, 1), (1, 5), (33, 4), (100, 14), (64, 48)])
 def test_route_invariants(B, T):
