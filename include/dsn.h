@@ -100,7 +100,9 @@ typedef struct dsn_linear_desc {
   const float* bias;    /* device [C_out] fp32 or NULL                                   */
   const float* bn_scale;/* device [T][C_out] fp32 or NULL: per-path affine a_t of Re-SBN (dsn_resbn_fold) */
   const float* bn_shift;/* device [T][C_out] fp32 (required with bn_scale): b_t          */
-  int32_t act;          /* dsn_act; order of operations: contraction, + bias, * a_t + b_t, activation */
+  const void* residual; /* device, same dtype, order and leading dimension as y, or NULL: the skip features of a
+                           residual block (Sec. 5, DS-ResNet), added before the activation; may not alias y */
+  int32_t act;          /* dsn_act; order of operations: contraction, + bias, * a_t + b_t, + residual, activation */
   int32_t in_order;     /* dsn_order of x: INPUT_ORDER [B][R][ldx] by sample, or GROUPED by position */
   int32_t out_order;    /* dsn_order of y                                                */
   int32_t tail;         /* dsn_tail: columns >= k_out[t] left untouched, or zero-filled up to C_out */
@@ -121,6 +123,7 @@ typedef struct dsn_conv_desc {
   const float* bias;
   const float* bn_scale;/* as in dsn_linear_desc                                         */
   const float* bn_shift;
+  const void* residual; /* as in dsn_linear_desc                                         */
   int32_t act;
   int32_t in_order, out_order, tail;
 } dsn_conv_desc;

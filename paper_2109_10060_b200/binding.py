@@ -52,8 +52,8 @@ class LinearDesc(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("R", C.c_int32), ("C_in", C.c_int32), ("C_out", C.c_int32),
                 ("ldx", C.c_int64), ("ldw", C.c_int64), ("ldy", C.c_int64), ("T", C.c_int32),
                 ("k_in", C.POINTER(C.c_int32)), ("k_out", C.POINTER(C.c_int32)), ("W", C.c_void_p),
-                ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p), ("act", C.c_int32),
-                ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
+                ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p), ("residual", C.c_void_p),
+                ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
 
 
 class ConvDesc(C.Structure):
@@ -61,7 +61,8 @@ class ConvDesc(C.Structure):
                 ("C_in", C.c_int32), ("C_out", C.c_int32), ("ldx", C.c_int64), ("ldy", C.c_int64),
                 ("T", C.c_int32), ("k_in", C.POINTER(C.c_int32)), ("k_out", C.POINTER(C.c_int32)),
                 ("W", C.c_void_p), ("bias", C.c_void_p), ("bn_scale", C.c_void_p), ("bn_shift", C.c_void_p),
-                ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32), ("tail", C.c_int32)]
+                ("residual", C.c_void_p), ("act", C.c_int32), ("in_order", C.c_int32), ("out_order", C.c_int32),
+                ("tail", C.c_int32)]
 
 
 class AttentionDesc(C.Structure):
@@ -209,22 +210,23 @@ def make_gate_desc(dtype, B, R, C_full, C_mlp, T, W1, W2, b1=None, b2=None, c_va
 
 def make_linear_desc(dtype, R, C_in, C_out, k_in, k_out, W, bias=None, act=ACT_NONE, in_order=INPUT_ORDER,
                      out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldw=None, ldy=None, bn_scale=None,
-                     bn_shift=None) -> LinearDesc:
+                     bn_shift=None, residual=None) -> LinearDesc:
     ki, ko = _i32_array(k_in), _i32_array(k_out)
     d = LinearDesc(dtype, R, C_in, C_out, C_in if ldx is None else ldx, C_in if ldw is None else ldw,
                    C_out if ldy is None else ldy, len(k_in), ki, ko, _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift),
-                   act, in_order, out_order, tail)
-    d._keep = (ki, ko, W, bias, bn_scale, bn_shift)
+                   _ptr(residual), act, in_order, out_order, tail)
+    d._keep = (ki, ko, W, bias, bn_scale, bn_shift, residual)
     return d
 
 
 def make_conv_desc(dtype, H, Wd, K, pad, C_in, C_out, k_in, k_out, W, bias=None, act=ACT_NONE,
                    in_order=INPUT_ORDER, out_order=INPUT_ORDER, tail=TAIL_UNTOUCHED, ldx=None, ldy=None, bn_scale=None,
-                   bn_shift=None) -> ConvDesc:
+                   bn_shift=None, residual=None) -> ConvDesc:
     ki, ko = _i32_array(k_in), _i32_array(k_out)
     d = ConvDesc(dtype, H, Wd, K, pad, C_in, C_out, C_in if ldx is None else ldx, C_out if ldy is None else ldy,
-                 len(k_in), ki, ko, _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift), act, in_order, out_order, tail)
-    d._keep = (ki, ko, W, bias, bn_scale, bn_shift)
+                 len(k_in), ki, ko, _ptr(W), _ptr(bias), _ptr(bn_scale), _ptr(bn_shift), _ptr(residual), act, in_order,
+                 out_order, tail)
+    d._keep = (ki, ko, W, bias, bn_scale, bn_shift, residual)
     return d
 
 

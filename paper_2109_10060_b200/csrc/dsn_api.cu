@@ -61,6 +61,7 @@ struct LayerCall {
   const void* Wt;
   const float* bias;
   const float *bn_scale, *bn_shift;
+  const void* residual;
   int act, in_order, out_order, tail;
   const dsn_attention_desc* att;  // non-null: this chain element is the attention core, not a sliced layer
 };
@@ -82,6 +83,8 @@ int check_routing(const dsn_routing* r, int T) {
 int validate_call(const LayerCall& c, const dsn_routing* r, const void* x, const void* y) {
   if (!x || !y || !c.Wt) return DSN_ERR_INVALID_ARG;
   if ((c.bn_scale == nullptr) != (c.bn_shift == nullptr)) return DSN_ERR_INVALID_ARG;
+  if (c.residual && c.residual == y) return DSN_ERR_INVALID_ARG;
+  if (c.residual && c.dtype == DSN_BF16 && !aligned16(c.residual)) return DSN_ERR_ALIGNMENT;
   if (c.dtype != DSN_BF16 && c.dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
   if (c.H < 1 || c.W < 1 || c.C_in < 1 || c.C_out < 1 || c.C_in > 32767 || c.C_out > 32767) return DSN_ERR_INVALID_ARG;
   if (c.act < DSN_ACT_NONE || c.act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
@@ -171,6 +174,7 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
   p.bn_scale = c.bn_scale;
   p.bn_shift = c.bn_shift;
   p.bn_ld = c.C_out;
+  p.residual = static_cast<const __nv_bfloat16*>(c.residual);
   p.act = c.act;
   p.status = ctx->d_status;
   for (int t = 0; t < c.T; ++t) {
@@ -270,7 +274,7 @@ int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void
   } else {
     if (dsn_launch_linear_f32(st, c.T, c.H * c.W, static_cast<const float*>(x), c.ldx,
                               static_cast<const float*>(c.Wt), c.w_row, static_cast<float*>(y), c.ldy, c.bias, c.bn_scale, c.bn_shift,
-                              c.C_out, c.act,
+                              c.C_out, static_cast<const float*>(c.residual), c.act,
                               c.in_order == DSN_INPUT_ORDER, c.out_order == DSN_INPUT_ORDER, r->B, r->G, r->offsets,
                               r->perm, r->group_slice, ctx->sm_count, s) != cudaSuccess)
       return DSN_ERR_CUDA;
@@ -292,7 +296,7 @@ LayerCall from_linear(const dsn_linear_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = d->ldw; c.w_tap = d->ldw;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.att = nullptr;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.residual = d->residual; c.att = nullptr;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -305,7 +309,7 @@ LayerCall from_conv(const dsn_conv_desc* d) {
   c.ldx = d->ldx; c.ldy = d->ldy;
   c.w_row = (int64_t)d->K * d->K * d->C_in; c.w_tap = d->C_in;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
-  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.att = nullptr;
+  c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.residual = d->residual; c.att = nullptr;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }

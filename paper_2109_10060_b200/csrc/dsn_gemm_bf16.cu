@@ -251,6 +251,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
       const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      const __nv_bfloat16* res_row = (p.residual && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
@@ -265,14 +266,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
       const CUtensorMap* mY = &p.mapY[t.map];
-      const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
+      const int variant = p.act * 2 + ((brow || sc_row || p.residual) ? 1 : 0);
       switch (variant) {
-        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
       }
       tc_fence_before();
       __syncwarp();

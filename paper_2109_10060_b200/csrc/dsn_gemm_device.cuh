@@ -187,7 +187,7 @@ __device__ __forceinline__ float apply_act(float v) {
 // lanes store one 128-byte piece of a row each.
 template <int ACT, bool AFF>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
-                                              const float* sc_row, const float* sh_row, uint8_t* stage_w, __nv_bfloat16* yrow, int lane, bool contig,
+                                              const float* sc_row, const float* sh_row, const __nv_bfloat16* res_row, uint8_t* stage_w, __nv_bfloat16* yrow, int lane, bool contig,
                                               const CUtensorMap* mapY, int base_row) {
   for (int c0 = 64 * first; c0 < ncols; c0 += 128) {
     // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
@@ -209,14 +209,16 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
           for (int e = 0; e < 4; ++e) {
             const int c = 8 * jj + 2 * e;
             float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
-            if (AFF) {  // bias and / or the per-path Re-SBN scale and shift of this tile's columns
+            if (AFF) {  // bias, the per-path Re-SBN scale and shift of this tile's columns, the skip features of this row
               if (cb + c < ncols) {
                 if (brow) a += __ldg(brow + cb + c);
                 if (sc_row) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
+                if (res_row) a += __bfloat162float(res_row[cb + c]);
               }
               if (cb + c + 1 < ncols) {
                 if (brow) b += __ldg(brow + cb + c + 1);
                 if (sc_row) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
+                if (res_row) b += __bfloat162float(res_row[cb + c + 1]);
               }
             }
             __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));

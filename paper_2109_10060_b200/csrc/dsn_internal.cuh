@@ -104,6 +104,7 @@ struct GemmParams {
   const float* bn_scale;  // [T][bn_ld] per-path affine of Re-SBN, or nullptr
   const float* bn_shift;
   int32_t bn_ld;
+  const __nv_bfloat16* residual;  // laid out like y (same rows, same leading dimension), or nullptr
   int32_t act;
   int32_t* status;
 };
@@ -148,7 +149,7 @@ struct SliceTable {
 
 cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const float* x, int64_t ldx,
                                   const float* W, int64_t ldw, float* y, int64_t ldy, const float* bias,
-                                  const float* bn_scale, const float* bn_shift, int bn_ld, int act, int x_input_order, int y_input_order, int B, int G,
+                                  const float* bn_scale, const float* bn_shift, int bn_ld, const float* residual, int act, int x_input_order, int y_input_order, int B, int G,
                                   const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                   int sm_count, cudaStream_t s);
 

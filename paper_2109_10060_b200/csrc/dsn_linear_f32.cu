@@ -17,7 +17,8 @@ __device__ __forceinline__ float apply_act(float v, int act) {
 __global__ void __launch_bounds__(kThreads)
 linear_f32_kernel(SliceTable st, int R, const float* __restrict__ x, int64_t ldx, const float* __restrict__ W,
                   int64_t ldw, float* __restrict__ y, int64_t ldy, const float* __restrict__ bias,
-                  const float* __restrict__ bn_scale, const float* __restrict__ bn_shift, int bn_ld, int act,
+                  const float* __restrict__ bn_scale, const float* __restrict__ bn_shift, int bn_ld,
+                  const float* __restrict__ residual, int act,
                   int x_input_order, int y_input_order, int G, const int32_t* __restrict__ offsets,
                   const int32_t* __restrict__ perm, const int32_t* __restrict__ group_slice) {
   extern __shared__ int32_t s_prefix[];  // [G+1]
@@ -106,6 +107,7 @@ linear_f32_kernel(SliceTable st, int R, const float* __restrict__ x, int64_t ldx
         if (n < ko) {
           float v = acc[i][q] + (bias ? bias[n] : 0.f);
           if (bn_scale) v = fmaf(v, bn_scale[(int64_t)sl * bn_ld + n], bn_shift[(int64_t)sl * bn_ld + n]);
+          if (residual) v += residual[((int64_t)smp * R + rr) * ldy + n];
           yr[n] = apply_act(v, act);
         }
       }
@@ -117,7 +119,7 @@ linear_f32_kernel(SliceTable st, int R, const float* __restrict__ x, int64_t ldx
 
 cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const float* x, int64_t ldx,
                                   const float* W, int64_t ldw, float* y, int64_t ldy, const float* bias,
-                                  const float* bn_scale, const float* bn_shift, int bn_ld, int act, int x_input_order, int y_input_order, int B, int G,
+                                  const float* bn_scale, const float* bn_shift, int bn_ld, const float* residual, int act, int x_input_order, int y_input_order, int B, int G,
                                   const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                   int sm_count, cudaStream_t s) {
   (void)T;
@@ -128,6 +130,6 @@ cudaError_t dsn_launch_linear_f32(const SliceTable& st, int T, int R, const floa
   int64_t grid = bound < (int64_t)sm_count * 4 ? bound : (int64_t)sm_count * 4;
   if (grid < 1) grid = 1;
   return dsn_launch(linear_f32_kernel, dim3((unsigned)grid), dim3(kThreads), sizeof(int32_t) * (G + 1), s, 1, st, R, x,
-                    ldx, W, ldw, y, ldy, bias, bn_scale, bn_shift, bn_ld, act, x_input_order, y_input_order, G, offsets, perm,
+                    ldx, W, ldw, y, ldy, bias, bn_scale, bn_shift, bn_ld, residual, act, x_input_order, y_input_order, G, offsets, perm,
                     group_slice);
 }

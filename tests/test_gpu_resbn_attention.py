@@ -136,3 +136,58 @@ def test_gate_attention_head_and_scaling(dsn, ctx, B, R, C, M, T, cv):
     assert np.all(got[..., c_valid:] == SENTINEL) and np.all(gotg[..., c_valid:] == SENTINEL)
     # almost every element is the correctly rounded product (a different fp32 scale can flip a rounding)
     assert np.mean(got[..., :c_valid] != ref) < 0.02
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_residual_block_tail_with_sliced_shortcut(dsn, ctx, dtype):
+    """DS-ResNet first block of a stage: every width of the block follows the path, including the projection
+    shortcut; out = ReLU(Re-SBN(conv3(h)) + shortcut(x)) with shortcut = sliced 1x1 convolution."""
+    g = np.random.default_rng(21)
+    if dtype == "bf16":
+        B, hw, Cin, Cmid, Cout = 12, 14, 256, 128, 512
+    else:
+        B, hw, Cin, Cmid, Cout = 9, 1, 64, 32, 48          # the fp32 kernel is linear only (one row per sample)
+    ratios = [0.25, 0.5, 0.75, 1.0]
+    T = 4
+    k_in = [int(Cin * r) for r in ratios]
+    k_mid = [int(Cmid * r) for r in ratios]
+    k_out = [int(Cout * r) for r in ratios]
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    mk = (lambda a: wl.to_bf16_values(a)) if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    x = mk(np.maximum(g.standard_normal((B, hw, hw, Cin)), 0).astype(np.float32))
+    h = mk(np.maximum(g.standard_normal((B, hw, hw, Cmid)), 0).astype(np.float32))
+    Ws = mk((g.standard_normal((Cout, Cin, 1, 1)) * Cin ** -0.5).astype(np.float32))
+    W3 = mk((g.standard_normal((Cout, Cmid, 1, 1)) * Cmid ** -0.5).astype(np.float32))
+    gamma = (1.0 + 0.2 * g.standard_normal(Cout)).astype(np.float32)
+    beta = (0.3 * g.standard_normal(Cout)).astype(np.float32)
+    mu = (0.2 * g.standard_normal((T, Cout))).astype(np.float32)
+    sigma = (0.6 + np.abs(g.standard_normal((T, Cout))) * 0.5).astype(np.float32)
+    sc, sh = fold_on_gpu(dsn, ctx, gamma, beta, mu, sigma)
+    r = route_on_gpu(dsn, ctx, idx, T)
+    if dtype == "bf16":
+        up, tdt, code = up_bf16, torch.bfloat16, dsn.BF16
+        short = torch.full((B, hw, hw, Cout), SENTINEL, dtype=tdt, device=DEV)
+        y = torch.full((B, hw, hw, Cout), SENTINEL, dtype=tdt, device=DEV)
+        dsn.dsn_sliced_conv(ctx, dsn.make_conv_desc(code, hw, hw, 1, 0, Cin, Cout, k_in, k_out, up(Ws.reshape(Cout, Cin))), r, up(x), short)
+        dsn.dsn_sliced_conv(ctx, dsn.make_conv_desc(code, hw, hw, 1, 0, Cmid, Cout, k_mid, k_out, up(W3.reshape(Cout, Cmid)),
+                                                    act=dsn.ACT_RELU, bn_scale=sc, bn_shift=sh, residual=short), r, up(h), y)
+    else:
+        up, tdt, code = up_f32, torch.float32, dsn.F32
+        short = torch.full((B, 1, Cout), SENTINEL, dtype=tdt, device=DEV)
+        y = torch.full((B, 1, Cout), SENTINEL, dtype=tdt, device=DEV)
+        dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(code, 1, Cin, Cout, k_in, k_out, up(Ws.reshape(Cout, Cin))), r,
+                              up(x.reshape(B, 1, Cin)), short)
+        dsn.dsn_sliced_linear(ctx, dsn.make_linear_desc(code, 1, Cmid, Cout, k_mid, k_out, up(W3.reshape(Cout, Cmid)),
+                                                        act=dsn.ACT_RELU, bn_scale=sc, bn_shift=sh, residual=short), r,
+                              up(h.reshape(B, 1, Cmid)), y)
+    check_status(ctx, dsn)
+    s_ref = O.sliced_conv(x, Ws, idx, k_in, k_out, 0, fill=0.0)
+    if dtype == "bf16":
+        s_ref = O.round_bf16(s_ref)
+    ref = O.sliced_conv(h, W3, idx, k_mid, k_out, 0, act=O.ACT_RELU, bn=(gamma, beta, mu, sigma), residual=s_ref)
+    got = down(y).reshape(B, hw, hw, Cout)
+    if dtype == "bf16":
+        ref = O.round_bf16(ref)
+    errs = group_errors(got, ref, idx, k_out, T)
+    assert max(errs.values()) <= (1e-2 if dtype == "bf16" else 2e-5), errs     # bf16: two chained stages
+    assert_tail_untouched(got, idx, k_out)
