@@ -310,6 +310,17 @@ def run_table(args):
         with torch.cuda.stream(side):
             call(0)
         torch.cuda.synchronize()
+        if args.no_graph:   # direct calls (for profilers): two passes over the buffers, the second one timed
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(side):
+                for i in range(nbuf):
+                    call(i)
+                e0.record(side)
+                for i in range(nbuf):
+                    call(i)
+                e1.record(side)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / nbuf * 1e3
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=side):
             for i in range(nbuf):
@@ -327,7 +338,18 @@ def run_table(args):
     print("| config | layer | routing | us | executed TFLOP/s | % measured BF16 peak | bound (TFLOP/s) | % of bound | GB/s | samples/s |")
     print("|---|---|---|---|---|---|---|---|---|---|")
 
+    import re
+    want = (lambda *names: re.search(args.table_filter, " ".join(names)) is not None) if args.table_filter else (lambda *names: True)
+    div = max(1, args.table_batch_div)
+
     def layer(cfgname, lname, rname, B, H, Cin, Cout, k_in, k_out, idx, K=1, act=0, orders=(1, 1), group_list=None):
+        if not want(cfgname, lname, rname):
+            return
+        if div > 1:
+            if group_list is not None:
+                return
+            B = B // div
+            idx = idx[:B]
         T = len(k_in)
         R = H * H if K == 3 else H
         if group_list is None:
@@ -361,6 +383,9 @@ def run_table(args):
         del xs, ys
 
     def gate_route(cfgname, B, R, C, T):
+        if not want(cfgname, "gate route", "-"):
+            return
+        B = B // div
         per = B * R * C * 2
         nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
         xs = [torch.randn(B, R, C, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
@@ -399,6 +424,10 @@ def run_table(args):
         ki, ko = wl.vit_layer_slices(paths, 64, lname)
         layer("cfg3", lname, "uniform", B, 197, Cin, Cout, ki, ko, idx, act=act)
     def attention(cfgname, B, N, H, heads, idx, rname):
+        if not want(cfgname, "attention core", rname):
+            return
+        B = B // div
+        idx = idx[:B]
         T = len(heads)
         r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
         dsn.dsn_route(ctx, ints(idx), B, T, r)
@@ -441,6 +470,8 @@ def run_table(args):
         idx = wl.idx_quota_uniform(wl.rng(6, 6), 256, 14)
         layer(f"M {hw}x{hw}", f"pointwise 1x1 c->c (full {C})", "uniform", 256, hw * hw, C, C, widths, widths, idx, act=1)
     # config 1: fp32 single layer
+    if not want("cfg1", "fp32 linear", "iid"):
+        return
     c1 = wl.config1()
     x, W = torch.from_numpy(c1["x"]).to(dev), torch.from_numpy(c1["W"]).to(dev)
     y = torch.zeros(64, 1, 256, device=dev)
@@ -463,6 +494,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="print per-layer markdown rows for every configuration")
     ap.add_argument("--no-graph", action="store_true", help="time direct API calls instead of a CUDA-graph replay (for profilers)")
+    ap.add_argument("--table-filter", default=None, help="with --table: only rows whose 'config layer routing' text matches this regular expression")
+    ap.add_argument("--table-batch-div", type=int, default=1, help="with --table: divide every batch size by this (small cases for profilers)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

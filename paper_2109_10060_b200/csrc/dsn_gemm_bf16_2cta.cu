@@ -194,49 +194,61 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
-      bool ok = true;
-      for (int tile = pair; ok && tile < total; tile += npairs) {
-        const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
-        const CUtensorMap* mA = &p.mapA[t.map];
-        const CUtensorMap* mB = &p.mapB[t.map];
-        const int nkc = (t.ki + BK - 1) / BK;
-        int ncols = t.ko - t.n0;
-        ncols = ncols > g.BN ? g.BN : ncols;
-        const int n_inst = (ncols + 31) & ~31;
-        const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
-        int bsel = t.b0;
-        if (g.a_input_order) bsel = t.b0 < t.p_end ? p.perm[t.b0] : p.B;  // past the group: out of range, zeros
-        for (int tap = 0; ok && tap < g.taps; ++tap) {
-          const int r = tap / g.KW, s = tap - r * g.KW;
-          for (int kc = 0; kc < nkc; ++kc) {
-            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
+    // The whole warp walks the schedule (addresses, coordinates and the loop itself stay
+    // warp-uniform, which keeps the per-stage instruction count low); one elected lane issues.
+    int stage = 0;
+    uint32_t phase = 0;
+    const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
+    const uint32_t tx_bytes = 2u * (a_box_bytes + bh_bytes);
+    bool ok = true;
+    for (int tile = pair; ok && tile < total; tile += npairs) {
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const CUtensorMap* mA = &p.mapA[t.map];
+      const CUtensorMap* mB = &p.mapB[t.map];
+      const int nkc = (t.ki + BK - 1) / BK;
+      int ncols = t.ko - t.n0;
+      ncols = ncols > g.BN ? g.BN : ncols;
+      const int n_inst = (ncols + 31) & ~31;
+      const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
+      int bsel = t.b0;
+      if (g.a_input_order) bsel = t.b0 < t.p_end ? p.perm[t.b0] : p.B;  // past the group: out of range, zeros
+      for (int tap = 0; ok && tap < g.taps; ++tap) {
+        const int r = tap / g.KW, sx = tap - r * g.KW;
+        const int cx = g.flat ? t.row0 : t.x0 + sx - g.pad, cy = g.flat ? 0 : t.y0 + r - g.pad, cb = g.flat ? 0 : bsel;
+        for (int kc = 0; kc < nkc; ++kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 11));
+          if (!ok) break;
+          if (elect_one()) {
             const uint32_t full_lead = leader_addr(bar_full + 8 * stage);  // the even CTA's barrier
-            if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * (a_box_bytes + bh_bytes));
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, tx_bytes);
             const uint32_t sa = tiles_base + stage * stage_bytes;
-            if (g.flat) tma_load_4d_pair(sa, mA, kc * BK, t.row0, 0, 0, full_lead);
-            else tma_load_4d_pair(sa, mA, kc * BK, t.x0 + s - g.pad, t.y0 + r - g.pad, bsel, full_lead);
+            tma_load_4d_pair(sa, mA, kc * BK, cx, cy, cb, full_lead);
             tma_load_3d_pair(sa + kABytes, mB, kc * BK, tap, brow0, full_lead);
-            if (++stage == stages) { stage = 0; phase ^= 1u; }
           }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (even CTA only)
-    if (lane == 0 && rank == 0) {
+    // Warp-uniform loop, one elected lane issues.  The issuing warp is the critical resource of a tile with
+    // wide N (four instructions of 128 tensor-pipe cycles per stage), so the per-stage path is
+    // kept short: running descriptors, four unrolled K steps, a separate short loop for a partial
+    // last chunk.
+    if (rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
+      const uint64_t da0 = make_smem_desc(tiles_base), db0 = make_smem_desc(tiles_base + kABytes);
+      const uint64_t dstep = (uint64_t)(stage_bytes >> 4);
+      uint64_t da = da0, db = db0;
       for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
         const PairTile t = decode_pair_tile(p, s_prefix, tile, 0);
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-        if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
+        if (!ok) break;
         tc_fence_after();
         int ncols = t.ko - t.n0;
         ncols = ncols > g.BN ? g.BN : ncols;
@@ -244,24 +256,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
         const uint32_t idesc = make_idesc(2 * BM, n_inst);
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
         const int nkc = (t.ki + BK - 1) / BK;
+        const int tail_ks = ((t.ki & (BK - 1)) + 15) >> 4;  // K steps of a partial last chunk (0: none)
         uint32_t accumulate = 0;
         for (int tap = 0; ok && tap < g.taps; ++tap) {
-          for (int kc = 0; kc < nkc; ++kc) {
-            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13)) { ok = false; break; }
+          for (int kc = nkc; kc > 0; --kc) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13));
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t sa = tiles_base + stage * stage_bytes;
-            const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kABytes);
-            const int krem = t.ki - kc * BK;
-            const int nks = krem >= BK ? BK / 16 : (krem + 15) >> 4;
-            for (int ks = 0; ks < nks; ++ks) {
-              umma_bf16_pair(d_tmem, da + 2u * ks, db + 2u * ks, idesc, accumulate);
-              accumulate = 1;
+            const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
+            if (elect_one()) {
+              umma_bf16_pair(d_tmem, da, db, idesc, accumulate);  // +32 bytes per K step
+              if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, db + 2u, idesc, 1u);
+              if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, db + 4u, idesc, 1u);
+              if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, db + 6u, idesc, 1u);
+              umma_commit_pair(bar_empty + 8 * stage);
             }
-            umma_commit_pair(bar_empty + 8 * stage);
-            if (++stage == stages) { stage = 0; phase ^= 1u; }
+            accumulate = 1;
+            da += dstep;
+            db += dstep;
+            if (++stage == stages) { stage = 0; phase ^= 1u; da = da0; db = db0; }
           }
         }
-        if (ok) umma_commit_pair(bar_tfull + 8 * acc);
+        if (ok && elect_one()) umma_commit_pair(bar_tfull + 8 * acc);
       }
     }
   } else {
