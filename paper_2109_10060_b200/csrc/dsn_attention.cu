@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
     tmem_alloc(smem_u32(tmem_slot), kAttTmemCols);
     tmem_relinquish();
   }
-  if (tid == 0) {
+  if (warp == 0 && elect_one()) {  // one elected lane of a converged warp: operands stay in uniform registers
     mbar_expect_tx(bar_load, (uint32_t)kboxes * 2u * 16384u + kQBytes);
     for (int b2 = 0; b2 < kboxes; ++b2) {
       tma_load_3d(k_s + b2 * 16384, &p.map, 0, head * 3 + 1, (int)row0 + 128 * b2, bar_load);
@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
       *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
     fence_async_smem();
     __syncthreads();
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
       tc_fence_after();
       const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
 #pragma unroll
@@ -232,7 +232,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
     sum = s_red[m] + s_red[128 + m];
 
     // ---- O = P V, into the columns S occupied
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
       tc_fence_after();
       for (int ks = 0; ks < npad / 16; ++ks) {
         const uint64_t dp = make_smem_desc(p_s + (ks >> 2) * 16384) + 2u * (ks & 3);

@@ -208,7 +208,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
   for (int c0 = 64 * first; c0 < ncols; c0 += 16 * kEpiWarps) {
     // an earlier TMA store of this warp (this tile or the one before) must have finished reading the
     // staging tile before it is overwritten; free when nothing is outstanding
-    if (lane == 0) bulk_wait_read0();
+    if (elect_one()) bulk_wait_read0();
     __syncwarp();
     // phase 1: this thread's row, 64 columns -> bf16 -> its 128-byte row of the staging tile
 #pragma unroll
@@ -248,7 +248,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
     if (contig) {
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) {
+      if (elect_one()) {
         tma_store_2d(mapY, n0 + c0, base_row, smem_u32(stage_w));
         bulk_commit();
       }
