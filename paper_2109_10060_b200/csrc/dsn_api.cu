@@ -116,8 +116,8 @@ void fill_slice_table(SliceTable& st, const LayerCall& c) {
   }
 }
 
-// Tile geometry for the bf16 kernel.
-void choose_geometry(const LayerCall& c, GemmGeom& g) {
+// Tile geometry for the bf16 kernel.  `per_sample`: no tile spans two samples (chained layers).
+void choose_geometry(const LayerCall& c, GemmGeom& g, bool per_sample = false) {
   memset(&g, 0, sizeof(g));
   g.H = c.H;
   g.W = c.W;
@@ -131,7 +131,7 @@ void choose_geometry(const LayerCall& c, GemmGeom& g) {
   for (int t = 0; t < c.T; ++t) max_ko = c.k_out[t] > max_ko ? c.k_out[t] : max_ko;
   g.BN = max_ko > 128 ? 256 : (max_ko > 64 ? 128 : 64);
   g.stages = g.BN == 256 ? 4 : (g.BN == 128 ? 6 : 8);
-  if (c.K == 1 && !g.a_input_order) {
+  if (c.K == 1 && !g.a_input_order && !per_sample) {
     g.flat = 1;  // grouped rows are contiguous: tile them without regard to sample boundaries
     g.bw = DSN_GEMM_BM;
     g.bh = g.nb = g.tiles_x = g.tiles_y = 1;
@@ -149,7 +149,7 @@ void choose_geometry(const LayerCall& c, GemmGeom& g) {
     g.bh = (g.H + bands - 1) / bands;
   }
   g.nb = 1;
-  if (!g.a_input_order && g.bh == g.H && g.bw == g.W) {
+  if (!g.a_input_order && !per_sample && g.bh == g.H && g.bw == g.W) {
     g.nb = DSN_GEMM_BM / (g.bw * g.bh);
     if (g.nb < 1) g.nb = 1;
   }
@@ -157,11 +157,10 @@ void choose_geometry(const LayerCall& c, GemmGeom& g) {
   g.tiles_y = (g.H + g.bh - 1) / g.bh;
 }
 
-int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
-  GemmParams p;
+// Everything of the kernel parameters except the tensor maps.
+void fill_gemm_params(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, void* y, bool per_sample, GemmParams& p) {
   memset(&p, 0, sizeof(p));
-  choose_geometry(c, p.g);
-  const GemmGeom& g = p.g;
+  choose_geometry(c, p.g, per_sample);
   p.B = r->B;
   p.G = r->G;
   p.T = c.T;
@@ -181,77 +180,96 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     p.k_in[t] = (int16_t)c.k_in[t];
     p.k_out[t] = (int16_t)c.k_out[t];
   }
+}
+
+// Tensor maps for the next DSN_GEMM_MAX_MAPS distinct slices (k_in, k_out) not yet done; one map
+// triple per distinct slice.  `remaining` counts the paths still without a map afterwards.
+int fill_gemm_maps(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, GemmParams& p,
+                   int* done, int& remaining) {
+  const GemmGeom& g = p.g;
+  int nmaps = 0;
+  int map_k[DSN_GEMM_MAX_MAPS], map_n[DSN_GEMM_MAX_MAPS];
+  memset(p.map_id, 0xFF, sizeof(p.map_id));
+  for (int t = 0; t < c.T; ++t) {
+    if (done[t]) continue;
+    int id = -1;
+    for (int m = 0; m < nmaps; ++m)
+      if (map_k[m] == c.k_in[t] && map_n[m] == c.k_out[t]) id = m;
+    if (id < 0) {
+      if (nmaps == DSN_GEMM_MAX_MAPS) continue;  // next launch
+      id = nmaps++;
+      map_k[id] = c.k_in[t];
+      map_n[id] = c.k_out[t];
+    }
+    p.map_id[t] = (uint8_t)id;
+    done[t] = 1;
+    --remaining;
+  }
+  for (int m = 0; m < nmaps; ++m) {
+    const uint64_t kv = (uint64_t)map_k[m];
+    int e;
+    if (g.flat) {
+      const uint64_t rows = (uint64_t)r->B * g.R;
+      const uint64_t dims[4] = {kv, rows, 1, 1};
+      const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * rows, (uint64_t)c.ldx * 2 * rows};
+      const uint32_t box[4] = {DSN_GEMM_BK, DSN_GEMM_BM, 1, 1};
+      e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
+    } else {
+      const uint64_t dims[4] = {kv, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)r->B};
+      const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * g.W, (uint64_t)c.ldx * 2 * g.W * g.H};
+      const uint32_t box[4] = {DSN_GEMM_BK, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.nb};
+      e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
+    }
+    if (e) return e;
+    const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)map_n[m]};  // rows beyond k_out: zeros, not fetched
+    const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
+    const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)(g.pair ? g.BN / 2 : g.BN)};
+    e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
+    if (e) return e;
+    const uint64_t yd[2] = {(uint64_t)map_n[m], (uint64_t)r->B * g.R};  // columns clipped at k_out
+    const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
+    const uint32_t yb[2] = {64, 32};
+    e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
+    if (e) return e;
+  }
+  return DSN_OK;
+}
+
+// resident CTA pairs for this n-tile width (0: no pair can be resident, use one CTA per tile)
+int pair_clusters_for(dsn_ctx* ctx, int BN) {
+  if (ctx->gemm_mode != 0) return 0;
+  const int bn_slot = BN == 256 ? 2 : (BN == 128 ? 1 : 0);
+  if (ctx->pair_clusters[bn_slot] < 0) ctx->pair_clusters[bn_slot] = dsn_gemm_pair_max_clusters(227 * 1024);
+  int clusters = ctx->pair_clusters[bn_slot];
+  if (clusters > ctx->sm_count / 2) clusters = ctx->sm_count / 2;
+  return clusters;
+}
+
+int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
+  GemmParams p;
+  fill_gemm_params(ctx, c, r, y, false, p);
+  const GemmGeom& g = p.g;
   // CTA pairs (two SMs per 256-row tile) halve the weight traffic per SM; fall back to one CTA per
   // tile when no pair can be resident
-  const int bn_slot = g.BN == 256 ? 2 : (g.BN == 128 ? 1 : 0);
-  int clusters = 0;
+  const int clusters = pair_clusters_for(ctx, g.BN);
   size_t smem = 0;
-  if (ctx->gemm_mode == 0) {
+  if (clusters > 0) {
     p.g.pair = 1;
     p.g.stages = g.BN == 256 ? 6 : 8;
     while (p.g.stages > 2 && dsn_gemm_pair_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
     smem = dsn_gemm_pair_smem_bytes(g.BN, g.stages, r->G);
-    if (ctx->pair_clusters[bn_slot] < 0) ctx->pair_clusters[bn_slot] = dsn_gemm_pair_max_clusters(227 * 1024);
-    clusters = ctx->pair_clusters[bn_slot];
-    if (clusters > ctx->sm_count / 2) clusters = ctx->sm_count / 2;
-  }
-  if (clusters <= 0) {
+  } else {
     p.g.pair = 0;
     p.g.stages = g.BN == 256 ? 4 : (g.BN == 128 ? 6 : 8);
     while (p.g.stages > 2 && dsn_gemm_smem_bytes(g.BN, p.g.stages, r->G) > 227 * 1024) --p.g.stages;
     smem = dsn_gemm_smem_bytes(g.BN, g.stages, r->G);
   }
-
-  // one tensor-map pair per distinct slice (k_in, k_out), DSN_GEMM_MAX_MAPS pairs per launch
   int done[DSN_MAX_SLICES];
   memset(done, 0, sizeof(done));
   int remaining = c.T;
   while (remaining > 0) {
-    int nmaps = 0;
-    int map_k[DSN_GEMM_MAX_MAPS], map_n[DSN_GEMM_MAX_MAPS];
-    memset(p.map_id, 0xFF, sizeof(p.map_id));
-    for (int t = 0; t < c.T; ++t) {
-      if (done[t]) continue;
-      int id = -1;
-      for (int m = 0; m < nmaps; ++m)
-        if (map_k[m] == c.k_in[t] && map_n[m] == c.k_out[t]) id = m;
-      if (id < 0) {
-        if (nmaps == DSN_GEMM_MAX_MAPS) continue;  // next launch
-        id = nmaps++;
-        map_k[id] = c.k_in[t];
-        map_n[id] = c.k_out[t];
-      }
-      p.map_id[t] = (uint8_t)id;
-      done[t] = 1;
-      --remaining;
-    }
-    for (int m = 0; m < nmaps; ++m) {
-      const uint64_t kv = (uint64_t)map_k[m];
-      int e;
-      if (g.flat) {
-        const uint64_t rows = (uint64_t)r->B * g.R;
-        const uint64_t dims[4] = {kv, rows, 1, 1};
-        const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * rows, (uint64_t)c.ldx * 2 * rows};
-        const uint32_t box[4] = {DSN_GEMM_BK, DSN_GEMM_BM, 1, 1};
-        e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
-      } else {
-        const uint64_t dims[4] = {kv, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)r->B};
-        const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * g.W, (uint64_t)c.ldx * 2 * g.W * g.H};
-        const uint32_t box[4] = {DSN_GEMM_BK, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.nb};
-        e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
-      }
-      if (e) return e;
-      const uint64_t wd[3] = {kv, (uint64_t)g.taps, (uint64_t)map_n[m]};  // rows beyond k_out: zeros, not fetched
-      const uint64_t ws[2] = {(uint64_t)c.w_tap * 2, (uint64_t)c.w_row * 2};
-      const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)(g.pair ? g.BN / 2 : g.BN)};
-      e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
-      if (e) return e;
-      const uint64_t yd[2] = {(uint64_t)map_n[m], (uint64_t)r->B * g.R};  // columns clipped at k_out
-      const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
-      const uint32_t yb[2] = {64, 32};
-      e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
-      if (e) return e;
-    }
+    const int e = fill_gemm_maps(ctx, c, r, x, y, p, done, remaining);
+    if (e) return e;
     if (g.pair) {
       if (dsn_launch_gemm_bf16_pair(p, clusters, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
     } else if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) {
@@ -259,6 +277,54 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     }
   }
   return DSN_OK;
+}
+
+// A chain of bf16 sliced layers whose batch is small enough that every CTA pair owns at most two
+// samples runs as ONE launch (per-sample tiles, intermediates in grouped order): separate launches
+// would each pay their own set-up, ramp and tail for one or two tiles per pair.
+// Returns 1 when the chain was launched, 0 when the caller should run the layers one by one, < 0 on error.
+int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing* r, const void* const* in,
+                  void* const* out, cudaStream_t s) {
+  if (!ctx->chain_mode || ctx->gemm_mode != 0 || n < 2 || n > DSN_CHAIN_MAX_LAYERS) return 0;
+  if (r->group_slice || r->B < 1) return 0;
+  int bn_max = 64;
+  for (int j = 0; j < n; ++j) {
+    const LayerCall& c = calls[j];
+    if (c.att || c.dtype != DSN_BF16 || c.tail != DSN_TAIL_UNTOUCHED) return 0;
+    if (c.H * c.W < 150) return 0;  // a sample must fill most of a 256-row pair tile
+    int distinct = 0, seen_k[DSN_MAX_SLICES], seen_n[DSN_MAX_SLICES];
+    for (int t = 0; t < c.T; ++t) {
+      bool dup = false;
+      for (int u = 0; u < distinct; ++u) dup = dup || (seen_k[u] == c.k_in[t] && seen_n[u] == c.k_out[t]);
+      if (!dup) { seen_k[distinct] = c.k_in[t]; seen_n[distinct] = c.k_out[t]; ++distinct; }
+    }
+    if (distinct > DSN_GEMM_MAX_MAPS) return 0;
+  }
+  DsnChainParams cp;  // about 20 KB of kernel parameters
+  for (int j = 0; j < n; ++j) {
+    fill_gemm_params(ctx, calls[j], r, out[j], true, cp.L[j]);
+    cp.L[j].g.pair = 1;
+    if (cp.L[j].g.BN > bn_max) bn_max = cp.L[j].g.BN;
+  }
+  const int clusters = pair_clusters_for(ctx, bn_max);
+  if (clusters <= 0 || r->B > 2 * clusters) return 0;
+  int stages = bn_max == 256 ? 6 : 8;
+  while (stages > 2 && dsn_gemm_chain_smem_bytes(bn_max, stages, r->G) > 227 * 1024) --stages;
+  for (int j = 0; j < n; ++j) {
+    int done[DSN_MAX_SLICES];
+    memset(done, 0, sizeof(done));
+    int remaining = calls[j].T;
+    cp.L[j].g.stages = stages;
+    const int e = fill_gemm_maps(ctx, calls[j], r, in[j], out[j], cp.L[j], done, remaining);
+    if (e) return e;
+    if (remaining != 0) return 0;
+  }
+  cp.n_layers = n;
+  cp.stages = stages;
+  cp.bn_max = bn_max;
+  if (dsn_launch_gemm_bf16_chain(cp, clusters, dsn_gemm_chain_smem_bytes(bn_max, stages, r->G), s) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  return 1;
 }
 
 int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
@@ -428,6 +494,8 @@ int dsn_create(dsn_ctx** out, int device) {
   {
     const char* m = getenv("DSN_GEMM_MODE");  // "1cta" forces one CTA per tile (for comparisons)
     c->gemm_mode = (m && strcmp(m, "1cta") == 0) ? 1 : 0;
+    const char* ch = getenv("DSN_CHAIN");  // "0": one launch per layer even for small batches (for comparisons)
+    c->chain_mode = (ch && ch[0] == '0') ? 0 : 1;
   }
   cudaDriverEntryPointQueryResult q;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
@@ -723,6 +791,17 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     e = dsn_permute_rows(ctx, &r, c0.dtype, c0.H * c0.W, c0.T, c0.k_in, x, ld_src, ws + pl.off_gather, c0.C_in, 1,
                          stream);
     if (e) return e;
+  }
+  if (!pl.gather_first && L->B > 0) {
+    const void* ins[DSN_MAX_CHAIN];
+    void* outs[DSN_MAX_CHAIN];
+    for (int j = 0; j < L->n_layers; ++j) {
+      ins[j] = j == 0 ? x : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
+      outs[j] = j + 1 == L->n_layers ? y : (void*)(ws + pl.off_buf[j & 1]);
+    }
+    e = try_run_chain(ctx, calls, L->n_layers, &r, ins, outs, s);
+    if (e < 0) return e;
+    if (e == 1) return DSN_OK;
   }
   for (int j = 0; j < L->n_layers; ++j) {
     const bool first = j == 0, last = j + 1 == L->n_layers;

@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
     }
-    if (lane == 0) bulk_wait0();  // this warp's TMA stores are complete before the CTA retires
+    if (elect_one()) bulk_wait0();  // this warp's TMA stores (issued by the elected lane) are complete before the CTA retires
   }
 
   // ------------------------------------------------------------------ teardown

@@ -18,6 +18,7 @@ struct dsn_ctx {
   int32_t* d_status;   // DSN_STATUS_WORDS ints
   void* encode_tiled;  // cuTensorMapEncodeTiled entry point
   int gemm_mode;       // 0 = CTA pairs where possible (default), 1 = one CTA per tile (DSN_GEMM_MODE=1cta)
+  int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
 };
 
@@ -109,7 +110,18 @@ struct GemmParams {
   int32_t* status;
 };
 
+// A chain of up to three sliced layers run by one launch (every layer tiled per sample, CTA pairs).
+#define DSN_CHAIN_MAX_LAYERS 3
+struct DsnChainParams {
+  GemmParams L[DSN_CHAIN_MAX_LAYERS];
+  int32_t n_layers;
+  int32_t stages;   // depth of the operand ring
+  int32_t bn_max;   // widest n-tile of the layers: accumulator stride in TMEM, weight half-box of a ring slot
+};
+
 // launchers implemented in the .cu files
+size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G);
+cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s);
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
 size_t dsn_gemm_smem_bytes(int BN, int stages, int G);
 cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s);

@@ -1,0 +1,63 @@
+"""dsn_layer_forward runs a small-batch chain of sliced layers as one launch (every CTA pair owns
+whole samples and walks the layers itself); larger batches, and every batch with DSN_CHAIN=0 (read
+when a context is created), run one launch per layer.  The parity tests of the chained layers in
+this process use the default; here they run once more in a child process with chaining off, and the
+two modes are compared with each other on one bottleneck."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_layer_forward_parity_with_one_launch_per_layer():
+    env = dict(os.environ, DSN_CHAIN="0")
+    cmd = [sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "-p", "no:cacheprovider",
+           os.path.join(ROOT, "tests", "test_gpu_conv_layer.py"), "-k", "layer_forward"]
+    res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout
+
+
+_CHILD = r"""
+import sys, numpy as np, torch
+sys.path.insert(0, {root!r})
+import paper_2109_10060_b200 as dsn
+import dsn_workloads as wl
+dev = torch.device("cuda:0")
+cfg = wl.config2(B=40)
+B, H, Wd, C, Ci, T, widths = cfg["B"], cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"], cfg["widths"]
+up = lambda a: torch.from_numpy(wl.bf16_bits(np.ascontiguousarray(a)).view(np.int16)).to(dev).view(torch.bfloat16)
+x = up(cfg["x"]); W1 = up(cfg["W1"].reshape(Ci, C)); W2 = up(np.transpose(cfg["W2"], (0, 2, 3, 1))); W3 = up(cfg["W3"].reshape(C, Ci))
+ctx = dsn.Context(0)
+full = [C] * T
+layers = [dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, Ci, full, widths, W1, act=dsn.ACT_RELU),
+          dsn.make_conv_desc(dsn.BF16, H, Wd, 3, 1, Ci, Ci, widths, widths, W2, act=dsn.ACT_RELU),
+          dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, Ci, C, widths, full, W3)]
+L = dsn.make_layer_desc(B, T, layers, None)
+ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=dev)
+y = torch.zeros(B, H, Wd, C, dtype=torch.bfloat16, device=dev)
+idx = torch.from_numpy(cfg["idx"]).to(dev)
+dsn.dsn_layer_forward(ctx, L, x, idx, y, ws)
+code, detail = ctx.get_status()
+assert code == 0, (code, detail)
+np.save(sys.argv[1], y.view(torch.int16).cpu().numpy())
+"""
+
+
+def test_chained_and_unchained_outputs_are_bit_identical(tmp_path):
+    """Both modes run the same tiles' arithmetic (same K order per output element), so the bf16
+    outputs must agree bit for bit."""
+    outs = []
+    for mode in ("1", "0"):
+        path = str(tmp_path / f"y_{mode}.npy")
+        env = dict(os.environ, DSN_CHAIN=mode)
+        res = subprocess.run([sys.executable, "-c", _CHILD.format(root=ROOT), path], cwd=ROOT, env=env,
+                             capture_output=True, text=True, timeout=600)
+        assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-3000:]
+        outs.append(np.load(path))
+    assert np.array_equal(outs[0], outs[1])
