@@ -61,3 +61,57 @@ def test_chained_and_unchained_outputs_are_bit_identical(tmp_path):
         assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-3000:]
         outs.append(np.load(path))
     assert np.array_equal(outs[0], outs[1])
+
+
+# ------------------------------------------------------------------------------------------------
+# Edge cases of the chained launch against the oracle: batch sizes around the limits of the sample
+# hand-out (one sample, an odd count, exactly two per CTA pair, one more than that, which runs one
+# launch per layer), slice widths that are no multiple of 8, every sample on one path, and samples
+# whose index is out of range (they belong to no group; their output rows stay untouched).
+import torch  # noqa: E402
+
+import dsn_workloads as wl  # noqa: E402
+from oracle import dsn_oracle as O  # noqa: E402
+from gpu_util import DEV, SENTINEL, down, group_errors, up_bf16, up_i32  # noqa: E402
+
+
+def _small_bottleneck(dsn, ctx, B, idx, seed=77):
+    cfg = wl.bottleneck(seed, B, 14, 14, 256, 64, routing="uniform", with_gate=False)   # inner widths 22 .. 64
+    H, Wd, C, Ci, T, widths = cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"], cfg["widths"]
+    full = [C] * T
+    W2 = np.ascontiguousarray(np.transpose(cfg["W2"], (0, 2, 3, 1)))
+    layers = [dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, Ci, full, widths, up_bf16(cfg["W1"].reshape(Ci, C)), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 3, 1, Ci, Ci, widths, widths, up_bf16(W2), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, Ci, C, widths, full, up_bf16(cfg["W3"].reshape(C, Ci)))]
+    L = dsn.make_layer_desc(B, T, layers, None)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, H, Wd, C), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_layer_forward(ctx, L, up_bf16(cfg["x"]), up_i32(idx), y, ws)
+    return cfg, down(y)
+
+
+@pytest.mark.parametrize("B,routing", [(1, "uniform"), (2, "uniform"), (75, "uniform"), (148, "uniform"), (149, "uniform"),
+                                       (37, "one_path"), (60, "some_invalid")])
+def test_chained_bottleneck_edge_batches(dsn, B, routing):
+    ctx = dsn.Context(0)
+    T = 14
+    if routing == "one_path":
+        idx = np.full(B, 5, dtype=np.int32)
+    else:
+        idx = wl.idx_quota_uniform(wl.rng(77, 6), B, T)
+    if routing == "some_invalid":
+        idx = idx.copy()
+        idx[::7] = -1
+        idx[3::11] = T
+    cfg, got = _small_bottleneck(dsn, ctx, B, idx)
+    code, detail = ctx.get_status()
+    valid = (idx >= 0) & (idx < T)
+    if routing == "some_invalid":
+        assert code == dsn.ERR_BAD_INDEX and detail == int(np.sum(~valid))   # reported, not fatal
+        assert np.all(got[~valid] == SENTINEL)                                # rows of unrouted samples untouched
+    else:
+        assert code == 0, (code, detail)
+    sel = np.nonzero(valid)[0]
+    _, _, ref = O.bottleneck(cfg["x"][sel], cfg["W1"], cfg["W2"], cfg["W3"], idx[sel], cfg["widths"], mirror_bf16=True)
+    errs = group_errors(got[sel], ref, idx[sel], [cfg["C_outer"]] * T, T)
+    assert max(errs.values()) <= 1e-2, errs
