@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libdsn.so")
-SOURCES = ["dsn_api.cu", "dsn_gate.cu", "dsn_route.cu", "dsn_copy.cu", "dsn_linear_f32.cu", "dsn_gemm_bf16.cu", "dsn_gemm_bf16_2cta.cu", "dsn_gemm_bf16_chain.cu", "dsn_attention.cu", "dsn_depthwise.cu"]
+SOURCES = ["dsn_api.cu", "dsn_gate.cu", "dsn_route.cu", "dsn_copy.cu", "dsn_linear_f32.cu", "dsn_gemm_bf16.cu", "dsn_gemm_bf16_2cta.cu", "dsn_gemm_bf16_chain.cu", "dsn_conv3x3_halo.cu", "dsn_attention.cu", "dsn_depthwise.cu"]
 
 
 def _newest_source_mtime() -> float:

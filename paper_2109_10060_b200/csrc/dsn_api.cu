@@ -117,7 +117,7 @@ void fill_slice_table(SliceTable& st, const LayerCall& c) {
 }
 
 // Tile geometry for the bf16 kernel.  `per_sample`: no tile spans two samples (chained layers).
-void choose_geometry(const LayerCall& c, GemmGeom& g, bool per_sample = false) {
+void choose_geometry(const LayerCall& c, GemmGeom& g, bool per_sample = false, bool halo = false) {
   memset(&g, 0, sizeof(g));
   g.H = c.H;
   g.W = c.W;
@@ -135,6 +135,18 @@ void choose_geometry(const LayerCall& c, GemmGeom& g, bool per_sample = false) {
     g.flat = 1;  // grouped rows are contiguous: tile them without regard to sample boundaries
     g.bw = DSN_GEMM_BM;
     g.bh = g.nb = g.tiles_x = g.tiles_y = 1;
+    return;
+  }
+  if (halo) {  // 3x3: M rows run over the padded width, whole image rows per tile
+    g.halo = 1;
+    g.bw = g.W + 2;
+    g.bh = DSN_GEMM_BM / g.bw;
+    if (g.bh > g.H) g.bh = g.H;
+    const int bands = (g.H + g.bh - 1) / g.bh;
+    g.bh = (g.H + bands - 1) / bands;
+    g.nb = 1;
+    g.tiles_x = 1;
+    g.tiles_y = bands;
     return;
   }
   if (c.K == 1) {  // input order: a sample's R rows form one "image" of height 1
@@ -158,9 +170,10 @@ void choose_geometry(const LayerCall& c, GemmGeom& g, bool per_sample = false) {
 }
 
 // Everything of the kernel parameters except the tensor maps.
-void fill_gemm_params(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, void* y, bool per_sample, GemmParams& p) {
+void fill_gemm_params(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, void* y, bool per_sample, GemmParams& p,
+                      bool halo = false) {
   memset(&p, 0, sizeof(p));
-  choose_geometry(c, p.g, per_sample);
+  choose_geometry(c, p.g, per_sample, halo);
   p.B = r->B;
   p.G = r->G;
   p.T = c.T;
@@ -217,7 +230,7 @@ int fill_gemm_maps(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const
     } else {
       const uint64_t dims[4] = {kv, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)r->B};
       const uint64_t str[3] = {(uint64_t)c.ldx * 2, (uint64_t)c.ldx * 2 * g.W, (uint64_t)c.ldx * 2 * g.W * g.H};
-      const uint32_t box[4] = {DSN_GEMM_BK, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.nb};
+      const uint32_t box[4] = {DSN_GEMM_BK, (uint32_t)g.bw, (uint32_t)(g.bh + (g.halo ? 2 : 0)), (uint32_t)g.nb};
       e = encode_map(ctx, &p.mapA[m], x, 4, dims, str, box);
     }
     if (e) return e;
@@ -247,8 +260,40 @@ int pair_clusters_for(dsn_ctx* ctx, int BN) {
 
 int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
   GemmParams p;
-  fill_gemm_params(ctx, c, r, y, false, p);
+  // 3x3 layers with slices up to 128 wide on images of at least 12 pixels a side stage the input tile once,
+  // with its halo; smaller images (7x7) keep one load per tap, which packs two whole images into a tile
+  bool halo = ctx->conv_halo && ctx->gemm_mode == 0 && c.K == 3 && c.pad == 1 && c.W >= 12 && c.W + 2 <= DSN_GEMM_BM;
+  if (halo) {  // measured: a gain for n-tiles up to 128 wide (1.2-1.5x), none for 256-wide ones (tensor bound either way)
+    int max_ko = 1;
+    for (int t = 0; t < c.T; ++t) max_ko = c.k_out[t] > max_ko ? c.k_out[t] : max_ko;
+    halo = max_ko <= 128;
+  }
+  fill_gemm_params(ctx, c, r, y, false, p, halo);
   const GemmGeom& g = p.g;
+  if (halo) {
+    const int clusters_h = pair_clusters_for(ctx, g.BN);
+    if (clusters_h > 0) {
+      p.g.pair = 1;
+      // weight ring: a slot per tap for 256-wide n-tiles (6 slots of 16 KB), otherwise a slot holds all nine
+      // taps of a chunk (3 slots of 36 KB, 2 of 72 KB); the rest goes to activation blocks
+      p.g.tps = g.BN == 256 ? 1 : 9;
+      p.g.stages = g.BN == 256 ? 6 : (g.BN == 128 ? 2 : 3);
+      p.g.a_slots = g.BN == 256 ? 2 : 4;
+      while (p.g.a_slots > 2 && dsn_gemm_halo_smem_bytes(g.BN, g.stages, p.g.a_slots, r->G, g.bw, g.bh) > 227 * 1024) --p.g.a_slots;
+      while (p.g.stages > 2 && dsn_gemm_halo_smem_bytes(g.BN, p.g.stages, g.a_slots, r->G, g.bw, g.bh) > 227 * 1024) --p.g.stages;
+      const size_t smem_h = dsn_gemm_halo_smem_bytes(g.BN, g.stages, g.a_slots, r->G, g.bw, g.bh);
+      int done_h[DSN_MAX_SLICES];
+      memset(done_h, 0, sizeof(done_h));
+      int remaining_h = c.T;
+      while (remaining_h > 0) {
+        const int e = fill_gemm_maps(ctx, c, r, x, y, p, done_h, remaining_h);
+        if (e) return e;
+        if (dsn_launch_gemm_bf16_halo(p, clusters_h, smem_h, s) != cudaSuccess) return DSN_ERR_CUDA;
+      }
+      return DSN_OK;
+    }
+    fill_gemm_params(ctx, c, r, y, false, p, false);  // no pair can be resident: the one-CTA kernel, one load per tap
+  }
   // CTA pairs (two SMs per 256-row tile) halve the weight traffic per SM; fall back to one CTA per
   // tile when no pair can be resident
   const int clusters = pair_clusters_for(ctx, g.BN);
@@ -494,6 +539,8 @@ int dsn_create(dsn_ctx** out, int device) {
   {
     const char* m = getenv("DSN_GEMM_MODE");  // "1cta" forces one CTA per tile (for comparisons)
     c->gemm_mode = (m && strcmp(m, "1cta") == 0) ? 1 : 0;
+    const char* cv = getenv("DSN_CONV3X3");  // "taps": 3x3 layers load the tile once per tap (for comparisons)
+    c->conv_halo = (cv && strcmp(cv, "taps") == 0) ? 0 : 1;
     const char* ch = getenv("DSN_CHAIN");  // "0": one launch per layer even for small batches (for comparisons)
     c->chain_mode = (ch && ch[0] == '0') ? 0 : 1;
   }

@@ -1,0 +1,321 @@
+// 3x3 sliced convolution (stride 1, zero padding 1) on CTA pairs with the input tile staged ONCE.
+//
+// The tap-shifted form of the pair GEMM loads the activation tile nine times per 64-channel chunk
+// (one TMA box per tap).  Here one TMA box per chunk brings the tile WITH its one-pixel halo
+// ((bh + 2) image rows x (W + 2) pixels, out-of-image pixels zero-filled = the padding) into shared
+// memory, and the nine taps are nine views of that block: row m of the MMA's A operand for tap
+// (r, s) is halo pixel m + r (W + 2) + s, i.e. the same 128-byte rows read through a descriptor whose
+// start address is moved by (r (W + 2) + s) x 128 bytes.  The 128-byte swizzle is a function of the
+// shared-memory address bits for TMA and MMA alike, so a view that starts at any 128-byte row of a
+// 1024-byte-aligned block reads the layout TMA wrote; the descriptor's base-offset field stays 0
+// (checked on the device: with the row phase in that field the sums come out wrong).
+// M rows are numbered over the padded width: m = j (W + 2) + x; the two rows per image row with
+// x >= W compute nothing that is stored.  Weights stream through a ring of (tap, chunk) boxes as
+// before; the activation blocks have a ring of their own (2 to 6 slots, as many as fit).
+//
+// Same contract, roles, accumulators and epilogue as dsn_gemm_bf16_2cta.cu.  Added barriers:
+//   afull[a]   even CTA only: the activation boxes of both CTAs have landed
+//   aempty[a]  both CTAs: the MMAs of all nine taps that read the slot are done (multicast commit)
+#include <cuda_runtime.h>
+
+#include "dsn_gemm_pair_device.cuh"
+
+namespace {
+
+using namespace dsn_gemm;
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const GemmGeom& g = p.g;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+
+  const uint32_t bar_full = base;
+  const uint32_t bar_empty = base + 8 * kMaxStages;
+  const uint32_t bar_tfull = base + 16 * kMaxStages + 48 + 16 * kMaxStages;  // [8]
+  const uint32_t bar_tempty = bar_tfull + 64;                                // [8]
+  // accumulators: as many n-tile-wide buffers as TMEM's 512 columns hold (2, 4 or 8).  With narrow
+  // slices the main loop and the epilogue of a tile are both short, and what a tile costs is the
+  // hand-over between them; more buffers keep more tiles in flight.
+  const int acc_log2 = g.BN == 256 ? 1 : (g.BN == 128 ? 2 : 3);
+  const int nacc = 1 << acc_log2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16 * kMaxStages + 32);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxStages + 36);
+
+  const uint32_t bar_afull = base + 16 * kMaxStages + 48;   // [kMaxStages]
+  const uint32_t bar_aempty = bar_afull + 8 * kMaxStages;  // [kMaxStages]
+  const int aslots = g.a_slots;                            // depth of the activation ring
+  const int stages = g.stages;                             // depth of the weight ring
+  const uint32_t bh_bytes = (uint32_t)(g.BN / 2) * BK * 2;  // this CTA's half of the weight tile of one tap
+  // Narrow n-tiles put all nine taps of a chunk into ONE ring slot (one wait and one commit per 36
+  // instructions: with N <= 128 an instruction is too short to hide a barrier round per tap); the
+  // 16 KB boxes of 256-wide tiles keep a slot per tap.
+  const int tps = g.tps;                                    // taps per ring slot: 9 or 1
+  const uint32_t slot_b = (uint32_t)tps * bh_bytes;
+  const uint32_t a_slot = dsn_halo_slot_bytes(g.bw, g.bh);  // one activation block with halo (+ overrun rows)
+  const uint32_t a_base = base + kCtrlBytes;
+  const uint32_t b_base = a_base + (uint32_t)aslots * a_slot;
+  uint8_t* out_stage = smem + kCtrlBytes + (size_t)aslots * a_slot + (size_t)stages * slot_b;
+  int32_t* s_prefix = reinterpret_cast<int32_t*>(out_stage + kStageOutBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const uint32_t tmem_cols = 512u;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < nacc; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, 2 * kEpiWarps);
+    }
+    for (int a = 0; a < aslots; ++a) {
+      mbar_init(bar_afull + 8 * a, 1);
+      mbar_init(bar_aempty + 8 * a, 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), tmem_cols);
+    tmem_relinquish_pair();
+  }
+
+  auto ntiles_of = [&](int grp) {
+    const int sl = p.group_slice ? p.group_slice[grp] : grp;
+    if (sl < 0 || sl >= p.T || p.map_id[sl] == 0xFF) return 0;
+    const int cnt = p.offsets[grp + 1] - p.offsets[grp];
+    if (cnt <= 0) return 0;
+    const int mt = g.flat ? (cnt * g.R + BM - 1) / BM : ((cnt + g.nb - 1) / g.nb) * g.tiles_x * g.tiles_y;
+    return ((mt + 1) / 2) * ((p.k_out[sl] + g.BN - 1) / g.BN);
+  };
+  // barriers and TMEM are set up; everything below reads what earlier kernels wrote
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
+  // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group
+  for (int j = threadIdx.x; j <= p.G; j += blockDim.x) s_prefix[p.G + 1 + j] = p.offsets[j];
+  for (int j = threadIdx.x; j < p.G; j += blockDim.x) {
+    const int sl = p.group_slice ? p.group_slice[j] : j;
+    s_prefix[2 * p.G + 2 + j] = (sl >= 0 && sl < p.T) ? sl : 0;
+  }
+  dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything can arrive on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = s_prefix[p.G];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    // The whole warp walks the schedule (addresses, coordinates and the loop itself stay
+    // warp-uniform, which keeps the per-stage instruction count low); one elected lane issues.
+    int stage = 0, aslot = 0;
+    uint32_t phase = 0, aphase = 0;
+    const uint32_t a_box_bytes = (uint32_t)(g.bw * (g.bh + 2)) * BK * 2;  // (W + 2) x (bh + 2) pixels
+    bool ok = true;
+    for (int tile = pair; ok && tile < total; tile += npairs) {
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const CUtensorMap* mA = &p.mapA[t.map];
+      const CUtensorMap* mB = &p.mapB[t.map];
+      const int nkc = (t.ki + BK - 1) / BK;
+      int ncols = t.ko - t.n0;
+      ncols = ncols > g.BN ? g.BN : ncols;
+      const int n_inst = (ncols + 31) & ~31;
+      const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
+      int bsel = t.b0;
+      if (g.a_input_order) bsel = t.b0 < t.p_end ? p.perm[t.b0] : p.B;  // past the group: out of range, zeros
+      for (int kc = 0; ok && kc < nkc; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * aslot, aphase ^ 1u, abort_flag, p.status, 41));
+        if (!ok) break;
+        if (elect_one()) {
+          const uint32_t lead = leader_addr(bar_afull + 8 * aslot);
+          if (rank == 0) mbar_expect_tx(bar_afull + 8 * aslot, 2u * a_box_bytes);
+          tma_load_4d_pair(a_base + aslot * a_slot, mA, kc * BK, -1, t.y0 - 1, bsel, lead);  // halo: starts one pixel out
+        }
+        if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
+        for (int tap0 = 0; tap0 < 9; tap0 += tps) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 42));
+          if (!ok) break;
+          if (elect_one()) {
+            const uint32_t lead = leader_addr(bar_full + 8 * stage);
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * slot_b);
+            for (int u = 0; u < tps; ++u)
+              tma_load_3d_pair(b_base + stage * slot_b + u * bh_bytes, mB, kc * BK, tap0 + u, brow0, lead);
+          }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA only)
+    // Warp-uniform loop, one elected lane issues.  The issuing warp is the critical resource of a tile with
+    // wide N (four instructions of 128 tensor-pipe cycles per stage), so the per-stage path is
+    // kept short: running descriptors, four unrolled K steps, a separate short loop for a partial
+    // last chunk.
+    if (rank == 0) {
+      int stage = 0, aslot = 0;
+      uint32_t phase = 0, aphase = 0;
+      int it = 0;
+      bool ok = true;
+      const uint64_t db0 = make_smem_desc(b_base);
+      const uint64_t dbstep = (uint64_t)(slot_b >> 4), dbtap = (uint64_t)(bh_bytes >> 4);
+      const uint64_t darow = (uint64_t)(g.bw * 8);  // one image row of the padded block, in 16-byte units
+      uint64_t db = db0;
+      for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
+        const PairTile t = decode_pair_tile(p, s_prefix, tile, 0);
+        const int acc = it & (nacc - 1);
+        const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
+        if (!ok) break;
+        tc_fence_after();
+        int ncols = t.ko - t.n0;
+        ncols = ncols > g.BN ? g.BN : ncols;
+        const int n_inst = (ncols + 31) & ~31;
+        const uint32_t idesc = make_idesc(2 * BM, n_inst);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
+        const int nkc = (t.ki + BK - 1) / BK;
+        const int tail_ks = ((t.ki & (BK - 1)) + 15) >> 4;  // K steps of a partial last chunk (0: none)
+        uint32_t accumulate = 0;
+        for (int kc = nkc; ok && kc > 0; --kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * aslot, aphase, abort_flag, p.status, 43));
+          if (!ok) break;
+          const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
+          const uint32_t a_addr = a_base + aslot * a_slot;
+          const uint64_t da0 = make_smem_desc(a_addr);
+          for (int tap0 = 0; tap0 < 9; tap0 += tps) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13));
+            if (!ok) break;
+            tc_fence_after();
+            // a tap's view of the block: same rows, start moved by whole 128-byte rows (8 descriptor units each)
+            if (tps == 9) {
+              if (elect_one()) {
+#pragma unroll
+                for (int u = 0; u < 9; ++u) {
+                  const uint64_t da = da0 + (uint64_t)(u / 3) * darow + (uint64_t)(8 * (u % 3)), dbt = db + (uint64_t)u * dbtap;
+                  umma_bf16_pair(d_tmem, da, dbt, idesc, u == 0 ? accumulate : 1u);  // +32 bytes per K step
+                  if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, dbt + 2u, idesc, 1u);
+                  if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, dbt + 4u, idesc, 1u);
+                  if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, dbt + 6u, idesc, 1u);
+                }
+                umma_commit_pair(bar_empty + 8 * stage);
+              }
+            } else {
+              const int r = tap0 / 3, sx = tap0 - 3 * r;
+              const uint64_t da = da0 + (uint64_t)r * darow + (uint64_t)(8 * sx);
+              if (elect_one()) {
+                umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, db + 2u, idesc, 1u);
+                if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, db + 4u, idesc, 1u);
+                if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, db + 6u, idesc, 1u);
+                umma_commit_pair(bar_empty + 8 * stage);
+              }
+            }
+            accumulate = 1;
+            db += dbstep;
+            if (++stage == stages) { stage = 0; phase ^= 1u; db = db0; }
+          }
+          if (ok && elect_one()) umma_commit_pair(bar_aempty + 8 * aslot);  // all nine taps have read the block
+          if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
+        }
+        if (ok && elect_one()) umma_commit_pair(bar_tfull + 8 * acc);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int q = warp & 3;
+    const int first = (warp - 2) >> 2;
+    const int m = q * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    const int box_rows = g.bw * g.bh * g.nb, img_rows = g.bw * g.bh;
+    for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const int acc = it & (nacc - 1);
+      const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
+
+      bool valid;
+      int64_t out_row;
+      if (g.flat) {
+        const int gr = t.row0 + m;
+        valid = gr < t.rows_end;
+        out_row = gr;
+        if (valid && g.y_input_order) {
+          const int pp = gr / g.R;
+          out_row = (int64_t)p.perm[pp] * g.R + (gr - pp * g.R);
+        }
+      } else {
+        const int bi = m / img_rows, rem = m - bi * img_rows;
+        const int yy = t.y0 + rem / g.bw, xx = t.x0 + rem % g.bw;
+        const int pp = t.b0 + bi;
+        valid = m < box_rows && yy < g.H && xx < g.W && pp < t.p_end;
+        out_row = 0;
+        if (valid) {
+          const int smp = g.y_input_order ? p.perm[pp] : pp;
+          out_row = (int64_t)smp * g.R + yy * g.W + xx;
+        }
+      }
+      __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
+      const float* brow = p.bias ? p.bias + t.n0 : nullptr;
+      const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      const __nv_bfloat16* res_row = (p.residual && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
+      int ncols = t.ko - t.n0;
+      ncols = ncols > g.BN ? g.BN : ncols;
+      const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
+      uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
+      const CUtensorMap* mY = &p.mapY[t.map];
+      const int variant = p.act * 2 + ((brow || sc_row || p.residual) ? 1 : 0);
+      switch (variant) {
+        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it
+    }
+    if (elect_one()) bulk_wait0();  // the lane that issued this warp's TMA stores
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA retires while its partner may still read its memory or signal its barriers
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, tmem_cols);
+  }
+}
+
+}  // namespace
+
+size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int a_slots, int G, int wp, int bh) {
+  const int tps = BN == 256 ? 1 : 9;  // taps per ring slot
+  return 1024 + kCtrlBytes + (size_t)a_slots * dsn_halo_slot_bytes(wp, bh) + (size_t)stages * tps * ((size_t)(BN / 2) * BK * 2) +
+         kStageOutBytes + sizeof(int32_t) * (3 * (size_t)G + 3);
+}
+
+cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
+  static size_t configured = 0;
+  if (smem_bytes > configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) return e;
+    configured = smem_bytes;
+  }
+  return dsn_launch(gemm_bf16_halo_kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
+}

@@ -23,47 +23,6 @@ namespace {
 
 using namespace dsn_gemm;
 
-struct PairTile {
-  int map, ki, ko, n0, slice;
-  int p_end;
-  int row0, rows_end;
-  int b0, x0, y0;
-};
-
-// Tile `tile` of the pair schedule as seen by CTA `rank`: the pair owns m-tiles 2*mtp and 2*mtp+1 of
-// one (group, n-tile); an m-tile past the group's last one yields only invalid rows.
-__device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const int32_t* s_prefix, int tile, int rank) {
-  PairTile t;
-  const GemmGeom& g = p.g;
-  const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
-  const int grp = p.G - 1 - j;
-  const int sl = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
-  t.slice = sl;
-  t.map = p.map_id[sl];
-  t.ki = p.k_in[sl];
-  t.ko = p.k_out[sl];
-  const int p0 = s_prefix[p.G + 1 + grp];      // group offsets, cached in shared memory
-  t.p_end = s_prefix[p.G + 2 + grp];
-  const int ntn = (t.ko + g.BN - 1) / g.BN;
-  const int local = tile - s_prefix[j];
-  const int nt = local % ntn, mt = 2 * (local / ntn) + rank;
-  t.n0 = nt * g.BN;
-  if (g.flat) {
-    t.row0 = p0 * g.R + mt * BM;
-    t.rows_end = t.p_end * g.R;
-    t.b0 = t.x0 = t.y0 = 0;
-  } else {
-    const int per_img = g.tiles_x * g.tiles_y;
-    const int ib = mt / per_img, rem = mt - ib * per_img;
-    const int ty = rem / g.tiles_x, tx = rem - ty * g.tiles_x;
-    t.b0 = p0 + ib * g.nb;
-    t.y0 = ty * g.bh;
-    t.x0 = tx * g.bw;
-    t.row0 = t.rows_end = 0;
-  }
-  return t;
-}
-
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const GemmGeom& g = p.g;

@@ -18,6 +18,7 @@ struct dsn_ctx {
   int32_t* d_status;   // DSN_STATUS_WORDS ints
   void* encode_tiled;  // cuTensorMapEncodeTiled entry point
   int gemm_mode;       // 0 = CTA pairs where possible (default), 1 = one CTA per tile (DSN_GEMM_MODE=1cta)
+  int conv_halo;       // 1 = 3x3 layers stage the input tile once with its halo (default), 0 = one load per tap (DSN_CONV3X3=taps)
   int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
 };
@@ -85,7 +86,19 @@ struct GemmGeom {
   int32_t BN;              // n-tile (64, 128, 256) = rows of the weight box
   int32_t stages;
   int32_t pair;            // 1: tiles are owned by CTA pairs (256 rows), weight box holds BN/2 rows
+  int32_t a_slots;         // halo form: depth of the activation ring
+  int32_t tps;             // halo form: taps per weight-ring slot (9: all taps of a chunk in one slot, 1: a slot per tap)
+  int32_t halo;            // 1: 3x3 layer with the input tile staged once with its halo: bw = W + 2 is the M-row
+                           //    pitch, the activation box holds (W + 2) x (bh + 2) pixels, taps are descriptor shifts
 };
+
+// Shared-memory bytes of one activation block of the halo form: the box itself, and at least the rows
+// the last tap's view of 128 M rows reaches (128 + 2 (W + 2) + 2), rounded to the swizzle period.
+__host__ __device__ inline uint32_t dsn_halo_slot_bytes(int wp, int bh) {
+  const int box = wp * (bh + 2), reach = 128 + 2 * wp + 2;
+  const uint32_t rows = (uint32_t)(box > reach ? box : reach);
+  return (rows * 128u + 1023u) & ~1023u;
+}
 
 struct GemmParams {
   CUtensorMap mapA[DSN_GEMM_MAX_MAPS];
@@ -122,6 +135,8 @@ struct DsnChainParams {
 // launchers implemented in the .cu files
 size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G);
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s);
+size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int a_slots, int G, int wp, int bh);
+cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s);
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
 size_t dsn_gemm_smem_bytes(int BN, int stages, int G);
 cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s);
