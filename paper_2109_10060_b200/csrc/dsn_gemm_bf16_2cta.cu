@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = s_prefix[p.G];
+  PairCursor cursor;  // every role walks its own tile sequence
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
     const uint32_t tx_bytes = 2u * (a_box_bytes + bh_bytes);
     bool ok = true;
     for (int tile = pair; ok && tile < total; tile += npairs) {
-      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank, cursor);
       const CUtensorMap* mA = &p.mapA[t.map];
       const CUtensorMap* mB = &p.mapB[t.map];
       const int nkc = (t.ki + BK - 1) / BK;
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
       const uint64_t dstep = (uint64_t)(stage_bytes >> 4);
       uint64_t da = da0, db = db0;
       for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
-        const PairTile t = decode_pair_tile(p, s_prefix, tile, 0);
+        const PairTile t = decode_pair_tile(p, s_prefix, tile, 0, cursor);
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
@@ -187,8 +188,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
     int it = 0;
     bool ok = true;
     const int box_rows = g.bw * g.bh * g.nb, img_rows = g.bw * g.bh;
+    // this thread's place in a per-image tile does not change from tile to tile
+    const int row_bi = g.flat ? 0 : m / img_rows, row_rem = g.flat ? 0 : m - row_bi * img_rows;
+    const int row_j = g.flat ? 0 : row_rem / g.bw, row_x = g.flat ? 0 : row_rem - row_j * g.bw;
     for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
-      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank);
+      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank, cursor);
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
 
@@ -203,9 +207,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
           out_row = (int64_t)p.perm[pp] * g.R + (gr - pp * g.R);
         }
       } else {
-        const int bi = m / img_rows, rem = m - bi * img_rows;
-        const int yy = t.y0 + rem / g.bw, xx = t.x0 + rem % g.bw;
-        const int pp = t.b0 + bi;
+        const int yy = t.y0 + row_j, xx = t.x0 + row_x;
+        const int pp = t.b0 + row_bi;
         valid = m < box_rows && yy < g.H && xx < g.W && pp < t.p_end;
         out_row = 0;
         if (valid) {

@@ -74,33 +74,62 @@ struct PairTile {
   int b0, x0, y0;
 };
 
+// What a role remembers between two tiles: tiles come in increasing order, so the group found for one
+// tile usually still holds for the next and its data need not be looked up again.
+struct PairCursor {
+  int lo = 0, hi = 0;   // tiles [lo, hi) belong to the cached group (hi = 0: nothing cached)
+  int slice, map, ki, ko, p0, p_end, ntn;
+};
+
 // Tile `tile` of the pair schedule as seen by CTA `rank`: the pair owns m-tiles 2*mtp and 2*mtp+1 of
 // one (group, n-tile); an m-tile past the group's last one yields only invalid rows.
-__device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const int32_t* s_prefix, int tile, int rank) {
+__device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const int32_t* s_prefix, int tile, int rank,
+                                                     PairCursor& c) {
   PairTile t;
   const GemmGeom& g = p.g;
-  const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
-  const int grp = p.G - 1 - j;
-  const int sl = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
-  t.slice = sl;
-  t.map = p.map_id[sl];
-  t.ki = p.k_in[sl];
-  t.ko = p.k_out[sl];
-  const int p0 = s_prefix[p.G + 1 + grp];      // group offsets, cached in shared memory
-  t.p_end = s_prefix[p.G + 2 + grp];
-  const int ntn = (t.ko + g.BN - 1) / g.BN;
-  const int local = tile - s_prefix[j];
-  const int nt = local % ntn, mt = 2 * (local / ntn) + rank;
+  if (tile >= c.hi) {
+    const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
+    const int grp = p.G - 1 - j;
+    c.lo = s_prefix[j];
+    c.hi = s_prefix[j + 1];
+    c.slice = s_prefix[2 * p.G + 2 + grp];  // group -> slice, cached in shared memory
+    c.map = p.map_id[c.slice];
+    c.ki = p.k_in[c.slice];
+    c.ko = p.k_out[c.slice];
+    c.p0 = s_prefix[p.G + 1 + grp];         // group offsets, cached in shared memory
+    c.p_end = s_prefix[p.G + 2 + grp];
+    c.ntn = (c.ko + g.BN - 1) / g.BN;
+  }
+  t.slice = c.slice;
+  t.map = c.map;
+  t.ki = c.ki;
+  t.ko = c.ko;
+  t.p_end = c.p_end;
+  const int local = tile - c.lo;
+  int nt = 0, mtp = local;
+  if (c.ntn > 1) {
+    mtp = local / c.ntn;
+    nt = local - mtp * c.ntn;
+  }
+  const int mt = 2 * mtp + rank;
   t.n0 = nt * g.BN;
   if (g.flat) {
-    t.row0 = p0 * g.R + mt * BM;
-    t.rows_end = t.p_end * g.R;
+    t.row0 = c.p0 * g.R + mt * BM;
+    t.rows_end = c.p_end * g.R;
     t.b0 = t.x0 = t.y0 = 0;
   } else {
     const int per_img = g.tiles_x * g.tiles_y;
-    const int ib = mt / per_img, rem = mt - ib * per_img;
-    const int ty = rem / g.tiles_x, tx = rem - ty * g.tiles_x;
-    t.b0 = p0 + ib * g.nb;
+    int ib = 0, rem = mt;
+    if (mt >= per_img) {
+      ib = mt / per_img;
+      rem = mt - ib * per_img;
+    }
+    int ty = rem, tx = 0;
+    if (g.tiles_x > 1) {
+      ty = rem / g.tiles_x;
+      tx = rem - ty * g.tiles_x;
+    }
+    t.b0 = c.p0 + ib * g.nb;
     t.y0 = ty * g.bh;
     t.x0 = tx * g.bw;
     t.row0 = t.rows_end = 0;
