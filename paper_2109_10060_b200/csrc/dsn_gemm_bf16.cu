@@ -14,8 +14,8 @@
 // fetched from L2 and never multiplied.
 //
 // Structure of a CTA (persistent, one per SM, 320 threads):
-//   warp 0      one lane issues the TMA loads into a ring of shared-memory stages
-//   warp 1      one lane issues tcgen05.mma (M = 128, N = 16..256, K = 16) into a TMEM accumulator;
+//   warp 0      walks the tile schedule (warp-uniform loop), one elected lane issues the TMA loads into a ring of stages
+//   warp 1      same form, one elected lane issues tcgen05.mma (M = 128, N = 16..256, K = 16) into a TMEM accumulator;
 //               two accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
 //   warps 2..9  epilogue, two warps per TMEM lane quarter taking alternate 64-column chunks:
 //               tcgen05.ld (one accumulator row per thread), bias / activation, bf16 rounding into a
@@ -140,78 +140,87 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x) {
-        const TileInfo t = decode_tile(p, s_prefix, tile);
-        const CUtensorMap* mA = &p.mapA[t.map];
-        const CUtensorMap* mB = &p.mapB[t.map];
-        const int nkc = (t.ki + BK - 1) / BK;
-        int bsel = t.b0;
-        if (g.a_input_order) bsel = p.perm[t.b0];
-        for (int tap = 0; ok && tap < g.taps; ++tap) {
-          const int r = tap / g.KW, s = tap - r * g.KW;
-          for (int kc = 0; kc < nkc; ++kc) {
-            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+    // The whole warp walks the schedule (warp-uniform loop), one elected lane issues the copies.
+    int stage = 0;
+    uint32_t phase = 0;
+    const uint32_t a_box_bytes = g.flat ? kABytes : (uint32_t)(g.bw * g.bh * g.nb) * BK * 2;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x) {
+      const TileInfo t = decode_tile(p, s_prefix, tile);
+      const CUtensorMap* mA = &p.mapA[t.map];
+      const CUtensorMap* mB = &p.mapB[t.map];
+      const int nkc = (t.ki + BK - 1) / BK;
+      int bsel = t.b0;
+      if (g.a_input_order) bsel = p.perm[t.b0];
+      for (int tap = 0; ok && tap < g.taps; ++tap) {
+        const int r = tap / g.KW, sx = tap - r * g.KW;
+        const int cx = g.flat ? t.row0 : t.x0 + sx - g.pad, cy = g.flat ? 0 : t.y0 + r - g.pad, cb = g.flat ? 0 : bsel;
+        for (int kc = 0; kc < nkc; ++kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 1));
+          if (!ok) break;
+          if (elect_one()) {
             const uint32_t full = bar_full + 8 * stage;
             mbar_expect_tx(full, a_box_bytes + b_bytes);
             const uint32_t sa = tiles_base + stage * stage_bytes;
-            if (g.flat) tma_load_4d(sa, mA, kc * BK, t.row0, 0, 0, full);
-            else tma_load_4d(sa, mA, kc * BK, t.x0 + s - g.pad, t.y0 + r - g.pad, bsel, full);
+            tma_load_4d(sa, mA, kc * BK, cx, cy, cb, full);
             tma_load_3d(sa + kABytes, mB, kc * BK, tap, t.n0, full);
-            if (++stage == stages) { stage = 0; phase ^= 1u; }
           }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
-        // let copies already issued land before the CTA gives up its shared memory
-        for (int s = 0; s < stages; ++s) {
-          const uint64_t t0 = globaltimer_ns();
-          const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-          while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < 1000000ull) {}
-        }
+    }
+    if (!ok && lane == 0) {
+      // let copies already issued land before the CTA gives up its shared memory
+      for (int s = 0; s < stages; ++s) {
+        const uint64_t t0 = globaltimer_ns();
+        const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+        while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < 1000000ull) {}
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
-        const TileInfo t = decode_tile(p, s_prefix, tile);
-        const int acc = it & 1;
-        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-        if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
-        tc_fence_after();
-        int n_inst = t.ko - t.n0;
-        n_inst = n_inst > g.BN ? g.BN : ((n_inst + 15) & ~15);
-        const uint32_t idesc = make_idesc(BM, n_inst);
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
-        const int nkc = (t.ki + BK - 1) / BK;
-        uint32_t accumulate = 0;
-        for (int tap = 0; ok && tap < g.taps; ++tap) {
-          for (int kc = 0; kc < nkc; ++kc) {
-            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 3)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t sa = tiles_base + stage * stage_bytes;
-            const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kABytes);
-            const int krem = t.ki - kc * BK;
-            const int nks = krem >= BK ? BK / 16 : (krem + 15) >> 4;
-            for (int ks = 0; ks < nks; ++ks) {
-              umma_bf16(d_tmem, da + 2u * ks, db + 2u * ks, idesc, accumulate);  // +32 bytes per K step
-              accumulate = 1;
-            }
+    // Warp-uniform loop, one elected lane issues: running descriptors, four unrolled K steps.
+    int stage = 0;
+    uint32_t phase = 0;
+    int it = 0;
+    bool ok = true;
+    const uint64_t da0 = make_smem_desc(tiles_base), db0 = make_smem_desc(tiles_base + kABytes);
+    const uint64_t dstep = (uint64_t)(stage_bytes >> 4);
+    uint64_t da = da0, db = db0;
+    for (int tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
+      const TileInfo t = decode_tile(p, s_prefix, tile);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 2));
+      if (!ok) break;
+      tc_fence_after();
+      int n_inst = t.ko - t.n0;
+      n_inst = n_inst > g.BN ? g.BN : ((n_inst + 15) & ~15);
+      const uint32_t idesc = make_idesc(BM, n_inst);
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
+      const int nkc = (t.ki + BK - 1) / BK;
+      const int tail_ks = ((t.ki & (BK - 1)) + 15) >> 4;  // K steps of a partial last chunk (0: none)
+      uint32_t accumulate = 0;
+      for (int tap = 0; ok && tap < g.taps; ++tap) {
+        for (int kc = nkc; kc > 0; --kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 3));
+          if (!ok) break;
+          tc_fence_after();
+          const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
+          if (elect_one()) {
+            umma_bf16(d_tmem, da, db, idesc, accumulate);  // +32 bytes per K step
+            if (nks > 1) umma_bf16(d_tmem, da + 2u, db + 2u, idesc, 1u);
+            if (nks > 2) umma_bf16(d_tmem, da + 4u, db + 4u, idesc, 1u);
+            if (nks > 3) umma_bf16(d_tmem, da + 6u, db + 6u, idesc, 1u);
             umma_commit(bar_empty + 8 * stage);
-            if (++stage == stages) { stage = 0; phase ^= 1u; }
           }
+          accumulate = 1;
+          da += dstep;
+          db += dstep;
+          if (++stage == stages) { stage = 0; phase ^= 1u; da = da0; db = db0; }
         }
-        if (ok) umma_commit(bar_tfull + 8 * acc);
       }
+      if (ok && elect_one()) umma_commit(bar_tfull + 8 * acc);
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9)
