@@ -30,6 +30,7 @@ if ROOT not in sys.path:
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
+CHAIN_CFG2_DRAM_BYTES = 68.4e6   # per launch of gemm_bf16_chain_kernel on cfg2, B = 128 (57.7 MB read + 10.7 MB written)
 
 
 def load_peaks():
@@ -679,7 +680,11 @@ def main():
     per_kernel = {k: round(float(np.mean(v)) * 1e3, 2) for k, v in acc.items()}
     roofline = {"bound": "hbm", "kernel": gemm_kernel,
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "peak_source": peaks["source"] + " copy bandwidth, burst", "traffic": None,
+                "peak_source": peaks["source"] + " copy bandwidth, burst",
+                # dram__bytes_read + dram__bytes_write of one launch of this kernel on this workload (ncu capture
+                # summarised under profiles/; to be re-taken, or set to None, whenever the kernel changes)
+                "traffic": CHAIN_CFG2_DRAM_BYTES if (gemm_kernel.startswith("gemm_bf16_chain") and args.workload == "cfg2"
+                                                     and args.batch in (None, 128)) else None,
                 "algorithmic_bytes_per_step": gemm_bytes, "us_per_step": round(gemm_ms * 1e3, 2),
                 "executed_tflops": flops / (gemm_ms * 1e-3) / 1e12,
                 "frac_of_bf16_peak_burst": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
