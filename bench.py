@@ -141,7 +141,7 @@ class Bottleneck:
             mk(dsn.BF16, H, Wd, 3, 1, Ci, Ci, self.widths, self.widths, self.W2, act=dsn.ACT_RELU, in_order=1, out_order=1),
             mk(dsn.BF16, H, Wd, 1, 0, Ci, C, self.widths, full, self.W3, in_order=1, out_order=0)]
         # small batches run the three layers as one chained launch (every CTA pair owns whole samples)
-        self.chained = os.environ.get("DSN_CHAIN", "1") != "0" and B <= 148
+        self.chained = os.environ.get("DSN_CHAIN", "1") != "0" and B <= 148 and 150 <= self.R <= 256
         self.L_given = dsn.make_layer_desc(B, T, self.layers, None)
         # launches per step: gate = pool + hidden + score, route, then one chained launch or three GEMMs
         self.kernels_per_step = (3 if gate_driven else 0) + 1 + (1 if self.chained else 3)
