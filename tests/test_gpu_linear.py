@@ -239,3 +239,23 @@ def test_host_side_argument_errors_launch_nothing(dsn, ctx):
     assert code_of(k_in=[8] * 65, k_out=[8] * 65) == dsn.ERR_INVALID_ARG   # T too large
     assert np.all(down(y) == SENTINEL)
     check_status(ctx, dsn)
+
+
+@pytest.mark.parametrize("T,in_order,out_order", [(40, 0, 0), (64, 1, 1)])
+def test_bf16_linear_more_slices_than_one_launch_holds(dsn, ctx, T, in_order, out_order):
+    """A launch carries tensor maps for 16 distinct slices; a layer with more (here 40, and the maximum of
+    64 paths, all distinct) runs as several launches over disjoint sets of groups.  Every group must come out
+    right and nothing outside a group's own columns may be touched."""
+    g = np.random.default_rng(1000 + T)
+    B, R, Ci, Co = 3 * T + 5, 33, 264, 328
+    k_in = [8 * (1 + (5 * t) % 33) for t in range(T)]            # 8 .. 264, all multiples of 8
+    k_out = [8 * (1 + (7 * t + 3) % 41) for t in range(T)]       # 8 .. 328
+    assert len({(a, b) for a, b in zip(k_in, k_out)}) == T
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    x = wl.normal(g, (B, R, Ci))
+    W = wl.normal(g, (Co, Ci), std=Ci ** -0.5)
+    got = _run_bf16_linear(dsn, ctx, x, W, idx, k_in, k_out, R, in_order, out_order, act=dsn.ACT_RELU)
+    ref = O.round_bf16(O.sliced_linear(x, W, idx, k_in, k_out, act=O.ACT_RELU))
+    errs = group_errors(got, ref, idx, k_out, T)
+    assert max(errs.values()) <= TOL_BF16, errs
+    assert_tail_untouched(got, idx, k_out)
