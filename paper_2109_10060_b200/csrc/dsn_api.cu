@@ -274,14 +274,22 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     const int clusters_h = pair_clusters_for(ctx, g.BN);
     if (clusters_h > 0) {
       p.g.pair = 1;
-      // weight ring: a slot per tap for 256-wide n-tiles (6 slots of 16 KB), otherwise a slot holds all nine
-      // taps of a chunk (3 slots of 36 KB, 2 of 72 KB); the rest goes to activation blocks
-      p.g.tps = g.BN == 256 ? 1 : 9;
-      p.g.stages = g.BN == 256 ? 6 : (g.BN == 128 ? 2 : 3);
-      p.g.a_slots = g.BN == 256 ? 2 : 4;
-      while (p.g.a_slots > 2 && dsn_gemm_halo_smem_bytes(g.BN, g.stages, p.g.a_slots, r->G, g.bw, g.bh) > 227 * 1024) --p.g.a_slots;
-      while (p.g.stages > 2 && dsn_gemm_halo_smem_bytes(g.BN, p.g.stages, g.a_slots, r->G, g.bw, g.bh) > 227 * 1024) --p.g.stages;
-      const size_t smem_h = dsn_gemm_halo_smem_bytes(g.BN, g.stages, g.a_slots, r->G, g.bw, g.bh);
+      // Weight ring: a slot holds all nine taps of a chunk where that fits twice (36 KB slots for 64-wide
+      // n-tiles, 72 KB for 128-wide ones), otherwise one tap; the activation ring gets 2 to 4 blocks of what is
+      // left.  Wide images have large blocks: the choice is made on the actual sizes.
+      const size_t limit = 227 * 1024;
+      bool fits = false;
+      for (int tps = (g.BN == 256 ? 1 : 9); !fits; tps = 1) {
+        p.g.tps = tps;
+        p.g.stages = tps == 9 ? (g.BN == 128 ? 2 : 3) : (g.BN == 256 ? 6 : 8);
+        p.g.a_slots = 4;
+        while (p.g.a_slots > 2 && dsn_gemm_halo_smem_bytes(g.BN, g.stages, tps, p.g.a_slots, r->G, g.bw, g.bh) > limit) --p.g.a_slots;
+        while (p.g.stages > 2 && dsn_gemm_halo_smem_bytes(g.BN, p.g.stages, tps, g.a_slots, r->G, g.bw, g.bh) > limit) --p.g.stages;
+        fits = dsn_gemm_halo_smem_bytes(g.BN, g.stages, tps, g.a_slots, r->G, g.bw, g.bh) <= limit;
+        if (tps == 1) break;
+      }
+      if (!fits) return DSN_ERR_UNSUPPORTED;  // cannot happen for W + 2 <= 128: two blocks and two boxes always fit
+      const size_t smem_h = dsn_gemm_halo_smem_bytes(g.BN, g.stages, g.tps, g.a_slots, r->G, g.bw, g.bh);
       int done_h[DSN_MAX_SLICES];
       memset(done_h, 0, sizeof(done_h));
       int remaining_h = c.T;

@@ -307,8 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
 
 }  // namespace
 
-size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int a_slots, int G, int wp, int bh) {
-  const int tps = BN == 256 ? 1 : 9;  // taps per ring slot
+size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int tps, int a_slots, int G, int wp, int bh) {
   return 1024 + kCtrlBytes + (size_t)a_slots * dsn_halo_slot_bytes(wp, bh) + (size_t)stages * tps * ((size_t)(BN / 2) * BK * 2) +
          kStageOutBytes + sizeof(int32_t) * (3 * (size_t)G + 3);
 }

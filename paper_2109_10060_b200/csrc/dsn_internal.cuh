@@ -135,7 +135,7 @@ struct DsnChainParams {
 // launchers implemented in the .cu files
 size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G);
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s);
-size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int a_slots, int G, int wp, int bh);
+size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int tps, int a_slots, int G, int wp, int bh);
 cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s);
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s);
 size_t dsn_gemm_smem_bytes(int BN, int stages, int G);

@@ -215,3 +215,22 @@ def test_layer_forward_vit_mlp_and_config1(dsn, ctx):
     ref1 = O.sliced_linear(c1["x"], c1["W"], c1["idx"], c1["k_in"], c1["k_out"])
     assert max(group_errors(down(y1), ref1, c1["idx"], c1["k_out"], 4).values()) <= 1e-5
     assert_tail_untouched(down(y1), c1["idx"], c1["k_out"])
+
+
+@pytest.mark.parametrize("H,Wd,C,orders", [(20, 12, 48, (0, 0)), (3, 40, 96, (1, 1)), (5, 126, 32, (0, 1)), (33, 17, 128, (1, 0)),
+                                           (1, 13, 64, (0, 0))])
+def test_conv3x3_odd_geometries(dsn, ctx, H, Wd, C, orders):
+    """Non-square images, a last row band shorter than the others, a single image row, an image as wide as a
+    tile (126 + 2 halo pixels = 128 M rows), channel counts that are no multiple of 64: the form of the 3x3
+    layer that stages the tile with its halo must place every pixel and every zero of the padding right."""
+    g = np.random.default_rng(H * 131 + Wd)
+    B, T = 5, 4
+    widths = [max(8, C // 4 - 2), C // 2, (3 * C) // 4 + 2, C]
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    x = wl.normal(g, (B, H, Wd, C), relu=True)
+    W = wl.normal(g, (C, C, 3, 3), std=(9 * C) ** -0.5)
+    got = _run_conv(dsn, ctx, x, W, idx, widths, widths, 1, orders[0], orders[1], act=dsn.ACT_RELU)
+    ref = O.round_bf16(O.sliced_conv(x, W, idx, widths, widths, 1, act=O.ACT_RELU))
+    errs = group_errors(got, ref, idx, widths, T)
+    assert max(errs.values()) <= TOL_BF16, errs
+    assert_tail_untouched(got, idx, widths)
