@@ -99,7 +99,7 @@ def _small_bottleneck(dsn, ctx, B, idx, seed=77):
 
 
 @pytest.mark.parametrize("B,routing", [(1, "uniform"), (2, "uniform"), (75, "uniform"), (148, "uniform"), (149, "uniform"),
-                                       (37, "one_path"), (60, "some_invalid")])
+                                       (37, "one_path"), (60, "some_invalid"), (9, "all_invalid")])
 def test_chained_bottleneck_edge_batches(dsn, B, routing):
     ctx = dsn.Context(0)
     T = 14
@@ -111,15 +111,19 @@ def test_chained_bottleneck_edge_batches(dsn, B, routing):
         idx = idx.copy()
         idx[::7] = -1
         idx[3::11] = T
+    if routing == "all_invalid":
+        idx = np.full(B, T + 3, dtype=np.int32)
     cfg, got = _small_bottleneck(dsn, ctx, B, idx)
     code, detail = ctx.get_status()
     valid = (idx >= 0) & (idx < T)
-    if routing == "some_invalid":
+    if routing in ("some_invalid", "all_invalid"):
         assert code == dsn.ERR_BAD_INDEX and detail == int(np.sum(~valid))   # reported, not fatal
         assert np.all(got[~valid] == SENTINEL)                                # rows of unrouted samples untouched
     else:
         assert code == 0, (code, detail)
     sel = np.nonzero(valid)[0]
+    if len(sel) == 0:
+        return
     _, _, ref = O.bottleneck(cfg["x"][sel], cfg["W1"], cfg["W2"], cfg["W3"], idx[sel], cfg["widths"], mirror_bf16=True)
     errs = group_errors(got[sel], ref, idx[sel], [cfg["C_outer"]] * T, T)
     assert max(errs.values()) <= 1e-2, errs
