@@ -182,7 +182,12 @@ typedef struct dsn_layer_desc {
 
 /* ---- context ------------------------------------------------------------------------- */
 /* Creates a context on CUDA device `device` (allocates a few hundred bytes of device memory
- * for the status word; the only allocation the library ever makes). */
+ * for the status word; the only allocation the library ever makes).
+ * Environment switches, read here, that select between kernels computing the same results (for
+ * comparisons and as fallbacks): DSN_GEMM_MODE=1cta (one CTA per tile instead of CTA pairs),
+ * DSN_CHAIN=0 (dsn_layer_forward: one launch per layer even for small batches), DSN_CONV3X3=taps
+ * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_PDL=0 (no
+ * programmatic dependent launch). */
 int dsn_create(dsn_ctx** ctx, int device);
 int dsn_destroy(dsn_ctx* ctx);
 const char* dsn_strerror(int code);
@@ -286,7 +291,11 @@ int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_ro
 
 /* ---- whole dynamic block (Eq. (dyn_net)) ------------------------------------------------ */
 size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L);
-/* x, y in input order.  idx_in: device [B], required when L->gate is NULL, ignored otherwise.
+/* Gate (or the given indices) -> routing -> the block's layers, all layers under the one decision
+ * (Sec. 5).  Batches of at most two samples per SM pair whose samples have 150..256 rows (14x14
+ * images, 197 tokens) run their 2-3 sliced layers as ONE launch in which every SM pair walks whole
+ * samples through the layers; otherwise one launch per layer.  Same results either way.
+ * x, y in input order.  idx_in: device [B], required when L->gate is NULL, ignored otherwise.
  * r_out (optional): receives pointers into the workspace holding the block's routing arrays
  * (valid until the workspace is reused).  idx_out (optional): device [B], the gate's choice. */
 int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, const int32_t* idx_in,
