@@ -301,7 +301,7 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------------------- per-layer table
 def run_table(args):
-    """Per-layer numbers for every configuration (markdown rows for the benchmark spec): CUDA-graph replay over
+    """Per-layer numbers for every configuration (markdown table rows): CUDA-graph replay over
     rotating buffers larger than L2, executed TFLOP/s, fraction of the shape's roofline bound."""
     import torch
     from paper_2109_10060_b200.build import build
