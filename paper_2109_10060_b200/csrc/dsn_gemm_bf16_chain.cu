@@ -44,7 +44,8 @@ __device__ __forceinline__ uint32_t cta_addr_in_cluster(uint32_t local_addr, uin
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
   return r;
 }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// orders accesses to global memory through the generic proxy (plain loads / stores) and through the async proxy (TMA)
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
 // Bounded wait until the counter reaches `target`.
 static __device__ __noinline__ bool wait_counter(uint32_t addr, uint32_t target, volatile uint32_t* abort_flag,
