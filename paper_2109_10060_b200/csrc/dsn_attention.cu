@@ -168,42 +168,51 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   if (ok) {
     tc_fence_after();
     const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    // ---- this thread's part of the S row, in registers
-    uint32_t v[4][32];
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-      if (32 * c < cols_per) tmem_ld_32x32(trow + cbeg + 32 * c, v[c]);  // uniform over the CTA
-    tmem_ld_wait();
-    // Keys >= N (next sample's rows, or padding) are masked once, by overwriting their scores with -inf
-    // in the one 32-key block of this thread that straddles N; everything after that is free of
-    // per-element bounds checks (the inner loops are instruction-issue bound).
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int kb = cbeg + 32 * c;  // first key of the block
-      if (32 * c < cols_per && kb + 32 > N) {
+    // ---- pass 1 over this thread's part of the S row: the maximum.  The scores are read from TMEM one
+    // 32-key block at a time and not kept: 104 scores per thread would not fit the register budget of two
+    // CTAs per SM, and a second read of TMEM (pass 2) is cheaper than spilling them.
+    // Keys >= N (next sample's rows, or padding) count as -inf; only the block that straddles N pays for the test.
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int c = 0; 32 * c < cols_per; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(trow + cbeg + 32 * c, v);
+      tmem_ld_wait();
+      const int kb = cbeg + 32 * c;                                  // first key of the block
+      const int nk = cols_per - 32 * c < 32 ? cols_per - 32 * c : 32;  // keys of this part in the block (multiple of 8)
+      if (kb + nk > N) {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-          if (kb + i >= N) v[c][i] = 0xff800000u;  // -inf
+          if (i < nk && kb + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
+      } else if (nk == 32) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (i < nk) mx = fmaxf(mx, __uint_as_float(v[i]));
       }
     }
-    float mx = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-      if (32 * c < cols_per) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 2)
-          if (32 * c + i < cols_per)  // whole blocks except the last one of the part; multiple of 8, compile-time stride
-            mx = fmaxf(mx, fmaxf(__uint_as_float(v[c][i]), __uint_as_float(v[c][i + 1])));
-      }
     s_red[part * 128 + m] = mx;
-    tc_fence_before();
-    __syncthreads();  // also: every thread has its S values, and K and Q are no longer needed
+    __syncthreads();
     mx = fmaxf(s_red[m], s_red[128 + m]);
     __syncthreads();
     const float mxs = mx * sl2;
     float sum = 0.f;
+    // ---- pass 2: exp2(s * c - max * c), one FMA and one special-function instruction per key, probabilities
+    // rounded to bf16 into the swizzled P tile (which overlays K and Q: S has been computed, and pass 1 of
+    // every thread is over)
+#pragma unroll 1
+    for (int c = 0; 32 * c < cols_per; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(trow + cbeg + 32 * c, v);
+      tmem_ld_wait();
+      const int kb = cbeg + 32 * c;
+      if (kb + 32 > N) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+        for (int i = 0; i < 32; ++i)
+          if (kb + i >= N) v[i] = 0xff800000u;  // -inf: probability 0
+      }
 #pragma unroll
       for (int jv = 0; jv < 4; ++jv) {
         const int j0 = 32 * c + 8 * jv;       // first of 8 keys, relative to the part
@@ -211,10 +220,9 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            // exp2(s * c - max * c): one FMA and one special-function instruction per key; -inf gives 0
             float a, b;
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[c][8 * jv + 2 * e]), sl2, -mxs)));
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[c][8 * jv + 2 * e + 1]), sl2, -mxs)));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e]), sl2, -mxs)));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e + 1]), sl2, -mxs)));
             sum += a + b;
             __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
             w[e] = *reinterpret_cast<uint32_t*>(&hb);
@@ -225,6 +233,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
         }
       }
     }
+    tc_fence_before();  // the PV product writes its accumulator over the columns just read
     s_red[part * 128 + m] = sum;
     fence_async_smem();
     tc_fence_before();
