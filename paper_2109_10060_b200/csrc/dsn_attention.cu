@@ -14,9 +14,9 @@
 //   used as loaded (its rows >= N are cleared: they belong to the next sample);
 //   S = Q K^T: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
 //   two threads share one query row (warps w and w + 4 own the same TMEM lanes and half of the keys
-//   each): one pass over their part of the S row held in registers gives the row maximum, the
-//   exponentials, the row sum and P as bf16 in a swizzled K-major shared-memory tile that reuses the
-//   space of K and Q (keys >= N: zeros);
+//   each): a first pass over their part of the S row, read from TMEM 32 keys at a time, gives the row
+//   maximum; a second pass the exponentials, the row sum and P as bf16 in a swizzled K-major
+//   shared-memory tile that reuses the space of K and Q (keys >= N: zeros);
 //   O = P V: tcgen05.mma M = 128, N = 64, K = keys rounded to 16, into the TMEM columns S has left;
 //   the row is scaled by 1 / sum, rounded to bf16 and stored (each of the two threads writes 64 bytes
 //   of the 128-byte line).
