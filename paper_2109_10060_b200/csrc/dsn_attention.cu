@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   const int npad = (N + 15) & ~15;
   const int kboxes = npad > 128 ? 2 : 1;
 
-  if (warp == 0) {
+  if (warp == 1) {  // not the warp that issues the loads: the allocation may have to wait for the SM's other CTA
     tmem_alloc(smem_u32(tmem_slot), kAttTmemCols);
     tmem_relinquish();
   }
@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 1) {
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, kAttTmemCols);
