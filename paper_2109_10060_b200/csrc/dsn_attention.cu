@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   const uint32_t bar_load = base, bar_mma = base + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 20);
-  int32_t* s_info = reinterpret_cast<int32_t*>(smem + 24);
+  int32_t* s_heads = reinterpret_cast<int32_t*>(smem + 24);
   float* s_red = reinterpret_cast<float*>(smem + 64);  // [2 parts][128 rows]: maxima, then sums
   const uint32_t v_s = base + 2048, k_s = v_s + kVBytes, q_s = k_s + kKBytes, p_s = k_s;
   uint8_t* v_ptr = smem + 2048;
@@ -92,34 +92,30 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
   if (half * 128 >= p.N) return;
-  // Group of this position = (number of groups whose first position is <= pos) - 1, counted by the whole
-  // CTA in one round of loads instead of a chain of dependent ones; perm[pos] travels at the same time.
-  int blk_reg = 0;
-  if (tid == 0) blk_reg = p.grouped ? pos : p.perm[pos];
-  int n_le = 0;
-  for (int g0 = 0; g0 < p.G; g0 += kAttThreads) {
-    const int g = g0 + tid;
-    n_le += __syncthreads_count(g < p.G && p.offsets[g] <= pos);
-  }
   if (tid == 0) {
-    int h = 0;
-    const int g = n_le - 1;
-    if (g >= 0 && pos < p.offsets[p.G]) {
-      const int sl = p.group_slice ? p.group_slice[g] : g;
-      if (sl >= 0 && sl < p.T) h = p.heads[sl];
-      if (blk_reg < 0) h = 0;
-    }
-    s_info[0] = h;
-    s_info[1] = blk_reg;
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();
-  if (head >= s_info[0]) return;  // this sample's path has fewer heads (uniform over the CTA)
+  // The group of this position is the one with offsets[g] <= pos < offsets[g+1] (empty groups never match).
+  // Thread g tests group g and fetches that group's head count at the same time, so the lookup costs two
+  // dependent loads instead of a chain of four; the owner leaves the count in shared memory and the barrier tells everybody whether there was an owner.
+  const int blk = p.grouped ? pos : p.perm[pos];
+  int owner = 0;
+  for (int g = tid; g < p.G; g += kAttThreads) {
+    const int lo = p.offsets[g], hi = p.offsets[g + 1];
+    const int sl = p.group_slice ? p.group_slice[g] : g;
+    const int hh = (sl >= 0 && sl < p.T) ? p.heads[sl] : 0;
+    if (lo <= pos && pos < hi) {
+      owner = 1;
+      *s_heads = hh;
+    }
+  }
+  const int heads_here = (__syncthreads_or(owner) && blk >= 0) ? *s_heads : 0;
+  if (head >= heads_here) return;  // this sample's path has fewer heads (uniform over the CTA)
   const int N = p.N;
-  const int64_t row0 = (int64_t)s_info[1] * N;
+  const int64_t row0 = (int64_t)blk * N;
   const int npad = (N + 15) & ~15;
   const int kboxes = npad > 128 ? 2 : 1;
 
