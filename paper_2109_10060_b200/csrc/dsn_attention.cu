@@ -5,9 +5,12 @@
 // the output row holds [head][64] and feeds the sliced projection (k_in = h * 64).  Heads >= h of a
 // sample are neither read nor written.
 //
-// One CTA (256 threads) per (sample, head, half of the queries), N <= 256 tokens, D_h = 64; two CTAs
-// fit on an SM (about 99 KB of shared memory and 256 TMEM columns each), so one CTA's loads and
-// barriers hide behind the other's arithmetic:
+// One work item = (sample, head, half of the queries), N <= 256 tokens, D_h = 64, worked by one CTA of
+// 256 threads; two CTAs fit on an SM (about 99 KB of shared memory and 256 TMEM columns each), so one
+// CTA's loads and barriers hide behind the other's arithmetic.  Two CTAs per SM walk the list of items
+// that exist (heads a path does not have are not in it) and fetch the next item's tiles while the
+// current output leaves; with more groups than the item table holds, one CTA per item of the dense grid.
+// Per item:
 //   Q [128 queries][64], K [256 keys][64] and V [256 keys][64] arrive by TMA (128-byte rows,
 //   128-byte swizzle).  K is the K-major B operand of S = Q K^T; V, whose rows are keys and whose
 //   64 contiguous elements are the head dimension, is the MN-major B operand of O = P V, so it is
@@ -70,67 +73,126 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
   return d;
 }
 
+constexpr int kAttTableGroups = 64;  // groups the persistent form can hold in its shared-memory table
+
+// One work item = (sample position, head, half of the queries).  kPersist = false: one CTA per item of
+// the dense grid (head, position, half); items of heads the sample's path does not have return at once.
+// kPersist = true (G <= kAttTableGroups): a fixed grid of CTAs walks the list of existing items
+// (group by group: position, half, head fastest) with a stride of gridDim.x.  Each CTA builds the
+// per-group item prefix once, so that finding an item needs no global load, allocates TMEM and
+// initialises its barriers once, and issues the loads of its next item as soon as the P V product of
+// the current one has finished with shared memory, i.e. under the read-out and store of O.
+template <bool kPersist>
 __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_constant__ AttParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  // layout: control 2 KB (barriers, row maxima and sums) | V 32 KB | K 32 KB | Q 16 KB | 16 KB;
+  // layout: control 2 KB (barriers, row maxima and sums, item table) | V 32 KB | K 32 KB | Q 16 KB | 16 KB;
   // P (64 KB) overlays K, Q and the last 16 KB once S has been computed
   const uint32_t bar_load = base, bar_mma = base + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 20);
   int32_t* s_heads = reinterpret_cast<int32_t*>(smem + 24);
   float* s_red = reinterpret_cast<float*>(smem + 64);  // [2 parts][128 rows]: maxima, then sums
+  int32_t* s_pre = reinterpret_cast<int32_t*>(smem + 1088);  // [G + 1] items before group g
+  int32_t* s_off = s_pre + kAttTableGroups + 1;              // [G] first position of group g
+  int32_t* s_h = s_off + kAttTableGroups;                    // [G] heads of group g's path
   const uint32_t v_s = base + 2048, k_s = v_s + kVBytes, q_s = k_s + kKBytes, p_s = k_s;
   uint8_t* v_ptr = smem + 2048;
   uint8_t* p_ptr = v_ptr + kVBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int head = blockIdx.x, pos = blockIdx.y, half = blockIdx.z;
+  const int N = p.N;
+  const int halves = N > 128 ? 2 : 1;
 
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
-  if (half * 128 >= p.N) return;
   if (tid == 0) {
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // The group of this position is the one with offsets[g] <= pos < offsets[g+1] (empty groups never match).
-  // Thread g tests group g and fetches that group's head count at the same time, so the lookup costs two
-  // dependent loads instead of a chain of four; the owner leaves the count in shared memory and the barrier tells everybody whether there was an owner.
-  const int blk = p.grouped ? pos : p.perm[pos];
-  int owner = 0;
-  for (int g = tid; g < p.G; g += kAttThreads) {
-    const int lo = p.offsets[g], hi = p.offsets[g + 1];
-    const int sl = p.group_slice ? p.group_slice[g] : g;
-    const int hh = (sl >= 0 && sl < p.T) ? p.heads[sl] : 0;
-    if (lo <= pos && pos < hi) {
-      owner = 1;
-      *s_heads = hh;
+
+  int head, half, blk;       // the current item
+  int it = 0, total = 0;     // persistent form: its index in the item list, and the length of the list
+  const int stride = kPersist ? (int)gridDim.x : 1;
+  // item `i` of the list -> (head, half, row block); false when the sample is not part of the batch
+  auto decode = [&](int i, int& hd, int& hf, int& bk) {
+    int g = 0;
+    while (s_pre[g + 1] <= i) ++g;  // i < s_pre[G]: ends; empty groups are stepped over
+    const int local = i - s_pre[g], hg = s_h[g];
+    const int r = local / hg;
+    hd = local - r * hg;
+    hf = halves == 2 ? (r & 1) : 0;
+    const int pos = s_off[g] + (halves == 2 ? (r >> 1) : r);
+    bk = p.grouped ? pos : p.perm[pos];
+    return bk >= 0;
+  };
+  if (kPersist) {
+    for (int g = tid; g < p.G; g += kAttThreads) {
+      const int lo = p.offsets[g], hi = p.offsets[g + 1];
+      const int sl = p.group_slice ? p.group_slice[g] : g;
+      const int hh = (sl >= 0 && sl < p.T) ? p.heads[sl] : 0;
+      s_off[g] = lo;
+      s_h[g] = hh;
+      s_pre[g + 1] = (hi - lo) * hh * halves;
     }
+    __syncthreads();
+    if (tid == 0) {
+      int acc = 0;
+      s_pre[0] = 0;
+      for (int g = 0; g < p.G; ++g) {
+        acc += s_pre[g + 1];
+        s_pre[g + 1] = acc;
+      }
+    }
+    __syncthreads();
+    total = s_pre[p.G];
+    it = blockIdx.x;
+    while (it < total && !decode(it, head, half, blk)) it += stride;
+    if (it >= total) return;  // nothing for this CTA (uniform)
+  } else {
+    head = blockIdx.x;
+    half = blockIdx.z;
+    const int pos = blockIdx.y;
+    if (half * 128 >= N) return;
+    // The group of this position is the one with offsets[g] <= pos < offsets[g+1] (empty groups never match).
+    // Thread g tests group g and fetches that group's head count at the same time, so the lookup costs two
+    // dependent loads instead of a chain of four; the owner leaves the count in shared memory and the
+    // barrier tells everybody whether there was an owner.
+    blk = p.grouped ? pos : p.perm[pos];
+    int owner = 0;
+    for (int g = tid; g < p.G; g += kAttThreads) {
+      const int lo = p.offsets[g], hi = p.offsets[g + 1];
+      const int sl = p.group_slice ? p.group_slice[g] : g;
+      const int hh = (sl >= 0 && sl < p.T) ? p.heads[sl] : 0;
+      if (lo <= pos && pos < hi) {
+        owner = 1;
+        *s_heads = hh;
+      }
+    }
+    const int heads_here = (__syncthreads_or(owner) && blk >= 0) ? *s_heads : 0;
+    if (head >= heads_here) return;  // this sample's path has fewer heads (uniform over the CTA)
   }
-  const int heads_here = (__syncthreads_or(owner) && blk >= 0) ? *s_heads : 0;
-  if (head >= heads_here) return;  // this sample's path has fewer heads (uniform over the CTA)
-  const int N = p.N;
-  const int64_t row0 = (int64_t)blk * N;
   const int npad = (N + 15) & ~15;
   const int kboxes = npad > 128 ? 2 : 1;
+  auto issue_loads = [&](int hd, int hf, int bk) {  // by one elected lane
+    const int r0 = bk * N;
+    mbar_expect_tx(bar_load, (uint32_t)kboxes * 2u * 16384u + kQBytes);
+    for (int b2 = 0; b2 < kboxes; ++b2) {
+      tma_load_3d(k_s + b2 * 16384, &p.map, 0, hd * 3 + 1, r0 + 128 * b2, bar_load);
+      tma_load_3d(v_s + b2 * 16384, &p.map, 0, hd * 3 + 2, r0 + 128 * b2, bar_load);
+    }
+    tma_load_3d(q_s, &p.map, 0, hd * 3 + 0, r0 + 128 * hf, bar_load);
+  };
 
   if (warp == 1) {  // not the warp that issues the loads: the allocation may have to wait for the SM's other CTA
     tmem_alloc(smem_u32(tmem_slot), kAttTmemCols);
     tmem_relinquish();
   }
-  if (warp == 0 && elect_one()) {  // one elected lane of a converged warp: operands stay in uniform registers
-    mbar_expect_tx(bar_load, (uint32_t)kboxes * 2u * 16384u + kQBytes);
-    for (int b2 = 0; b2 < kboxes; ++b2) {
-      tma_load_3d(k_s + b2 * 16384, &p.map, 0, head * 3 + 1, (int)row0 + 128 * b2, bar_load);
-      tma_load_3d(v_s + b2 * 16384, &p.map, 0, head * 3 + 2, (int)row0 + 128 * b2, bar_load);
-    }
-    tma_load_3d(q_s, &p.map, 0, head * 3 + 0, (int)row0 + 128 * half, bar_load);
-  }
+  if (warp == 0 && elect_one()) issue_loads(head, half, blk);  // operands stay in uniform registers
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -138,55 +200,68 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   const uint32_t idesc_s = make_idesc(128, npad);
   const uint32_t idesc_o = make_idesc(128, 64) | (1u << 16);  // B operand MN-major
   const float sl2 = 0.125f * 1.4426950408889634f;             // 1/sqrt(64) * log2(e)
-
-  bool ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag, p.status, 21) ? 1 : 0) != 0;
-  if (ok) {
-    // V rows >= N belong to the next sample (or to nobody): clear them so that 0 * garbage cannot appear
-    for (int e = tid; e < (npad - N) * 8; e += kAttThreads)
-      *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-    fence_async_smem();
-    __syncthreads();
-    if (warp == 0 && elect_one()) {
-      tc_fence_after();
-      const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_base, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-      umma_commit(bar_mma);
-    }
-    ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag, p.status, 22) ? 1 : 0) != 0;
-  }
-
   const int part = warp >> 2;                 // which half of the keys this thread owns
   const int m = (warp & 3) * 32 + lane;       // query row within the half = TMEM lane
   const int cols_per = npad >> 1;             // keys per part, a multiple of 8
   const int cbeg = part * cols_per;
+  const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
 
-  if (ok) {
+  for (uint32_t n_done = 0;; ++n_done) {
+    // the item after this one (persistent form); its row block may need one load from the permutation
+    int head_n = 0, half_n = 0, blk_n = 0, it_n = total;
+    if (kPersist) {
+      it_n = it + stride;
+      while (it_n < total && !decode(it_n, head_n, half_n, blk_n)) it_n += stride;
+    }
+    const int64_t row0 = (int64_t)blk * N;
+    // a warp whose 32 query rows all lie beyond N has no row to normalise: it only keeps the barriers
+    const bool rows_live = half * 128 + (warp & 3) * 32 < N;
+
+    bool ok = __syncthreads_and(mbar_wait(bar_load, n_done & 1u, abort_flag, p.status, 21) ? 1 : 0) != 0;
+    if (ok) {
+      // V rows >= N belong to the next sample (or to nobody): clear them so that 0 * garbage cannot appear
+      for (int e = tid; e < (npad - N) * 8; e += kAttThreads)
+        *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+      fence_async_smem();
+      tc_fence_before();  // the O columns of the item before have been read by every thread
+      __syncthreads();
+      if (warp == 0 && elect_one()) {
+        tc_fence_after();
+        const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) umma_bf16(tmem_base, dq + 2u * ks, dk + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
+        umma_commit(bar_mma);
+      }
+      ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag, p.status, 22) ? 1 : 0) != 0;
+    }
+    if (!ok) break;
+
     tc_fence_after();
-    const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     // ---- pass 1 over this thread's part of the S row: the maximum.  The scores are read from TMEM one
     // 32-key block at a time and not kept: 104 scores per thread would not fit the register budget of two
     // CTAs per SM, and a second read of TMEM (pass 2) is cheaper than spilling them.
     // Keys >= N (next sample's rows, or padding) count as -inf; only the block that straddles N pays for the test.
     float mx = -INFINITY;
+    if (rows_live) {
 #pragma unroll 1
-    for (int c = 0; 32 * c < cols_per; ++c) {
-      uint32_t v[32];
-      tmem_ld_32x32(trow + cbeg + 32 * c, v);
-      tmem_ld_wait();
-      const int kb = cbeg + 32 * c;                                  // first key of the block
-      const int nk = cols_per - 32 * c < 32 ? cols_per - 32 * c : 32;  // keys of this part in the block (multiple of 8)
-      if (kb + nk > N) {
+      for (int c = 0; 32 * c < cols_per; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(trow + cbeg + 32 * c, v);
+        tmem_ld_wait();
+        const int kb = cbeg + 32 * c;                                  // first key of the block
+        const int nk = cols_per - 32 * c < 32 ? cols_per - 32 * c : 32;  // keys of this part in the block (multiple of 8)
+        if (kb + nk > N) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i < nk && kb + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
-      } else if (nk == 32) {
+          for (int i = 0; i < 32; ++i)
+            if (i < nk && kb + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
+        } else if (nk == 32) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
-      } else {
+          for (int i = 0; i < 32; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+        } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i < nk) mx = fmaxf(mx, __uint_as_float(v[i]));
+          for (int i = 0; i < 32; ++i)
+            if (i < nk) mx = fmaxf(mx, __uint_as_float(v[i]));
+        }
       }
     }
     s_red[part * 128 + m] = mx;
@@ -197,42 +272,44 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
     float sum = 0.f;
     // ---- pass 2: exp2(s * c - max * c), one FMA and one special-function instruction per key, probabilities
     // rounded to bf16 into the swizzled P tile (which overlays K and Q: S has been computed, and pass 1 of
-    // every thread is over)
+    // every thread is over).  Rows of a warp that is not live keep whatever the tile held: a row of P only
+    // reaches the same row of O, which is not stored.
+    if (rows_live) {
 #pragma unroll 1
-    for (int c = 0; 32 * c < cols_per; ++c) {
-      uint32_t v[32];
-      tmem_ld_32x32(trow + cbeg + 32 * c, v);
-      tmem_ld_wait();
-      const int kb = cbeg + 32 * c;
-      if (kb + 32 > N) {
+      for (int c = 0; 32 * c < cols_per; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(trow + cbeg + 32 * c, v);
+        tmem_ld_wait();
+        const int kb = cbeg + 32 * c;
+        if (kb + 32 > N) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (kb + i >= N) v[i] = 0xff800000u;  // -inf: probability 0
-      }
+          for (int i = 0; i < 32; ++i)
+            if (kb + i >= N) v[i] = 0xff800000u;  // -inf: probability 0
+        }
 #pragma unroll
-      for (int jv = 0; jv < 4; ++jv) {
-        const int j0 = 32 * c + 8 * jv;       // first of 8 keys, relative to the part
-        if (j0 < cols_per) {
-          uint32_t w[4];
+        for (int jv = 0; jv < 4; ++jv) {
+          const int j0 = 32 * c + 8 * jv;       // first of 8 keys, relative to the part
+          if (j0 < cols_per) {
+            uint32_t w[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float a, b;
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e]), sl2, -mxs)));
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e + 1]), sl2, -mxs)));
-            sum += a + b;
-            __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
-            w[e] = *reinterpret_cast<uint32_t*>(&hb);
+            for (int e = 0; e < 4; ++e) {
+              float a, b;
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e]), sl2, -mxs)));
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e + 1]), sl2, -mxs)));
+              sum += a + b;
+              __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
+              w[e] = *reinterpret_cast<uint32_t*>(&hb);
+            }
+            const int key = cbeg + j0;
+            *reinterpret_cast<uint4*>(p_ptr + (key >> 6) * 16384 + m * 128 + ((((key & 63) >> 3) ^ (m & 7)) << 4)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
           }
-          const int key = cbeg + j0;
-          *reinterpret_cast<uint4*>(p_ptr + (key >> 6) * 16384 + m * 128 + ((((key & 63) >> 3) ^ (m & 7)) << 4)) =
-              make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }
     tc_fence_before();  // the PV product writes its accumulator over the columns just read
     s_red[part * 128 + m] = sum;
     fence_async_smem();
-    tc_fence_before();
     __syncthreads();
     sum = s_red[m] + s_red[128 + m];
 
@@ -247,29 +324,36 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
       umma_commit(bar_mma);
     }
     ok = __syncthreads_and(mbar_wait(bar_mma, 1, abort_flag, p.status, 23) ? 1 : 0) != 0;
-    if (ok) {
-      tc_fence_after();
-      const uint32_t orow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + 32 * part;
+    if (!ok) break;
+    // the tensor core has finished with P and V: the next item's tiles may land while O leaves
+    if (kPersist && it_n < total && warp == 0 && elect_one()) issue_loads(head_n, half_n, blk_n);
+    tc_fence_after();
+    {
+      const uint32_t orow = trow + 32 * part;
       const int q = half * 128 + m;
       const float inv = 1.f / sum;
       __nv_bfloat16* dst = p.out + (row0 + q) * p.ld_out + (int64_t)head * 64 + 32 * part;
-      uint32_t o[32];
-      tmem_ld_32x32(orow, o);
-      tmem_ld_wait();
-      if (q < N) {
+      if (rows_live) {
+        uint32_t o[32];
+        tmem_ld_32x32(orow, o);
+        tmem_ld_wait();
+        if (q < N) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t w[4];
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 hb = __floats2bfloat162_rn(__uint_as_float(o[8 * j + 2 * e]) * inv,
-                                                      __uint_as_float(o[8 * j + 2 * e + 1]) * inv);
-            w[e] = *reinterpret_cast<uint32_t*>(&hb);
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 hb = __floats2bfloat162_rn(__uint_as_float(o[8 * j + 2 * e]) * inv,
+                                                        __uint_as_float(o[8 * j + 2 * e + 1]) * inv);
+              w[e] = *reinterpret_cast<uint32_t*>(&hb);
+            }
+            *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(w[0], w[1], w[2], w[3]);
           }
-          *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }
+    if (!kPersist || it_n >= total) break;
+    it = it_n; head = head_n; half = half_n; blk = blk_n;
   }
 
   tc_fence_before();
@@ -303,10 +387,23 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   p.status = status;
   const size_t smem = 1024 + 2048 + kVBytes + kPBytes;  // P overlays K, Q and 16 KB more
   static bool configured = false;
+  static int resident = 0;  // CTAs the persistent form keeps in flight: two per SM
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    int dev = 0, sms = 0;
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
+    resident = 2 * sms;
     configured = true;
   }
-  return dsn_launch(attention_kernel, dim3(H, B, N > 128 ? 2 : 1), dim3(kAttThreads), smem, s, 1, p);
+  const int halves = N > 128 ? 2 : 1;
+  if (G <= kAttTableGroups) {
+    const long long dense = (long long)H * B * halves;
+    return dsn_launch(attention_kernel<true>, dim3((unsigned)(dense < resident ? dense : resident)), dim3(kAttThreads), smem, s,
+                      1, p);
+  }
+  return dsn_launch(attention_kernel<false>, dim3(H, B, halves), dim3(kAttThreads), smem, s, 1, p);
 }

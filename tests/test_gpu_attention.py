@@ -25,7 +25,10 @@ def head_major(q, k, v, H, Dh):
 
 @pytest.mark.parametrize("B,N,H,heads,order", [(24, 197, 6, [3, 4, 5, 6], 0), (24, 197, 6, [3, 4, 5, 6], 1),
                                                (10, 197, 12, [5, 6, 7, 8, 9, 10, 11, 12], 1), (6, 64, 4, [1, 4], 0),
-                                               (5, 256, 2, [2, 1], 1), (7, 130, 3, [3], 0), (4, 16, 2, [2, 1], 0)])
+                                               (5, 256, 2, [2, 1], 1), (7, 130, 3, [3], 0), (4, 16, 2, [2, 1], 0),
+                                               # more (sample, head, half) items than resident CTAs: several per CTA
+                                               (96, 197, 6, [3, 4, 5, 6], 0), (96, 197, 6, [3, 4, 5, 6], 1),
+                                               (200, 100, 3, [1, 2, 3], 1)])
 def test_attention_matches_oracle(dsn, ctx, B, N, H, heads, order):
     g = np.random.default_rng(B * 1000 + N + H)
     Dh, T = 64, len(heads)
@@ -51,6 +54,32 @@ def test_attention_matches_oracle(dsn, ctx, B, N, H, heads, order):
         err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
         assert err <= TOL, (i, int(idx[i]), err)
         assert np.all(got[i, :, w:] == SENTINEL)          # heads the path does not have stay untouched
+
+
+def test_attention_more_groups_than_the_item_table_holds(dsn, ctx):
+    """Caller-built list of 70 one-sample groups (slice g mod T): the one-CTA-per-item form of the kernel."""
+    B, N, H, Dh, heads = 70, 197, 4, 64, [2, 4, 3]
+    g = np.random.default_rng(11)
+    T = len(heads)
+    order = g.permutation(B).astype(np.int32)             # group j holds sample order[j]
+    idx = (np.arange(B) % T).astype(np.int32)
+    slices = idx[order]
+    inv = np.empty(B, np.int32)
+    inv[order] = np.arange(B, dtype=np.int32)
+    q, k, v = (wl.normal(g, (B, N, H * Dh)) for _ in range(3))
+    bufs = [torch.from_numpy(a.astype(np.int32)).to(DEV) for a in (np.ones(B), np.arange(B + 1), order, inv, slices)]
+    r = dsn.make_routing(B, B, *bufs)
+    out = torch.full((B, N, H * Dh), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(N, H, Dh, heads, order=0), r,
+                             up_bf16(head_major(q, k, v, H, Dh)), out)
+    check_status(ctx, dsn)
+    got = down(out)
+    ref = O.attention(q, k, v, idx, heads, Dh)
+    for i in range(B):
+        w = heads[idx[i]] * Dh
+        err = np.max(np.abs(got[i, :, :w] - ref[i, :, :w])) / np.max(np.abs(ref[i, :, :w]))
+        assert err <= TOL, (i, int(idx[i]), err)
+        assert np.all(got[i, :, w:] == SENTINEL)
 
 
 def test_attention_closed_forms_on_device(dsn, ctx):
