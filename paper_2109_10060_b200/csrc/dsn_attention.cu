@@ -88,18 +88,19 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  // layout: control 2 KB (barriers, row maxima and sums, item table) | V 32 KB | K 32 KB | Q 16 KB | 16 KB;
+  // layout: control 3 KB (barriers, row maxima, row sums, item table) | V 32 KB | K 32 KB | Q 16 KB | 16 KB;
   // P (64 KB) overlays K, Q and the last 16 KB once S has been computed
   const uint32_t bar_load = base, bar_mma = base + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 20);
   int32_t* s_heads = reinterpret_cast<int32_t*>(smem + 24);
-  float* s_red = reinterpret_cast<float*>(smem + 64);  // [2 parts][128 rows]: maxima, then sums
-  int32_t* s_pre = reinterpret_cast<int32_t*>(smem + 1088);  // [G + 1] items before group g
+  float* s_max = reinterpret_cast<float*>(smem + 64);     // [2 parts][128 rows] row maxima
+  float* s_sum = reinterpret_cast<float*>(smem + 1088);   // [2 parts][128 rows] row sums
+  int32_t* s_pre = reinterpret_cast<int32_t*>(smem + 2112);  // [G + 1] items before group g
   int32_t* s_off = s_pre + kAttTableGroups + 1;              // [G] first position of group g
   int32_t* s_h = s_off + kAttTableGroups;                    // [G] heads of group g's path
-  const uint32_t v_s = base + 2048, k_s = v_s + kVBytes, q_s = k_s + kKBytes, p_s = k_s;
-  uint8_t* v_ptr = smem + 2048;
+  const uint32_t v_s = base + 3072, k_s = v_s + kVBytes, q_s = k_s + kKBytes, p_s = k_s;
+  uint8_t* v_ptr = smem + 3072;
   uint8_t* p_ptr = v_ptr + kVBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -222,9 +223,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
       // V rows >= N belong to the next sample (or to nobody): clear them so that 0 * garbage cannot appear
       for (int e = tid; e < (npad - N) * 8; e += kAttThreads)
         *reinterpret_cast<uint4*>(v_ptr + (N + (e >> 3)) * 128 + (e & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-      fence_async_smem();
-      tc_fence_before();  // the O columns of the item before have been read by every thread
-      __syncthreads();
+      // (these rows are first read by the P V product, behind the barrier that follows the softmax)
       if (warp == 0 && elect_one()) {
         tc_fence_after();
         const uint64_t dq = make_smem_desc(q_s), dk = make_smem_desc(k_s);
@@ -264,10 +263,9 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
         }
       }
     }
-    s_red[part * 128 + m] = mx;
+    s_max[part * 128 + m] = mx;
     __syncthreads();
-    mx = fmaxf(s_red[m], s_red[128 + m]);
-    __syncthreads();
+    mx = fmaxf(s_max[m], s_max[128 + m]);
     const float mxs = mx * sl2;
     float sum = 0.f;
     // ---- pass 2: exp2(s * c - max * c), one FMA and one special-function instruction per key, probabilities
@@ -308,10 +306,10 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
       }
     }
     tc_fence_before();  // the PV product writes its accumulator over the columns just read
-    s_red[part * 128 + m] = sum;
+    s_sum[part * 128 + m] = sum;
     fence_async_smem();
     __syncthreads();
-    sum = s_red[m] + s_red[128 + m];
+    sum = s_sum[m] + s_sum[128 + m];
 
     // ---- O = P V, into the columns S occupied
     if (warp == 0 && elect_one()) {
@@ -353,6 +351,7 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
       }
     }
     if (!kPersist || it_n >= total) break;
+    tc_fence_before();  // O has been read: the next item's S may overwrite it once every thread has passed the load barrier
     it = it_n; head = head_n; half = half_n; blk = blk_n;
   }
 
@@ -385,7 +384,7 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   p.qkv = static_cast<const __nv_bfloat16*>(qkv); p.ld_qkv = ld_qkv;
   p.out = static_cast<__nv_bfloat16*>(out); p.ld_out = ld_out;
   p.status = status;
-  const size_t smem = 1024 + 2048 + kVBytes + kPBytes;  // P overlays K, Q and 16 KB more
+  const size_t smem = 1024 + 3072 + kVBytes + kPBytes;  // P overlays K, Q and 16 KB more
   static bool configured = false;
   static int resident = 0;  // CTAs the persistent form keeps in flight: two per SM
   if (!configured) {
