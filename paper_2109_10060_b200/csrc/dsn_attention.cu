@@ -17,7 +17,7 @@
 //   used as loaded (its rows >= N are cleared: they belong to the next sample);
 //   S = Q K^T: tcgen05.mma M = 128, N = keys rounded to 16, K = 64, fp32 in TMEM;
 //   two threads share one query row (warps w and w + 4 own the same TMEM lanes and half of the keys
-//   each): a first pass over their part of the S row, read from TMEM 32 keys at a time, gives the row
+//   each): a first pass over their part of the S row, read from TMEM 16 keys at a time into two alternating register blocks, gives the row
 //   maximum; a second pass the exponentials, the row sum and P as bf16 in a swizzled K-major
 //   shared-memory tile that reuses the space of K and Q (keys >= N: zeros);
 //   O = P V: tcgen05.mma M = 128, N = 64, K = keys rounded to 16, into the TMEM columns S has left;
@@ -71,6 +71,16 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
   d |= (uint64_t)1 << 46;
   d |= (uint64_t)2 << 61;
   return d;
+}
+
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
 }
 
 constexpr int kAttTableGroups = 64;  // groups the persistent form can hold in its shared-memory table
@@ -237,29 +247,40 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
 
     tc_fence_after();
     // ---- pass 1 over this thread's part of the S row: the maximum.  The scores are read from TMEM one
-    // 32-key block at a time and not kept: 104 scores per thread would not fit the register budget of two
+    // 16-key block at a time and not kept: 104 scores per thread would not fit the register budget of two
     // CTAs per SM, and a second read of TMEM (pass 2) is cheaper than spilling them.
     // Keys >= N (next sample's rows, or padding) count as -inf; only the block that straddles N pays for the test.
     float mx = -INFINITY;
+    const int nblk = (cols_per + 15) >> 4;  // blocks of 16 keys; two register blocks alternate (see pass 2)
+    auto max_block = [&](const uint32_t (&v)[16], int c) {
+      const int kb = cbeg + 16 * c;                                  // first key of the block
+      const int nk = cols_per - 16 * c < 16 ? cols_per - 16 * c : 16;  // keys of this part in the block (multiple of 8)
+      if (kb + nk > N) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (i < nk && kb + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
+      } else if (nk == 16) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (i < nk) mx = fmaxf(mx, __uint_as_float(v[i]));
+      }
+    };
     if (rows_live) {
+      uint32_t va[16], vb[16];
+      tmem_ld_32x16(trow + cbeg, va);
+      tmem_ld_wait();
 #pragma unroll 1
-      for (int c = 0; 32 * c < cols_per; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(trow + cbeg + 32 * c, v);
+      for (int c = 0; c < nblk; c += 2) {
+        if (c + 1 < nblk) tmem_ld_32x16(trow + cbeg + 16 * (c + 1), vb);
+        max_block(va, c);
         tmem_ld_wait();
-        const int kb = cbeg + 32 * c;                                  // first key of the block
-        const int nk = cols_per - 32 * c < 32 ? cols_per - 32 * c : 32;  // keys of this part in the block (multiple of 8)
-        if (kb + nk > N) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (i < nk && kb + i < N) mx = fmaxf(mx, __uint_as_float(v[i]));
-        } else if (nk == 32) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (i < nk) mx = fmaxf(mx, __uint_as_float(v[i]));
+        if (c + 1 < nblk) {
+          if (c + 2 < nblk) tmem_ld_32x16(trow + cbeg + 16 * (c + 2), va);
+          max_block(vb, c + 1);
+          tmem_ld_wait();
         }
       }
     }
@@ -272,36 +293,48 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
     // rounded to bf16 into the swizzled P tile (which overlays K and Q: S has been computed, and pass 1 of
     // every thread is over).  Rows of a warp that is not live keep whatever the tile held: a row of P only
     // reaches the same row of O, which is not stored.
-    if (rows_live) {
-#pragma unroll 1
-      for (int c = 0; 32 * c < cols_per; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(trow + cbeg + 32 * c, v);
-        tmem_ld_wait();
-        const int kb = cbeg + 32 * c;
-        if (kb + 32 > N) {
+    // 16 keys at a time, two register blocks alternating: the TMEM load of the next block is in flight
+    // while the exponentials of this one are computed.
+    auto exp_block = [&](uint32_t (&v)[16], int c) {
+      const int kb = cbeg + 16 * c;
+      if (kb + 16 > N) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (kb + i >= N) v[i] = 0xff800000u;  // -inf: probability 0
-        }
+        for (int i = 0; i < 16; ++i)
+          if (kb + i >= N) v[i] = 0xff800000u;  // -inf: probability 0
+      }
 #pragma unroll
-        for (int jv = 0; jv < 4; ++jv) {
-          const int j0 = 32 * c + 8 * jv;       // first of 8 keys, relative to the part
-          if (j0 < cols_per) {
-            uint32_t w[4];
+      for (int jv = 0; jv < 2; ++jv) {
+        const int j0 = 16 * c + 8 * jv;       // first of 8 keys, relative to the part
+        if (j0 < cols_per) {
+          uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float a, b;
-              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e]), sl2, -mxs)));
-              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e + 1]), sl2, -mxs)));
-              sum += a + b;
-              __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
-              w[e] = *reinterpret_cast<uint32_t*>(&hb);
-            }
-            const int key = cbeg + j0;
-            *reinterpret_cast<uint4*>(p_ptr + (key >> 6) * 16384 + m * 128 + ((((key & 63) >> 3) ^ (m & 7)) << 4)) =
-                make_uint4(w[0], w[1], w[2], w[3]);
+          for (int e = 0; e < 4; ++e) {
+            float a, b;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(a) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e]), sl2, -mxs)));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(b) : "f"(fmaf(__uint_as_float(v[8 * jv + 2 * e + 1]), sl2, -mxs)));
+            sum += a + b;
+            __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
+            w[e] = *reinterpret_cast<uint32_t*>(&hb);
           }
+          const int key = cbeg + j0;
+          *reinterpret_cast<uint4*>(p_ptr + (key >> 6) * 16384 + m * 128 + ((((key & 63) >> 3) ^ (m & 7)) << 4)) =
+              make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    };
+    if (rows_live) {
+      uint32_t va[16], vb[16];
+      tmem_ld_32x16(trow + cbeg, va);
+      tmem_ld_wait();
+#pragma unroll 1
+      for (int c = 0; c < nblk; c += 2) {
+        if (c + 1 < nblk) tmem_ld_32x16(trow + cbeg + 16 * (c + 1), vb);
+        exp_block(va, c);
+        tmem_ld_wait();
+        if (c + 1 < nblk) {
+          if (c + 2 < nblk) tmem_ld_32x16(trow + cbeg + 16 * (c + 2), va);
+          exp_block(vb, c + 1);
+          tmem_ld_wait();
         }
       }
     }
