@@ -82,6 +82,35 @@ def test_attention_more_groups_than_the_item_table_holds(dsn, ctx):
         assert np.all(got[i, :, w:] == SENTINEL)
 
 
+def test_attention_full_size_vit_small_sampled(dsn, ctx):
+    """The ViT-S style configuration at its full size (256 samples, 48 paths, grouped order, as the per-layer
+    benchmark launches it): every CTA works several items.  The oracle is evaluated on a spread of samples."""
+    B, N, H, Dh = 256, 197, 6, 64
+    heads = [p_[1] for p_ in wl.vit_small_paths()]
+    T = len(heads)
+    idx = np.asarray(wl.idx_quota_uniform(wl.rng(3, 9), B, T), np.int32)
+    g = np.random.default_rng(77)
+    q, k, v = (wl.to_bf16_values(wl.normal(g, (B, N, H * Dh))) for _ in range(3))
+    r = route_on_gpu(dsn, ctx, idx, T)
+    perm = O.route(idx, T)[2]
+    out = torch.full((B, N, H * Dh), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(N, H, Dh, heads, order=dsn.GROUPED), r,
+                             up_bf16(head_major(q, k, v, H, Dh)[perm]), out)
+    check_status(ctx, dsn)
+    got = np.empty((B, N, H * Dh), np.float32)
+    got[perm] = down(out)
+    sel = np.unique(np.concatenate([[0, 1, B // 2, B - 2, B - 1], g.integers(0, B, size=11)]))
+    ref = O.attention(q[sel], k[sel], v[sel], idx[sel], heads, Dh)
+    for j, i in enumerate(sel):
+        w = heads[idx[i]] * Dh
+        err = np.max(np.abs(got[i, :, :w] - ref[j, :, :w])) / np.max(np.abs(ref[j, :, :w]))
+        assert err <= TOL, (int(i), int(idx[i]), err)
+    for i in range(B):                                    # every sample: written where it has heads, untouched beyond
+        w = heads[idx[i]] * Dh
+        assert np.all(got[i, :, w:] == SENTINEL)
+        assert np.all(got[i, :, :w] != SENTINEL)
+
+
 def test_attention_closed_forms_on_device(dsn, ctx):
     """Zero queries -> every output row is the mean of the values; a dominant key copies its value."""
     B, N, H, Dh = 2, 197, 2, 64
