@@ -24,6 +24,9 @@ namespace {
 
 using namespace dsn_gemm;
 
+// kRes: the layer has skip features (residual add before the activation).  The form without them holds no
+// trace of that code: its registers and code size weighed on every other epilogue variant.
+template <bool kRes>
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const GemmGeom& g = p.g;
@@ -266,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
       const float* brow = p.bias ? p.bias + t.n0 : nullptr;
       const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
-      const __nv_bfloat16* res_row = (p.residual && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
+      const __nv_bfloat16* res_row = (kRes && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
@@ -278,14 +281,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
       uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
       const CUtensorMap* mY = &p.mapY[t.map];
-      const int variant = p.act * 2 + ((brow || sc_row || p.residual) ? 1 : 0);
-      switch (variant) {
-        case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+      if constexpr (kRes) {
+        switch (p.act) {
+          case DSN_ACT_NONE: epilogue_tile<DSN_ACT_NONE, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case DSN_ACT_RELU: epilogue_tile<DSN_ACT_RELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          default: epilogue_tile<DSN_ACT_GELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        }
+      } else {
+        const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
+        switch (variant) {
+          case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -313,11 +324,13 @@ size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int tps, int a_slots, int G,
 }
 
 cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured = 0;
-  if (smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  static size_t configured[2] = {0, 0};
+  const int res = p.residual ? 1 : 0;
+  void (*kernel)(GemmParams) = res ? gemm_bf16_halo_kernel<true> : gemm_bf16_halo_kernel<false>;
+  if (smem_bytes > configured[res]) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) return e;
-    configured = smem_bytes;
+    configured[res] = smem_bytes;
   }
-  return dsn_launch(gemm_bf16_halo_kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
+  return dsn_launch(kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
 }

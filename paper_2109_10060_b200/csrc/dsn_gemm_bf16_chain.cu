@@ -321,7 +321,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       const float* brow = P.bias ? P.bias + t.n0 : nullptr;
       const float* sc_row = P.bn_scale ? P.bn_scale + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
       const float* sh_row = P.bn_scale ? P.bn_shift + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
-      const __nv_bfloat16* res_row = (P.residual && valid) ? P.residual + out_row * P.ldy + t.n0 : nullptr;
+      const __nv_bfloat16* res_row = nullptr;  // layers with skip features do not run chained
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
@@ -335,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * cp.bn_max);
       const CUtensorMap* mY = &P.mapY[t.map];
-      const int variant = any_valid ? P.act * 2 + ((brow || sc_row || P.residual) ? 1 : 0) : -1;
+      const int variant = any_valid ? P.act * 2 + ((brow || sc_row) ? 1 : 0) : -1;
       switch (variant) {
         case -1: break;  // none of this warp's 32 rows belongs to the sample
         case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
@@ -343,7 +343,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
         case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 5: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        default: break;
       }
       tc_fence_before();
       __syncwarp();

@@ -201,7 +201,7 @@ __device__ __forceinline__ float apply_act(float v) {
 // result).  With `contig` the 32 rows are consecutive output rows starting at
 // `base_row` and each chunk leaves as one TMA store (columns clipped by the map); otherwise eight
 // lanes store one 128-byte piece of a row each.
-template <int ACT, bool AFF>
+template <int ACT, bool AFF, bool RES = false>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0, int first, const float* brow,
                                               const float* sc_row, const float* sh_row, const __nv_bfloat16* res_row, uint8_t* stage_w, __nv_bfloat16* yrow, int lane, bool contig,
                                               const CUtensorMap* mapY, int base_row) {
@@ -214,6 +214,18 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       if (c0 + 32 * half < ncols) {  // warp-uniform
+        // the skip features of this row's 32 columns: four 16-byte loads in flight at once, issued ahead of
+        // the TMEM load (a ragged or unaligned piece takes scalar loads)
+        uint4 rres[4];
+        bool rvec = false;
+        if (RES && res_row) {
+          const __nv_bfloat16* rp = res_row + c0 + 32 * half;
+          rvec = c0 + 32 * half + 32 <= ncols && (reinterpret_cast<uintptr_t>(rp) & 15u) == 0;
+          if (rvec) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rres[i] = __ldg(reinterpret_cast<const uint4*>(rp) + i);
+          }
+        }
         uint32_t v[32];
         tmem_ld_32x32(taddr + c0 + 32 * half, v);
         tmem_ld_wait();
@@ -221,6 +233,8 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj) {
           uint32_t w[4];
+          const uint4 rv = rvec ? rres[jj] : make_uint4(0u, 0u, 0u, 0u);
+          const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int c = 8 * jj + 2 * e;
@@ -229,12 +243,14 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
               if (cb + c < ncols) {
                 if (brow) a += __ldg(brow + cb + c);
                 if (sc_row) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
-                if (res_row) a += __bfloat162float(res_row[cb + c]);
+                if (RES && rvec) a += __uint_as_float(rw[e] << 16);
+                else if (RES && res_row) a += __bfloat162float(res_row[cb + c]);
               }
               if (cb + c + 1 < ncols) {
                 if (brow) b += __ldg(brow + cb + c + 1);
                 if (sc_row) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
-                if (res_row) b += __bfloat162float(res_row[cb + c + 1]);
+                if (RES && rvec) b += __uint_as_float(rw[e] & 0xffff0000u);
+                else if (RES && res_row) b += __bfloat162float(res_row[cb + c + 1]);
               }
             }
             __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
