@@ -125,6 +125,10 @@ __device__ __forceinline__ void chain_walk(const DsnChainParams& cp, const int32
   }
 }
 
+// kAff: some layer of the block has a bias or a per-path affine; kGelu: some layer ends in GELU.  A form
+// without one of them holds none of that code: the kernel is sensitive to its own size (each of the two cuts
+// took about 1 us off the bottleneck step).
+template <bool kAff, bool kGelu>
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __grid_constant__ DsnChainParams cp) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -318,9 +322,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
         out_row = (int64_t)smp * g.R + yy * g.W + xx;
       }
       __nv_bfloat16* yrow = valid ? P.y + out_row * P.ldy + t.n0 : nullptr;
-      const float* brow = P.bias ? P.bias + t.n0 : nullptr;
-      const float* sc_row = P.bn_scale ? P.bn_scale + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
-      const float* sh_row = P.bn_scale ? P.bn_shift + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
+      const float* brow = (kAff && P.bias) ? P.bias + t.n0 : nullptr;
+      const float* sc_row = (kAff && P.bn_scale) ? P.bn_scale + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
+      const float* sh_row = (kAff && P.bn_scale) ? P.bn_shift + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
       const __nv_bfloat16* res_row = nullptr;  // layers with skip features do not run chained
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
@@ -339,11 +343,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       switch (variant) {
         case -1: break;  // none of this warp's 32 rows belongs to the sample
         case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 1: if constexpr (kAff) epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-        case 5: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 3: if constexpr (kAff) epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 4: if constexpr (kGelu) epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 5: if constexpr (kAff && kGelu) epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         default: break;
       }
       tc_fence_before();
@@ -375,11 +379,19 @@ size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured = 0;
-  if (smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-    if (e != cudaSuccess) return e;
-    configured = smem_bytes;
+  static size_t configured[4] = {0, 0, 0, 0};
+  int aff = 0, gelu = 0;
+  for (int l = 0; l < cp.n_layers; ++l) {
+    aff |= (cp.L[l].bias || cp.L[l].bn_scale) ? 1 : 0;
+    gelu |= cp.L[l].act == DSN_ACT_GELU ? 1 : 0;
   }
-  return dsn_launch(gemm_bf16_chain_kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, cp);
+  void (*kernel)(DsnChainParams) = aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
+                                       : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
+  const int form = 2 * aff + gelu;
+  if (smem_bytes > configured[form]) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) return e;
+    configured[form] = smem_bytes;
+  }
+  return dsn_launch(kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, cp);
 }
