@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
-CHAIN_CFG2_DRAM_BYTES = 68.8e6   # per launch of gemm_bf16_chain_kernel on cfg2, B = 128 (57.7 MB read + 11.1 MB written)
+CHAIN_CFG2_DRAM_BYTES = 68.5e6   # per launch of gemm_bf16_chain_kernel on cfg2, B = 128 (57.6 MB read + 10.9 MB written)
 
 
 def load_peaks():
