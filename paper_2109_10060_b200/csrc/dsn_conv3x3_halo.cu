@@ -26,7 +26,9 @@ using namespace dsn_gemm;
 
 // kRes: the layer has skip features (residual add before the activation).  The form without them holds no
 // trace of that code: its registers and code size weighed on every other epilogue variant.
-template <bool kRes>
+// kLean (only without kRes): no bias, no per-path affine, no GELU: the epilogue holds the plain and the ReLU
+// variant only.
+template <bool kRes, bool kLean>
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const GemmGeom& g = p.g;
@@ -291,11 +293,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
         const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
         switch (variant) {
           case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 1: epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 1: if constexpr (!kLean) epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
           case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 3: epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 4: epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          default: epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 3: if constexpr (!kLean) epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 4: if constexpr (!kLean) epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          default: if constexpr (!kLean) epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         }
       }
       tc_fence_before();
@@ -324,13 +326,15 @@ size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int tps, int a_slots, int G,
 }
 
 cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[2] = {0, 0};
-  const int res = p.residual ? 1 : 0;
-  void (*kernel)(GemmParams) = res ? gemm_bf16_halo_kernel<true> : gemm_bf16_halo_kernel<false>;
-  if (smem_bytes > configured[res]) {
+  static size_t configured[3] = {0, 0, 0};
+  const bool lean = !p.residual && !p.bias && !p.bn_scale && p.act != DSN_ACT_GELU;
+  const int form = p.residual ? 2 : (lean ? 1 : 0);
+  void (*kernel)(GemmParams) = form == 2 ? gemm_bf16_halo_kernel<true, false>
+                               : form == 1 ? gemm_bf16_halo_kernel<false, true> : gemm_bf16_halo_kernel<false, false>;
+  if (smem_bytes > configured[form]) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) return e;
-    configured[res] = smem_bytes;
+    configured[form] = smem_bytes;
   }
   return dsn_launch(kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
 }
