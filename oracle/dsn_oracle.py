@@ -333,6 +333,22 @@ def attention(q, k, v, idx, heads, D_h, samples=None, fill=np.nan):
     return out
 
 
+def vit_attention_half(x, Wq, Wk, Wv, Wproj, idx, paths, D_h, mirror_bf16=True, samples=None):
+    """Attention half of a slimmable ViT block (Sec. 3.4): Q, K, V from the sliced projections, the h heads of
+    the sample's path through Softmax(Q K^T / sqrt(D_h)) V, concatenated, then W_proj[:d_e, :h*D_h].
+    With mirror_bf16 the three stored tensors (QKV, attention output, projection output) are rounded to
+    bfloat16 where a device that stores bfloat16 activations would round.  Returns (q, k, v, a, out);
+    out holds NaN beyond the sample's d_e columns, a holds zeros beyond its heads."""
+    heads = [p[1] for p in paths]
+    q, k, v = vit_qkv(x, Wq, Wk, Wv, idx, paths, D_h, samples=samples)
+    q, k, v = (_store(np.nan_to_num(t), mirror_bf16) for t in (q, k, v))
+    a = _store(attention(q, k, v, idx, heads, D_h, samples=samples, fill=0.0), mirror_bf16)
+    k_in = [p[1] * D_h for p in paths]
+    k_out = [p[0] for p in paths]
+    out = _store(sliced_linear(a, Wproj, idx, k_in, k_out, samples=samples), mirror_bf16)
+    return q, k, v, a, out
+
+
 def vit_mlp(x, Wfc1, Wfc2, idx, paths, mirror_bf16=True, samples=None):
     """W2[:d_e, :d_mlp] GELU(W1[:d_mlp, :d_e] X) (Eq. slimmableMLP).  Returns (hidden, out)."""
     de = [p[0] for p in paths]

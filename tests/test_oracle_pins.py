@@ -459,6 +459,33 @@ def test_vit_pieces_against_library():
         np.testing.assert_allclose(out[i, :, :de], orf.numpy(), rtol=1e-11, atol=1e-12)
 
 
+def test_vit_attention_half_against_library_composition():
+    """Sliced QKV -> h heads of softmax attention -> sliced projection, against torch's own
+    scaled_dot_product_attention and matmul on hand-sliced tensors (unrounded), and the mirrored form
+    within bf16 error of it."""
+    B, N, De, H, Dh = 3, 6, 16, 4, 4
+    paths = [(8, 2, 16), (16, 4, 32), (12, 3, 24)]
+    x = rand(B, N, De)
+    Wq, Wk, Wv, Wp = rand(H * Dh, De) / 3, rand(H * Dh, De) / 3, rand(H * Dh, De) / 3, rand(De, H * Dh) / 3
+    idx = np.array([1, 2, 0])
+    q, k, v, a, out = O.vit_attention_half(x, Wq, Wk, Wv, Wp, idx, paths, Dh, mirror_bf16=False)
+    for i in range(B):
+        de, h, _ = paths[idx[i]]
+        xi = torch.from_numpy(x[i, :, :de].copy())
+        qt, kt, vt = ((xi @ torch.from_numpy(Wm[:h * Dh, :de].copy()).T).reshape(N, h, Dh).permute(1, 0, 2)
+                      for Wm in (Wq, Wk, Wv))
+        at = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt).permute(1, 0, 2).reshape(N, h * Dh)
+        ref = at @ torch.from_numpy(Wp[:de, :h * Dh].copy()).T
+        np.testing.assert_allclose(a[i, :, :h * Dh], at.numpy(), rtol=1e-10, atol=1e-12)
+        assert np.all(a[i, :, h * Dh:] == 0)
+        np.testing.assert_allclose(out[i, :, :de], ref.numpy(), rtol=1e-10, atol=1e-12)
+        assert np.all(np.isnan(out[i, :, de:]))
+    m = O.vit_attention_half(x, Wq, Wk, Wv, Wp, idx, paths, Dh, mirror_bf16=True)[4]
+    ok = ~np.isnan(out)
+    np.testing.assert_array_equal(O.round_bf16(m[ok]), m[ok])
+    assert np.max(np.abs(m[ok] - out[ok])) / np.max(np.abs(out[ok])) < 4 * 2.0 ** -8
+
+
 def test_attention_library_brute_force_and_closed_forms():
     B, N, H, Dh = 3, 7, 4, 5
     q, k, v = rand(B, N, H * Dh), rand(B, N, H * Dh), rand(B, N, H * Dh)
