@@ -2,20 +2,28 @@
 """Benchmark of the dynamic-weight-slicing hot path on B200.
 
 A step is one pass of the whole path over one batch of synthetic input: gate (average pool,
-FC-ReLU-FC, arg-max) -> routing (stable grouping) -> the block's sliced grouped GEMMs -> outputs in
-input order.  Default workload: ResNet-50 stage-3 dynamic bottleneck, bf16 NHWC, batch 128, 14x14,
-1x1 1024->w, 3x3 w->w, 1x1 w->1024 with 14 inner widths, gate-driven routing.
+FC-ReLU-FC, arg-max) -> routing (stable grouping) -> the block's sliced grouped GEMMs (and, for a
+ViT block, the attention core between QKV and the projection) -> outputs in input order.
+
+Default workload (--workload cfg5): serving-scale ViT-B-width dynamic block, bf16, 1024 samples x 197
+tokens, embed 768, 12 heads, MLP 3072, 8 diagonal paths, quota-uniform routing: gate, then
+dsn_layer_forward(QKV -> attention -> proj), then dsn_layer_forward(fc1-GELU -> fc2) on the same
+routing.  Other workloads: cfg2, cfg3, cfg4-stage{1..4}[-uniform], M (DS-MBNet depthwise + pointwise).
 
 Prints ONE JSON line (see --help).  `value` is executed TFLOP/s of the whole step (2 x multiply-adds
-of the sliced layers actually run, divided by the step time, gate and routing included), inputs
+of the contractions actually run, divided by the step time, gate and routing included), inputs
 resident in HBM.  `e2e` is the same metric with the batch starting and ending in pinned host memory.
-`roofline` describes the grouped-GEMM kernel, `cpu_baseline` the fp64 CPU oracle on a bounded sample.
+`roofline` describes the dominant grouped-GEMM launch, `cpu_baseline` the fp64 CPU oracle on a bounded
+sample, `per_config` holds the per-layer rows of every configuration.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
+import re
 import subprocess
 import sys
 import threading
@@ -30,7 +38,7 @@ if ROOT not in sys.path:
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
-CHAIN_CFG2_DRAM_BYTES = 68.5e6   # per launch of gemm_bf16_chain_kernel on cfg2, B = 128 (57.6 MB read + 10.9 MB written)
+MIN_TIMED_SECONDS = 0.2           # the timed region lasts at least this long whatever --steps says
 
 
 def load_peaks():
@@ -97,8 +105,129 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+# --------------------------------------------------------------------------------------------- helpers
+def kernel_source_digest(files):
+    """sha256 over the named kernel sources (relative to the package's csrc folder)."""
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2109_10060_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel, workload):
+    """DRAM bytes per launch from an ncu summary under profiles/, or None.  A summary carries a line
+    `bench-traffic: kernel=<k> workload=<w> bytes=<n> sources=<a.cu,b.cuh> sha256=<digest>`; the figure is
+    used only while the digest of those sources is unchanged (a changed kernel invalidates its counters)."""
+    pdir = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(pdir):
+        return None
+    for name in sorted(os.listdir(pdir)):
+        try:
+            text = open(os.path.join(pdir, name)).read()
+        except OSError:
+            continue
+        for m in re.finditer(r"bench-traffic: kernel=(\S+) workload=(\S+) bytes=(\d+) sources=(\S+) sha256=(\w+)", text):
+            if m.group(1) == kernel and m.group(2) == workload:
+                try:
+                    if kernel_source_digest(m.group(4).split(",")) == m.group(5):
+                        return int(m.group(3))
+                except OSError:
+                    pass
+    return None
+
+
+class GraphTimer:
+    """Times a sequence of API calls on the device: one CUDA graph holding `nbuf` calls (one per rotating
+    buffer set), replayed until the timed region is long enough; CUDA events on the replaying stream."""
+
+    def __init__(self, torch, use_graph=True):
+        self.torch = torch
+        self.use_graph = use_graph
+        self.side = torch.cuda.Stream()
+
+    def time_us(self, call, nbuf, min_seconds=0.05, max_replays=4000):
+        t = self.torch
+        with t.cuda.stream(self.side):
+            call(0)
+        t.cuda.synchronize()
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        if not self.use_graph:   # direct calls: one untimed pass over the buffers, then timed passes
+            with t.cuda.stream(self.side):
+                for i in range(nbuf):
+                    call(i)
+                e0.record(self.side)
+                for i in range(2 * nbuf):
+                    call(i)
+                e1.record(self.side)
+            t.cuda.synchronize()
+            return e0.elapsed_time(e1) / (2 * nbuf) * 1e3
+        g = t.cuda.CUDAGraph()
+        with t.cuda.graph(g, stream=self.side):
+            for i in range(nbuf):
+                call(i)
+        cur = t.cuda.current_stream()
+        for _ in range(3):
+            g.replay()
+        e0.record(cur)
+        g.replay()
+        e1.record(cur)
+        t.cuda.synchronize()
+        once = max(e0.elapsed_time(e1) * 1e-3, 1e-6)
+        reps = int(min(max_replays, max(3, math.ceil(min_seconds / once))))
+        e0.record(cur)
+        for _ in range(reps):
+            g.replay()
+        e1.record(cur)
+        t.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * nbuf) * 1e3
+
+
+def gemm_algorithmic_bytes(counts, R, k_in, k_out, K=1):
+    """Sliced input read once, sliced output written once, every used weight slice read once (bf16)."""
+    return sum(2 * (int(n) * R * (k_in[t] + k_out[t]) + k_in[t] * k_out[t] * K * K) for t, n in enumerate(counts) if n)
+
+
 # --------------------------------------------------------------------------------------------- workloads
-class Bottleneck:
+class Workload:
+    """What the timing code needs from a workload."""
+    gate_driven = False
+
+    def x_buffers(self):
+        return self.xs
+
+    def y_buffers(self):
+        return self.ys
+
+    def e2e_io(self):
+        t = self.torch
+        hx = t.from_numpy(self.x_host_bits.copy()).pin_memory()
+        hy = t.empty(self.ys[0].numel(), dtype=t.int16).pin_memory()
+        return hx, hy
+
+    def e2e_pipeline(self, ctx, hx, hy, n, streams, events):
+        """n steps with the batch starting and ending in pinned host memory: the upload of step i+1, the
+        compute of step i and the download of step i-1 run on three streams over the rotating buffer sets."""
+        t = self.torch
+        s_up, s_run, s_down = streams
+        for i in range(n):
+            k = i % len(events)
+            up_done, run_done, down_done = events[k]
+            with t.cuda.stream(s_up):
+                s_up.wait_event(down_done)          # buffer set k is free again
+                self.xs[k].view(t.int16).view(-1).copy_(hx.view(-1), non_blocking=True)
+                up_done.record(s_up)
+            with t.cuda.stream(s_run):
+                s_run.wait_event(up_done)
+                self.step(ctx, k)
+                run_done.record(s_run)
+            with t.cuda.stream(s_down):
+                s_down.wait_event(run_done)
+                hy.copy_(self.ys[k].view(t.int16).view(-1), non_blocking=True)
+                down_done.record(s_down)
+
+
+class Bottleneck(Workload):
     """ResNet-50-style dynamic bottleneck (configs 2 and 4)."""
 
     def __init__(self, dsn, torch, dev, cfg, gate_driven=True, copies=None):
@@ -118,7 +247,8 @@ class Bottleneck:
         self.W2 = up(np.transpose(cfg["W2"], (0, 2, 3, 1)))
         self.W3 = up(cfg["W3"].reshape(C, Ci))
         full = [C] * T
-        self.slices = [(full, self.widths, 1), (self.widths, self.widths, 3), (self.widths, full, 1)]
+        self.slices = [("conv1_1x1", full, self.widths, 1), ("conv2_3x3", self.widths, self.widths, 3),
+                       ("conv3_1x1", self.widths, full, 1)]
         mk = dsn.make_conv_desc
         self.layers = [mk(dsn.BF16, H, Wd, 1, 0, C, Ci, full, self.widths, self.W1, act=dsn.ACT_RELU),
                        mk(dsn.BF16, H, Wd, 3, 1, Ci, Ci, self.widths, self.widths, self.W2, act=dsn.ACT_RELU),
@@ -128,6 +258,7 @@ class Bottleneck:
         self.gate = dsn.make_gate_desc(dsn.BF16, B, self.R, C, self.gW1.shape[0], T, self.gW1, self.gW2)
         self.idx_given = torch.from_numpy(cfg["idx"]).to(dev)
         self.L = dsn.make_layer_desc(B, T, self.layers, self.gate if gate_driven else None)
+        self.L_given = dsn.make_layer_desc(B, T, self.layers, None)
         self.ws = torch.empty(dsn.dsn_layer_workspace_bytes(self.L), dtype=torch.uint8, device=dev)
         self.idx_out = torch.zeros(B, dtype=torch.int32, device=dev)
         # decomposed form (same kernels, one C call per step of the path) for per-kernel timing
@@ -142,147 +273,370 @@ class Bottleneck:
             mk(dsn.BF16, H, Wd, 1, 0, Ci, C, self.widths, full, self.W3, in_order=1, out_order=0)]
         # small batches run the three layers as one chained launch (every CTA pair owns whole samples)
         self.chained = os.environ.get("DSN_CHAIN", "1") != "0" and B <= 148 and 150 <= self.R <= 256
-        self.L_given = dsn.make_layer_desc(B, T, self.layers, None)
         # launches per step: gate = pool + hidden + score, route, then one chained launch or three GEMMs
         self.kernels_per_step = (3 if gate_driven else 0) + 1 + (1 if self.chained else 3)
         self.name = cfg["name"]
+        self.path = "gate -> route -> 1x1 -> 3x3 -> 1x1 -> input order (one dsn_layer_forward call)"
+        self.routing_name = "gate-driven" if gate_driven else cfg["routing"]
+        self.flops_note = "2 x multiply-adds of the three sliced convolutions at the routing histogram"
 
     def step(self, ctx, i):
         k = i % self.copies
         self.dsn.dsn_layer_forward(ctx, self.L, self.xs[k], None if self.gate_driven else self.idx_given, self.ys[k],
-                                   self.ws, idx_out=self.idx_out)
-
-    def _parts(self):
-        d = self.dsn
-        parts = []
-        if self.gate_driven:
-            parts.append(("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)))
-            parts.append(("route", lambda ctx, k: d.dsn_route(ctx, self.idx_out, self.B, self.T, self.routing)))
-        else:
-            parts.append(("route", lambda ctx, k: d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)))
-        if self.chained:
-            # the step's own GEMM launch cannot be called without its routing: timed together with the route
-            # kernel (dsn_layer_forward on given indices); the three single-layer calls below are reference points
-            src = self.idx_out if self.gate_driven else self.idx_given
-            parts.append(("route+gemm_chain", lambda ctx, k: d.dsn_layer_forward(ctx, self.L_given, self.xs[k], src, self.ys[k], self.ws)))
-        parts.append(("gemm:conv1_1x1", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[0], self.routing, self.xs[k], self.t1)))
-        parts.append(("gemm:conv2_3x3", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[1], self.routing, self.t1, self.t2)))
-        parts.append(("gemm:conv3_1x1", lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[2], self.routing, self.t2, self.ys[k])))
-        return parts
-
-    def decomposed_step(self, ctx, i, mark):
-        """Same path as separate C calls; mark(name) is called after each."""
-        k = i % self.copies
-        mark("start")
-        for name, fn in self._parts():
-            fn(ctx, k)
-            mark(name)
-
-    def decomposed_part(self, ctx, i, part):
-        self._parts()[part][1](ctx, i % self.copies)
+                                   self.ws, idx_out=self.idx_out if self.gate_driven else None)
 
     def histogram(self):
         return np.bincount(self.idx_out.cpu().numpy() if self.gate_driven else self.cfg["idx"], minlength=self.T)
 
+    def parts(self, counts):
+        """(name, call(ctx, k), flops, algorithmic bytes, kind) of every step of the path as its own C call."""
+        d, c = self.dsn, counts.tolist()
+        src = self.idx_out if self.gate_driven else self.idx_given
+        out = []
+        if self.gate_driven:
+            out.append(("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws),
+                        0, 2 * self.B * self.R * self.C, "hbm"))
+        out.append(("route", lambda ctx, k: d.dsn_route(ctx, src, self.B, self.T, self.routing), 0, 20 * self.B, "latency"))
+        fl = [2 * d.dsn_executed_macs(c, self.R, ki, ko, K) for _, ki, ko, K in self.slices]
+        by = [gemm_algorithmic_bytes(c, self.R, ki, ko, K) for _, ki, ko, K in self.slices]
+        if self.chained:
+            # the step's own launch: route + the chained GEMM launch on given indices (one API call)
+            out.append(("route+gemm_chain", lambda ctx, k: d.dsn_layer_forward(ctx, self.L_given, self.xs[k], src, self.ys[k], self.ws),
+                        sum(fl), sum(by), "chain"))
+        calls = [lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[0], self.routing, self.xs[k], self.t1),
+                 lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[1], self.routing, self.t1, self.t2),
+                 lambda ctx, k: d.dsn_sliced_conv(ctx, self.dec_layers[2], self.routing, self.t2, self.ys[k])]
+        for (lname, _, _, _), call, f, b in zip(self.slices, calls, fl, by):
+            out.append(("gemm:" + lname, call, f, b, "gemm"))
+        return out
+
     def exec_flops(self, counts):
-        return sum(2 * self.dsn.dsn_executed_macs(counts.tolist(), self.R, ki, ko, K) for ki, ko, K in self.slices)
+        return sum(2 * self.dsn.dsn_executed_macs(counts.tolist(), self.R, ki, ko, K) for _, ki, ko, K in self.slices)
 
-    def gemm_bytes(self, counts):
-        """Algorithmic bytes of the three GEMM launches: sliced input read once, sliced output written
-        once, each used weight slice read once (bf16)."""
-        total = 0
-        for ki, ko, K in self.slices:
-            for t, n in enumerate(counts):
-                if n:
-                    total += 2 * (int(n) * self.R * (ki[t] + ko[t]) + ki[t] * ko[t] * K * K)
-        return total
-
-    def e2e_io(self):
-        t = self.torch
-        hx = t.from_numpy(self.x_host_bits.copy()).pin_memory()
-        hy = t.empty(self.ys[0].numel(), dtype=t.int16).pin_memory()
-        return hx, hy
-
-    def e2e_step(self, ctx, hx, hy):
-        t = self.torch
-        self.xs[0].view(t.int16).view(-1).copy_(hx.view(-1), non_blocking=True)
-        self.step(ctx, 0)
-        hy.copy_(self.ys[0].view(t.int16).view(-1), non_blocking=True)
-
-    def e2e_pipeline(self, ctx, hx, hy, n, streams, events):
-        """n steps with the batch starting and ending in pinned host memory: the upload of step i+1, the
-        compute of step i and the download of step i-1 run on three streams over the rotating buffer sets."""
-        t = self.torch
-        s_up, s_run, s_down = streams
-        for i in range(n):
-            k = i % self.copies
-            up_done, run_done, down_done = events[k]
-            with t.cuda.stream(s_up):
-                s_up.wait_event(down_done)          # buffer set k is free again
-                self.xs[k].view(t.int16).view(-1).copy_(hx.view(-1), non_blocking=True)
-                up_done.record(s_up)
-            with t.cuda.stream(s_run):
-                s_run.wait_event(up_done)
-                self.step(ctx, k)
-                run_done.record(s_run)
-            with t.cuda.stream(s_down):
-                s_down.wait_event(run_done)
-                hy.copy_(self.ys[k].view(t.int16).view(-1), non_blocking=True)
-                down_done.record(s_down)
-
-    def oracle_sample(self, n):
-        """Times the fp64 oracle on the first n samples (gate + bottleneck chain)."""
+    def oracle_run(self, samples, idx_given=None):
+        """Runs the fp64 oracle on the given samples (gate + route + bottleneck chain); returns executed flops."""
         from oracle import dsn_oracle as O
         cfg = self.cfg
-        x = cfg["x"][:n]
-        t0 = time.perf_counter()
-        idx, _, _ = O.gate(x.reshape(n, self.R, self.C), cfg["gate_W1"], cfg["gate_W2"])
+        x = cfg["x"][samples]
+        idx, _, _ = O.gate(x.reshape(len(samples), self.R, self.C), cfg["gate_W1"], cfg["gate_W2"])
         if not self.gate_driven:
-            idx = cfg["idx"][:n]
+            idx = cfg["idx"][samples]
         O.route(idx, self.T)
         O.bottleneck(x, cfg["W1"], cfg["W2"], cfg["W3"], idx, self.widths, mirror_bf16=True)
-        dt = time.perf_counter() - t0
-        flops = sum(2 * O.executed_macs(idx, self.R, ki, ko, K) for ki, ko, K in self.slices)
-        return flops, dt
+        return sum(2 * O.executed_macs(idx, self.R, ki, ko, K) for _, ki, ko, K in self.slices)
+
+    def oracle_samples(self, n, offset=0):
+        return [(offset * n + j) % self.B for j in range(n)]
+
+    oracle_what = "gate + route + bottleneck chain, fp64 numpy (threaded BLAS)"
 
 
-def make_workload(name, dsn, torch, dev, batch=None):
+class ViTBlock(Workload):
+    """DS-ViT-style dynamic transformer block (configs 3 and 5): gate on the mean token, then one
+    dsn_layer_forward call whose five elements inherit one routing: QKV -> attention core -> proj ->
+    fc1(GELU) -> fc2.  routing = "gate" lets the gate's own choice route the batch;
+    any other name routes by the given seeded draw (the gate still runs and its choice is recorded)."""
+
+    def __init__(self, dsn, torch, dev, cfg, routing, copies=None):
+        import dsn_workloads as wl
+        self.dsn, self.torch, self.dev, self.cfg = dsn, torch, dev, cfg
+        B, R, De, H, Dh, Dm, T, paths = (cfg["B"], cfg["R"], cfg["D_e"], cfg["H"], cfg["D_h"], cfg["D_mlp"], cfg["T"],
+                                         cfg["paths"])
+        self.B, self.R, self.De, self.H, self.Dh, self.Dm, self.T, self.paths = B, R, De, H, Dh, Dm, T, paths
+        self.gate_driven = routing == "gate"
+        self.heads = [p[1] for p in paths]
+        up = lambda a: torch.from_numpy(wl.bf16_bits(np.ascontiguousarray(a)).view(np.int16)).to(dev).view(torch.bfloat16).reshape(a.shape)
+        self.x_host_bits = wl.bf16_bits(cfg["x"]).view(np.int16)
+        x_bytes = self.x_host_bits.nbytes
+        # the block input alone is larger than L2 for the serving-scale config; smaller batches rotate buffer sets
+        self.copies = copies or max(2, -(-2 * L2_BYTES // (2 * x_bytes)) + 1)   # two sets at least: the host pipeline overlaps them
+        self.xs = [torch.from_numpy(self.x_host_bits).to(dev).view(torch.bfloat16).reshape(B, R, De) for _ in range(self.copies)]
+        self.ys = [torch.zeros(B, R, De, dtype=torch.bfloat16, device=dev) for _ in range(self.copies)]
+        self.Wqkv = up(wl.pack_qkv_head_major(cfg["Wq"], cfg["Wk"], cfg["Wv"], Dh))
+        self.Wproj, self.Wfc1, self.Wfc2 = up(cfg["Wproj"]), up(cfg["Wfc1"]), up(cfg["Wfc2"])
+        sl = {n: wl.vit_layer_slices(paths, Dh, n) for n in ("qkv", "proj", "fc1", "fc2")}
+        self.sl = sl
+        ml, ma = dsn.make_linear_desc, dsn.make_attention_desc
+        HD = H * Dh
+        self.att_layers = [ml(dsn.BF16, R, De, 3 * HD, *sl["qkv"], self.Wqkv), ma(R, H, Dh, self.heads),
+                           ml(dsn.BF16, R, HD, De, *sl["proj"], self.Wproj)]
+        self.mlp_layers = [ml(dsn.BF16, R, De, Dm, *sl["fc1"], self.Wfc1, act=dsn.ACT_GELU),
+                           ml(dsn.BF16, R, Dm, De, *sl["fc2"], self.Wfc2)]
+        self.gW1 = torch.from_numpy(cfg["gate_W1"]).to(dev)
+        self.gW2 = torch.from_numpy(cfg["gate_W2"]).to(dev)
+        self.gate = dsn.make_gate_desc(dsn.BF16, B, R, De, self.gW1.shape[0], T, self.gW1, self.gW2)
+        self.L = dsn.make_layer_desc(B, T, self.att_layers + self.mlp_layers, self.gate if self.gate_driven else None)
+        self.ws = torch.empty(dsn.dsn_layer_workspace_bytes(self.L), dtype=torch.uint8, device=dev)
+        self.gate_ws = torch.empty(dsn.dsn_gate_workspace_bytes(self.gate), dtype=torch.uint8, device=dev)
+        self.idx_given = torch.from_numpy(np.ascontiguousarray(cfg["idx"], dtype=np.int32)).to(dev)
+        self.idx_out = torch.zeros(B, dtype=torch.int32, device=dev)
+        # decomposed form for per-kernel timing: the same kernels, one C call each, on buffers of their own
+        ints = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+        self.routing = dsn.make_routing(B, T, ints(T), ints(T + 1), ints(B), ints(B))
+        self.t_qkv = torch.zeros(B, R, 3 * HD, dtype=torch.bfloat16, device=dev)
+        self.t_att = torch.zeros(B, R, HD, dtype=torch.bfloat16, device=dev)
+        self.t_h = torch.zeros(B, R, De, dtype=torch.bfloat16, device=dev)
+        self.t_hid = torch.zeros(B, R, Dm, dtype=torch.bfloat16, device=dev)
+        G, I = dsn.GROUPED, dsn.INPUT_ORDER
+        self.dec = {
+            "qkv": ml(dsn.BF16, R, De, 3 * HD, *sl["qkv"], self.Wqkv, in_order=I, out_order=G),
+            "attention": ma(R, H, Dh, self.heads, order=G),
+            "proj": ml(dsn.BF16, R, HD, De, *sl["proj"], self.Wproj, in_order=G, out_order=G),
+            "fc1": ml(dsn.BF16, R, De, Dm, *sl["fc1"], self.Wfc1, act=dsn.ACT_GELU, in_order=G, out_order=G),
+            "fc2": ml(dsn.BF16, R, Dm, De, *sl["fc2"], self.Wfc2, in_order=G, out_order=I)}
+        # launches per step: gate (pool, hidden, scores), route, five layers
+        self.kernels_per_step = 3 + 1 + 5
+        self.name = cfg["name"]
+        self.routing_name = "gate-driven" if self.gate_driven else cfg["routing"]
+        self.path = ("gate -> route -> QKV -> attention core -> proj -> fc1(GELU) -> fc2 -> input order: "
+                     + ("one dsn_layer_forward call, all five elements under the gate's one decision" if self.gate_driven
+                        else "dsn_gate, then one dsn_layer_forward call on the given routing (all five elements under one decision)"))
+        self.flops_note = ("2 x multiply-adds of QKV, proj, fc1, fc2 at the routing histogram + 4 N^2 D_h per executed "
+                           "head for the attention core (QK^T and PV)")
+
+    def step(self, ctx, i):
+        k, d = i % self.copies, self.dsn
+        if self.gate_driven:
+            d.dsn_layer_forward(ctx, self.L, self.xs[k], None, self.ys[k], self.ws, idx_out=self.idx_out)
+        else:
+            d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)
+            d.dsn_layer_forward(ctx, self.L, self.xs[k], self.idx_given, self.ys[k], self.ws)
+
+    def histogram(self):
+        return np.bincount(self.idx_out.cpu().numpy() if self.gate_driven else self.cfg["idx"], minlength=self.T)
+
+    def attention_flops(self, counts):
+        return sum(4.0 * self.R * self.R * self.Dh * self.heads[t] * int(n) for t, n in enumerate(counts))
+
+    def parts(self, counts):
+        d, c = self.dsn, counts.tolist()
+        src = self.idx_out if self.gate_driven else self.idx_given
+        fl = {n: 2 * d.dsn_executed_macs(c, self.R, *self.sl[n], 1) for n in self.sl}
+        by = {n: gemm_algorithmic_bytes(c, self.R, *self.sl[n]) for n in self.sl}
+        att_bytes = sum(2.0 * self.R * 4 * self.Dh * self.heads[t] * int(n) for t, n in enumerate(c))
+        r = self.routing
+        return [
+            ("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws), 0,
+             2 * self.B * self.R * self.De, "hbm"),
+            ("route", lambda ctx, k: d.dsn_route(ctx, src, self.B, self.T, r), 0, 20 * self.B, "latency"),
+            ("gemm:qkv", lambda ctx, k: d.dsn_sliced_linear(ctx, self.dec["qkv"], r, self.xs[k], self.t_qkv), fl["qkv"], by["qkv"], "gemm"),
+            ("attention", lambda ctx, k: d.dsn_sliced_attention(ctx, self.dec["attention"], r, self.t_qkv, self.t_att),
+             self.attention_flops(c), att_bytes, "attention"),
+            ("gemm:proj", lambda ctx, k: d.dsn_sliced_linear(ctx, self.dec["proj"], r, self.t_att, self.t_h), fl["proj"], by["proj"], "gemm"),
+            ("gemm:fc1", lambda ctx, k: d.dsn_sliced_linear(ctx, self.dec["fc1"], r, self.t_h, self.t_hid), fl["fc1"], by["fc1"], "gemm"),
+            ("gemm:fc2", lambda ctx, k: d.dsn_sliced_linear(ctx, self.dec["fc2"], r, self.t_hid, self.ys[k]), fl["fc2"], by["fc2"], "gemm"),
+        ]
+
+    def exec_flops(self, counts):
+        c = counts.tolist()
+        return sum(2 * self.dsn.dsn_executed_macs(c, self.R, *self.sl[n], 1) for n in self.sl) + self.attention_flops(c)
+
+    def oracle_run(self, samples, idx_given=None):
+        from oracle import dsn_oracle as O
+        cfg = self.cfg
+        x = cfg["x"][samples]
+        idx, _, _ = O.gate(x, cfg["gate_W1"], cfg["gate_W2"])
+        if not self.gate_driven:
+            idx = np.asarray(cfg["idx"])[samples]
+        O.route(idx, self.T)
+        h = O.vit_attention_half(x, cfg["Wq"], cfg["Wk"], cfg["Wv"], cfg["Wproj"], idx, self.paths, self.Dh)[4]
+        O.vit_mlp(np.nan_to_num(h), cfg["Wfc1"], cfg["Wfc2"], idx, self.paths, mirror_bf16=True)
+        counts = np.bincount(idx, minlength=self.T)
+        return (sum(2 * O.executed_macs(idx, self.R, *self.sl[n]) for n in self.sl) + self.attention_flops(counts))
+
+    def oracle_samples(self, n, offset=0):
+        """n samples spread over the paths in use (one per path first)."""
+        idx = np.asarray(self.cfg["idx"])
+        order = np.argsort(idx, kind="stable")
+        firsts = [int(order[np.searchsorted(idx[order], t)]) for t in np.unique(idx)]
+        pick = [(firsts[j % len(firsts)] + offset * 7 + (j // len(firsts)) * 13) % self.B for j in range(n)]
+        return pick
+
+    oracle_what = "gate + route + QKV + attention + proj + fc1(GELU) + fc2, fp64 numpy (threaded BLAS)"
+
+
+class MobileNetBlock(Workload):
+    """DS-MBNet separable block (supplementary workload): gate, route, slice-able depthwise 3x3 on the c_t
+    leading channels (ReLU), pointwise 1x1 c_t -> c_t (ReLU), outputs in input order."""
+
+    def __init__(self, dsn, torch, dev, cfg, copies=None):
+        import dsn_workloads as wl
+        self.dsn, self.torch, self.dev, self.cfg = dsn, torch, dev, cfg
+        B, H, Wd, C, K, T = cfg["B"], cfg["H"], cfg["W"], cfg["C"], cfg["K"], cfg["T"]
+        self._host(cfg)
+        up = lambda a: torch.from_numpy(wl.bf16_bits(np.ascontiguousarray(a)).view(np.int16)).to(dev).view(torch.bfloat16).reshape(a.shape)
+        self.x_host_bits = wl.bf16_bits(cfg["x"]).view(np.int16)
+        self.copies = copies or -(-2 * L2_BYTES // (2 * self.x_host_bits.nbytes)) + 1
+        self.xs = [torch.from_numpy(self.x_host_bits).to(dev).view(torch.bfloat16).reshape(B, H, Wd, C) for _ in range(self.copies)]
+        self.ys = [torch.zeros(B, H, Wd, C, dtype=torch.bfloat16, device=dev) for _ in range(self.copies)]
+        self.Wdw = up(np.transpose(cfg["Wdw"], (1, 2, 0)))
+        self.Wpw = up(cfg["Wpw"].reshape(C, C))
+        w = self.widths
+        self.dw = dsn.make_depthwise_desc(H, Wd, K, 1, C, w, [K] * T, self.Wdw, act=dsn.ACT_RELU,
+                                          in_order=dsn.INPUT_ORDER, out_order=dsn.GROUPED)
+        self.pw = dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, C, w, w, self.Wpw, act=dsn.ACT_RELU,
+                                     in_order=dsn.GROUPED, out_order=dsn.INPUT_ORDER)
+        self.gW1 = torch.from_numpy(cfg["gate_W1"]).to(dev)
+        self.gW2 = torch.from_numpy(cfg["gate_W2"]).to(dev)
+        self.gate = dsn.make_gate_desc(dsn.BF16, B, self.R, C, self.gW1.shape[0], T, self.gW1, self.gW2)
+        self.gate_ws = torch.empty(dsn.dsn_gate_workspace_bytes(self.gate), dtype=torch.uint8, device=dev)
+        self.idx_given = torch.from_numpy(np.ascontiguousarray(cfg["idx"], dtype=np.int32)).to(dev)
+        self.idx_out = torch.zeros(B, dtype=torch.int32, device=dev)
+        ints = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+        self.routing = dsn.make_routing(B, T, ints(T), ints(T + 1), ints(B), ints(B))
+        self.t_dw = torch.zeros(B, H, Wd, C, dtype=torch.bfloat16, device=dev)
+        self.kernels_per_step = 3 + 1 + 2
+        self.name = cfg["name"]
+        self.routing_name = cfg["routing"]
+        self.path = "gate -> route -> depthwise 3x3 (ReLU) -> pointwise 1x1 (ReLU) -> input order"
+        self.flops_note = "2 x multiply-adds of the depthwise (9 c_t per pixel) and pointwise (c_t^2 per pixel) layers"
+
+    def _host(self, cfg):
+        self.cfg = cfg
+        self.B, self.R, self.C, self.K, self.T, self.widths = cfg["B"], cfg["H"] * cfg["W"], cfg["C"], cfg["K"], cfg["T"], cfg["widths"]
+
+    @classmethod
+    def host_only(cls, cfg):
+        w = cls.__new__(cls)
+        w._host(cfg)
+        return w
+
+    def step(self, ctx, i):
+        k, d = i % self.copies, self.dsn
+        d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)
+        d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)
+        d.dsn_sliced_depthwise(ctx, self.dw, self.routing, self.xs[k], self.t_dw)
+        d.dsn_sliced_conv(ctx, self.pw, self.routing, self.t_dw, self.ys[k])
+
+    def histogram(self):
+        return np.bincount(self.cfg["idx"], minlength=self.T)
+
+    def _flops(self, counts):
+        dw = sum(2.0 * self.R * self.K * self.K * self.widths[t] * int(n) for t, n in enumerate(counts))
+        pw = sum(2.0 * self.R * self.widths[t] ** 2 * int(n) for t, n in enumerate(counts))
+        return dw, pw
+
+    def parts(self, counts):
+        d, c, r, w = self.dsn, counts.tolist(), self.routing, self.widths
+        dwf, pwf = self._flops(c)
+        dw_bytes = sum(2.0 * 2 * self.R * w[t] * int(n) for t, n in enumerate(c))
+        return [
+            ("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws), 0,
+             2 * self.B * self.R * self.C, "hbm"),
+            ("route", lambda ctx, k: d.dsn_route(ctx, self.idx_given, self.B, self.T, r), 0, 20 * self.B, "latency"),
+            ("depthwise", lambda ctx, k: d.dsn_sliced_depthwise(ctx, self.dw, r, self.xs[k], self.t_dw), dwf, dw_bytes, "hbm"),
+            ("gemm:pointwise", lambda ctx, k: d.dsn_sliced_conv(ctx, self.pw, r, self.t_dw, self.ys[k]), pwf,
+             gemm_algorithmic_bytes(c, self.R, w, w), "gemm"),
+        ]
+
+    def exec_flops(self, counts):
+        return sum(self._flops(counts.tolist()))
+
+    def oracle_run(self, samples, idx_given=None):
+        from oracle import dsn_oracle as O
+        cfg = self.cfg
+        x = cfg["x"][samples]
+        O.gate(x.reshape(len(samples), self.R, self.C), cfg["gate_W1"], cfg["gate_W2"])
+        idx = np.asarray(cfg["idx"])[samples]
+        O.route(idx, self.T)
+        t = O.round_bf16(O.sliced_depthwise(x, cfg["Wdw"], idx, self.widths, [self.K] * self.T, act=O.ACT_RELU, fill=0.0))
+        O.round_bf16(O.sliced_conv(t, cfg["Wpw"], idx, self.widths, self.widths, 0, act=O.ACT_RELU))
+        return sum(self._flops(np.bincount(idx, minlength=self.T).tolist()))
+
+    def oracle_samples(self, n, offset=0):
+        return [(offset * n + j) % self.B for j in range(n)]
+
+    oracle_what = "gate + route + depthwise 3x3 + pointwise 1x1, fp64 numpy"
+
+
+WORKLOADS = ("cfg2", "cfg3", "cfg4-stage1", "cfg4-stage2", "cfg4-stage3", "cfg4-stage4", "cfg4-stage1-uniform",
+             "cfg4-stage2-uniform", "cfg4-stage3-uniform", "cfg4-stage4-uniform", "cfg5", "M")
+
+
+def make_workload(name, dsn, torch, dev, batch=None, routing=None):
     import dsn_workloads as wl
+    vit_routing = {"uniform": dict(routing="uniform"), "zipf": dict(routing="zipf"), "gate": dict(routing="uniform"),
+                   "one0": dict(routing="one", one_path=0), "one7": dict(routing="one", one_path=7)}
     if name == "cfg2":
-        return Bottleneck(dsn, torch, dev, wl.config2(B=batch or 128), gate_driven=True)
+        return Bottleneck(dsn, torch, dev, wl.config2(B=batch or 128), gate_driven=routing in (None, "gate"))
     if name.startswith("cfg4-stage"):
         stage = int(name[len("cfg4-stage")])
-        routing = "uniform" if name.endswith("uniform") else "skewed"
-        return Bottleneck(dsn, torch, dev, wl.config4(stage, B=batch or 256, routing=routing), gate_driven=False)
-    raise SystemExit(f"unknown workload {name}")
+        r = "uniform" if name.endswith("uniform") else "skewed"
+        return Bottleneck(dsn, torch, dev, wl.config4(stage, B=batch or 256, routing=r), gate_driven=False)
+    if name in ("cfg3", "cfg5"):
+        r = routing or "uniform"
+        if r not in vit_routing:
+            raise SystemExit(f"unknown routing {r} for {name}")
+        kw = dict(vit_routing[r])
+        if name == "cfg3":
+            kw.pop("one_path", None)
+            cfg = wl.config3(B=batch or 256, routing=kw["routing"])
+        else:
+            cfg = wl.config5(B=batch or 1024, **kw)
+        return ViTBlock(dsn, torch, dev, cfg, routing=r)
+    if name == "M":
+        return MobileNetBlock(dsn, torch, dev, wl.mobilenet_block(B=batch or 256))
+    raise SystemExit(f"unknown workload {name}; choose from {', '.join(WORKLOADS)}")
+
+
+def workload_title(name):
+    return {"cfg2": "cfg2 ResNet-50 stage-3 dynamic bottleneck, bf16 NHWC, 14x14, 1024->w->w->1024, 14 inner widths",
+            "cfg3": "cfg3 DS-ViT-style block, bf16, 197 tokens, embed 384, 6 heads, MLP 1536, 48 paths",
+            "cfg5": "cfg5 serving-scale ViT-B-width dynamic block, bf16, 197 tokens, embed 768, 12 heads, MLP 3072, 8 diagonal paths",
+            "M": "M DS-MBNet separable block, bf16 NHWC, 14x14, depthwise 3x3 + pointwise 1x1, 14 widths 224..640"}.get(
+                name, f"{name} ResNet-50 dynamic bottleneck of that stage, bf16 NHWC, 14 inner widths")
 
 
 # --------------------------------------------------------------------------------------------- reference arm
+class _HostOnly:
+    """Stands in for the torch / library handles when only a workload's host-side data is wanted."""
+    def __getattr__(self, name):
+        raise RuntimeError("the reference arm runs on the host only")
+
+
+def host_workload(name, batch, routing):
+    """The workload object without any device allocation: only what oracle_run / oracle_samples use."""
+    import dsn_workloads as wl
+    if name == "cfg2" or name.startswith("cfg4-stage"):
+        if name == "cfg2":
+            cfg, gd = wl.config2(B=batch or 128), routing in (None, "gate")
+        else:
+            cfg, gd = wl.config4(int(name[len("cfg4-stage")]), B=batch or 256,
+                                 routing="uniform" if name.endswith("uniform") else "skewed"), False
+        w = Bottleneck.__new__(Bottleneck)
+        C, T = cfg["C_outer"], cfg["T"]
+        w.cfg, w.B, w.R, w.C, w.T, w.widths, w.gate_driven = cfg, cfg["B"], cfg["H"] * cfg["W"], C, T, cfg["widths"], gd
+        w.slices = [("conv1_1x1", [C] * T, w.widths, 1), ("conv2_3x3", w.widths, w.widths, 3), ("conv3_1x1", w.widths, [C] * T, 1)]
+        return w
+    if name in ("cfg3", "cfg5"):
+        r = routing or "uniform"
+        kind = {"uniform": "uniform", "zipf": "zipf", "gate": "uniform", "one0": "one", "one7": "one"}[r]
+        cfg = (wl.config3(B=batch or 256, routing=kind) if name == "cfg3"
+               else wl.config5(B=batch or 1024, routing=kind, one_path=0 if r == "one0" else 7))
+        w = ViTBlock.__new__(ViTBlock)
+        w.cfg, w.B, w.R, w.Dh, w.T, w.paths = cfg, cfg["B"], cfg["R"], cfg["D_h"], cfg["T"], cfg["paths"]
+        w.heads = [p[1] for p in w.paths]
+        w.gate_driven = r == "gate"
+        w.sl = {n: wl.vit_layer_slices(w.paths, w.Dh, n) for n in ("qkv", "proj", "fc1", "fc2")}
+        return w
+    if name == "M":
+        return MobileNetBlock.host_only(wl.mobilenet_block(B=batch or 256))
+    raise SystemExit(f"unknown workload {name}")
+
+
 def run_reference(args):
-    """Times the CPU oracle (the only 'reference implementation' this method has) on host cores."""
+    """Times the CPU oracle (the only 'reference implementation' this method has) on host cores: every
+    step is a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import dsn_workloads as wl
-    from oracle import dsn_oracle as O
-    cfg = wl.config2(B=128)
-    n = 8
-    R, C, T, widths = cfg["H"] * cfg["W"], cfg["C_outer"], cfg["T"], cfg["widths"]
-    full = [C] * T
-    slices = [(full, widths, 1), (widths, widths, 3), (widths, full, 1)]
-
-    def one(i):
-        x = cfg["x"][(i * n) % 128:(i * n) % 128 + n]
-        idx, _, _ = O.gate(x.reshape(n, R, C), cfg["gate_W1"], cfg["gate_W2"])
-        O.route(idx, T)
-        O.bottleneck(x, cfg["W1"], cfg["W2"], cfg["W3"], idx, widths, mirror_bf16=True)
-        return sum(2 * O.executed_macs(idx, R, ki, ko, K) for ki, ko, K in slices)
-
-    for i in range(args.warmup):
-        one(i)
+    w = host_workload(args.workload, args.batch, args.routing)
+    n = {"cfg5": 8, "cfg3": 16}.get(args.workload, 8)
+    for i in range(min(args.warmup, 3)):
+        w.oracle_run(w.oracle_samples(n, i))
     flops, t0 = 0, time.perf_counter()
     for i in range(args.steps):
-        flops += one(i)
+        flops += w.oracle_run(w.oracle_samples(n, i))
     dt = time.perf_counter() - t0
     val = flops / dt / 1e12
     cores = os.cpu_count()
@@ -290,67 +644,43 @@ def run_reference(args):
         "impl": "reference", "metric": "sliced_gemm_executed_tflops", "value": val, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "cfg2 ResNet-50 stage-3 dynamic bottleneck, bf16-valued inputs, 14x14, 14 widths",
-                   "sample": f"{n} samples per step"},
+        "config": {"workload": workload_title(args.workload), "batch": w.B,
+                   "routing": "gate-driven" if w.gate_driven else w.cfg["routing"],
+                   "sample": f"{n} of {w.B} samples per step"},
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
-                         "sample": f"{n} of 128 samples per step, {args.steps} steps"},
+                         "sample": f"{n} of {w.B} samples per step, {args.steps} steps; {w.oracle_what}"},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-
-# --------------------------------------------------------------------------------------------- per-layer table
-def run_table(args):
-    """Per-layer numbers for every configuration (markdown table rows): CUDA-graph replay over
-    rotating buffers larger than L2, executed TFLOP/s, fraction of the shape's roofline bound."""
-    import torch
-    from paper_2109_10060_b200.build import build
-    build()
-    import paper_2109_10060_b200 as dsn
+# --------------------------------------------------------------------------------------------- per-layer rows
+def collect_rows(dsn, torch, ctx, dev, peaks, timer, row_filter=None, batch_div=1, emit=None):
+    """Per-layer numbers for every configuration: CUDA-graph replay over rotating buffers larger than L2,
+    executed TFLOP/s and fraction of the shape's roofline bound min(measured BF16 peak, intensity x measured
+    HBM bandwidth).  Returns a list of dict rows; `emit(row)` is called as each row is measured."""
     import dsn_workloads as wl
-    from oracle import dsn_oracle as O
-    dev = torch.device("cuda:0")
-    ctx = dsn.Context(0)
-    peaks = load_peaks()
     PEAK, HBM = peaks["bf16_tflops"], peaks["hbm_gbs"]
     ints = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
-    side = torch.cuda.Stream()
+    want = (lambda *names: re.search(row_filter, " ".join(names)) is not None) if row_filter else (lambda *names: True)
+    div = max(1, batch_div)
+    rows = []
 
-    def graph_time(call, nbuf, reps=10):
-        with torch.cuda.stream(side):
-            call(0)
-        torch.cuda.synchronize()
-        if args.no_graph:   # direct calls (for profilers): two passes over the buffers, the second one timed
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            with torch.cuda.stream(side):
-                for i in range(nbuf):
-                    call(i)
-                e0.record(side)
-                for i in range(nbuf):
-                    call(i)
-                e1.record(side)
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / nbuf * 1e3
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=side):
-            for i in range(nbuf):
-                call(i)
-        g.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
-            g.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / (reps * nbuf) * 1e3  # us
+    def add(row):
+        rows.append(row)
+        if emit:
+            emit(row)
 
-    print("| config | layer | routing | us | executed TFLOP/s | % measured BF16 peak | bound (TFLOP/s) | % of bound | GB/s | samples/s |")
-    print("|---|---|---|---|---|---|---|---|---|---|")
+    def gemm_row(cfgname, lname, rname, B, us, flops, byts):
+        tf = flops / us / 1e6
+        bound = min(PEAK, flops / byts * HBM / 1e3)
+        add({"config": cfgname, "layer": lname, "routing": rname, "us": round(us, 1), "tflops": round(tf, 1),
+             "pct_bf16_peak": round(100 * tf / PEAK, 1), "bound_tflops": round(bound), "pct_of_bound": round(100 * tf / bound),
+             "gbs": round(byts / us / 1e3), "samples_per_s": round(B / us * 1e6)})
 
-    import re
-    want = (lambda *names: re.search(args.table_filter, " ".join(names)) is not None) if args.table_filter else (lambda *names: True)
-    div = max(1, args.table_batch_div)
+    def routed(B, T, idx):
+        r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
+        dsn.dsn_route(ctx, ints(idx), B, T, r)
+        return r
 
     def layer(cfgname, lname, rname, B, H, Cin, Cout, k_in, k_out, idx, K=1, act=0, orders=(1, 1), group_list=None):
         if not want(cfgname, lname, rname):
@@ -362,11 +692,7 @@ def run_table(args):
             idx = idx[:B]
         T = len(k_in)
         R = H * H if K == 3 else H
-        if group_list is None:
-            r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
-            dsn.dsn_route(ctx, ints(idx), B, T, r)
-        else:
-            r = group_list
+        r = routed(B, T, idx) if group_list is None else group_list
         per = B * R * (Cin + Cout) * 2
         nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
         xs = [torch.randn(B, R, Cin, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
@@ -380,16 +706,12 @@ def run_table(args):
             d = dsn.make_conv_desc(dsn.BF16, H, H, K, 1, Cin, Cout, k_in, k_out, W, act=act, in_order=orders[0],
                                    out_order=orders[1])
             call = lambda i: dsn.dsn_sliced_conv(ctx, d, r, xs[i % nbuf], ys[i % nbuf])
-        us = graph_time(call, nbuf)
+        us = timer.time_us(call, nbuf)
         code, _ = ctx.get_status()
         assert code == 0, code
         counts = np.bincount(idx, minlength=T)
         flops = 2 * dsn.dsn_executed_macs(counts.tolist(), R, k_in, k_out, K)
-        byts = sum(2 * (int(n) * R * (k_in[t] + k_out[t]) + k_in[t] * k_out[t] * K * K) for t, n in enumerate(counts) if n)
-        tf = flops / us / 1e6
-        bound = min(PEAK, flops / byts * HBM / 1e3)
-        print(f"| {cfgname} | {lname} | {rname} | {us:.1f} | {tf:.0f} | {100 * tf / PEAK:.1f} | {bound:.0f} | "
-              f"{100 * tf / bound:.0f} | {byts / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
+        gemm_row(cfgname, lname, rname, B, us, flops, gemm_algorithmic_bytes(counts, R, k_in, k_out, K))
         del xs, ys
 
     def gate_route(cfgname, B, R, C, T):
@@ -405,13 +727,31 @@ def run_table(args):
         ws = torch.empty(dsn.dsn_gate_workspace_bytes(g), dtype=torch.uint8, device=dev)
         idx = torch.zeros(B, dtype=torch.int32, device=dev)
         r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
-        us = graph_time(lambda i: dsn.dsn_gate(ctx, g, xs[i % nbuf], idx, None, ws), nbuf)
-        print(f"| {cfgname} | gate (pool + FC-ReLU-FC + arg-max) | - | {us:.1f} | - | - | HBM {HBM:.0f} GB/s | "
-              f"{100 * per / us / 1e3 / HBM:.0f} | {per / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
-        us = graph_time(lambda i: dsn.dsn_route(ctx, idx, B, T, r), 8)
-        print(f"| {cfgname} | route | - | {us:.1f} | - | - | launch latency | - | - | {B / us * 1e6:.0f} |", flush=True)
+        us = timer.time_us(lambda i: dsn.dsn_gate(ctx, g, xs[i % nbuf], idx, None, ws), nbuf)
+        add({"config": cfgname, "layer": "gate (pool + FC-ReLU-FC + arg-max)", "routing": "-", "us": round(us, 1),
+             "bound": f"HBM {HBM:.0f} GB/s", "pct_of_bound": round(100 * per / us / 1e3 / HBM), "gbs": round(per / us / 1e3),
+             "samples_per_s": round(B / us * 1e6)})
+        us = timer.time_us(lambda i: dsn.dsn_route(ctx, idx, B, T, r), 8)
+        add({"config": cfgname, "layer": "route", "routing": "-", "us": round(us, 1), "bound": "launch latency",
+             "samples_per_s": round(B / us * 1e6)})
 
-    # config 2 / 4: bottlenecks
+    def attention(cfgname, B, N, H, heads, idx, rname):
+        if not want(cfgname, "attention core", rname):
+            return
+        B = B // div
+        idx = idx[:B]
+        r = routed(B, len(heads), idx)
+        per = B * N * 4 * H * 64 * 2
+        nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
+        qs = [torch.randn(B, N, 3 * H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        os_ = [torch.zeros(B, N, H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
+        d = dsn.make_attention_desc(N, H, 64, heads, order=dsn.GROUPED)
+        us = timer.time_us(lambda i: dsn.dsn_sliced_attention(ctx, d, r, qs[i % nbuf], os_[i % nbuf]), nbuf)
+        assert ctx.get_status()[0] == 0
+        hsum = sum(heads[t] for t in idx)
+        gemm_row(cfgname, f"attention core (N={N})", rname, B, us, 4.0 * N * N * 64 * hsum, 2.0 * N * 4 * 64 * hsum)
+
+    # configs 2 / 4: bottlenecks
     for cfgname, B, stages in (("cfg2", 128, (3,)), ("cfg4", 256, (1, 2, 3, 4))):
         for stage in stages:
             hw, outer, inner = wl.RESNET_STAGES[stage]
@@ -433,29 +773,6 @@ def run_table(args):
     for lname, Cin, Cout, act in (("qkv", 384, 1152, 0), ("proj", 384, 384, 0), ("fc1", 384, 1536, 2), ("fc2", 1536, 384, 0)):
         ki, ko = wl.vit_layer_slices(paths, 64, lname)
         layer("cfg3", lname, "uniform", B, 197, Cin, Cout, ki, ko, idx, act=act)
-    def attention(cfgname, B, N, H, heads, idx, rname):
-        if not want(cfgname, "attention core", rname):
-            return
-        B = B // div
-        idx = idx[:B]
-        T = len(heads)
-        r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
-        dsn.dsn_route(ctx, ints(idx), B, T, r)
-        per = B * N * 4 * H * 64 * 2
-        nbuf = max(2, int(2.2 * L2_BYTES // per) + 1)
-        qs = [torch.randn(B, N, 3 * H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
-        os_ = [torch.zeros(B, N, H * 64, device=dev, dtype=torch.bfloat16) for _ in range(nbuf)]
-        d = dsn.make_attention_desc(N, H, 64, heads, order=dsn.GROUPED)
-        us = graph_time(lambda i: dsn.dsn_sliced_attention(ctx, d, r, qs[i % nbuf], os_[i % nbuf]), nbuf)
-        assert ctx.get_status()[0] == 0
-        hsum = sum(heads[t] for t in idx)
-        flops = 4.0 * N * N * 64 * hsum
-        byts = 2.0 * N * 4 * 64 * hsum
-        tf = flops / us / 1e6
-        bound = min(PEAK, flops / byts * HBM / 1e3)
-        print(f"| {cfgname} | attention core (N={N}) | {rname} | {us:.1f} | {tf:.0f} | {100 * tf / PEAK:.1f} | {bound:.0f} | "
-              f"{100 * tf / bound:.0f} | {byts / us / 1e3:.0f} | {B / us * 1e6:.0f} |", flush=True)
-
     attention("cfg3", 256, 197, 6, [p_[1] for p_ in wl.vit_small_paths()], wl.idx_quota_uniform(wl.rng(3, 9), 256, 48), "uniform")
     attention("cfg5", 1024, 197, 12, [p_[1] for p_ in wl.vit_base_paths()], wl.idx_quota_uniform(wl.rng(5, 9), 1024, 8), "uniform")
     # config 5: ViT-B width
@@ -464,7 +781,7 @@ def run_table(args):
     cases = [("all on path 7", wl.idx_all_one(B, 7)), ("all on path 0", wl.idx_all_one(B, 0)),
              ("uniform", wl.idx_quota_uniform(wl.rng(5, 9), B, 8)), ("zipf(1.2)", wl.idx_zipf(wl.rng(5, 9), B, 8))]
     for rname, idx in cases:
-        for lname, Cin, Cout, act in (("qkv", 768, 2304, 0), ("fc1", 768, 3072, 2), ("fc2", 3072, 768, 0)):
+        for lname, Cin, Cout, act in (("qkv", 768, 2304, 0), ("proj", 768, 768, 0), ("fc1", 768, 3072, 2), ("fc2", 3072, 768, 0)):
             ki, ko = wl.vit_layer_slices(paths, 64, lname)
             layer("cfg5", lname, rname, B, 197, Cin, Cout, ki, ko, idx, act=act)
     # singleton groups: 1024 caller-built groups of one sample each
@@ -480,47 +797,80 @@ def run_table(args):
         idx = wl.idx_quota_uniform(wl.rng(6, 6), 256, 14)
         layer(f"M {hw}x{hw}", f"pointwise 1x1 c->c (full {C})", "uniform", 256, hw * hw, C, C, widths, widths, idx, act=1)
     # config 1: fp32 single layer
-    if not want("cfg1", "fp32 linear", "iid"):
-        return
-    c1 = wl.config1()
-    x, W = torch.from_numpy(c1["x"]).to(dev), torch.from_numpy(c1["W"]).to(dev)
-    y = torch.zeros(64, 1, 256, device=dev)
-    r = dsn.make_routing(64, 4, ints(np.zeros(4)), ints(np.zeros(5)), ints(np.zeros(64)), ints(np.zeros(64)))
-    dsn.dsn_route(ctx, ints(c1["idx"]), 64, 4, r)
-    d = dsn.make_linear_desc(dsn.F32, 1, 256, 256, c1["k_in"], c1["k_out"], W)
-    us = graph_time(lambda i: dsn.dsn_sliced_linear(ctx, d, r, x, y), 8)
-    fl = 2 * dsn.dsn_executed_macs(np.bincount(c1["idx"], minlength=4).tolist(), 1, c1["k_in"], c1["k_out"], 1)
-    print(f"| cfg1 | fp32 linear 256x256, B=64 | iid | {us:.1f} | {fl / us / 1e6:.3f} | - | launch latency | - | - | {64 / us * 1e6:.0f} |")
+    if want("cfg1", "fp32 linear", "iid"):
+        c1 = wl.config1()
+        x, W = torch.from_numpy(c1["x"]).to(dev), torch.from_numpy(c1["W"]).to(dev)
+        y = torch.zeros(64, 1, 256, device=dev)
+        r = routed(64, 4, c1["idx"])
+        d = dsn.make_linear_desc(dsn.F32, 1, 256, 256, c1["k_in"], c1["k_out"], W)
+        us = timer.time_us(lambda i: dsn.dsn_sliced_linear(ctx, d, r, x, y), 8)
+        fl = 2 * dsn.dsn_executed_macs(np.bincount(c1["idx"], minlength=4).tolist(), 1, c1["k_in"], c1["k_out"], 1)
+        add({"config": "cfg1", "layer": "fp32 linear 256x256, B=64", "routing": "iid", "us": round(us, 1),
+             "tflops": round(fl / us / 1e6, 3), "bound": "launch latency", "samples_per_s": round(64 / us * 1e6)})
+    return rows
+
+
+TABLE_HEADER = ("| config | layer | routing | us | executed TFLOP/s | % measured BF16 peak | bound (TFLOP/s) | % of bound | GB/s | samples/s |\n"
+                "|---|---|---|---|---|---|---|---|---|---|")
+
+
+def row_markdown(r):
+    g = lambda k: r.get(k, "-")
+    bound = r.get("bound_tflops", r.get("bound", "-"))
+    return (f"| {g('config')} | {g('layer')} | {g('routing')} | {g('us')} | {g('tflops')} | {g('pct_bf16_peak')} | {bound} | "
+            f"{g('pct_of_bound')} | {g('gbs')} | {g('samples_per_s')} |")
+
 
 # --------------------------------------------------------------------------------------------- main arm
+def spawn_ranks(args):
+    """`--gpus N` without a launcher: start N ranks (one process per GPU) and pass their output through."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    argv = [a for a in sys.argv[1:]]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    raise SystemExit(subprocess.call(cmd, env=env))
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="dsn", choices=["dsn", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg5", help="one of " + ", ".join(WORKLOADS))
+    ap.add_argument("--routing", default=None, help="cfg3/cfg5: uniform (default), zipf, one0, one7, gate; cfg2: gate (default) or uniform")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--table", action="store_true", help="print per-layer markdown rows for every configuration")
+    ap.add_argument("--no-per-config", action="store_true", help="leave the per-layer rows of every configuration out of the JSON line")
+    ap.add_argument("--table", action="store_true", help="print the per-layer rows of every configuration as a markdown table and exit")
     ap.add_argument("--no-graph", action="store_true", help="time direct API calls instead of a CUDA-graph replay (for profilers)")
-    ap.add_argument("--table-filter", default=None, help="with --table: only rows whose 'config layer routing' text matches this regular expression")
-    ap.add_argument("--table-batch-div", type=int, default=1, help="with --table: divide every batch size by this (small cases for profilers)")
+    ap.add_argument("--table-filter", default=None, help="per-layer rows: only those whose 'config layer routing' text matches this regular expression")
+    ap.add_argument("--table-batch-div", type=int, default=1, help="per-layer rows: divide every batch size by this (small cases for profilers)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
         return
-    if args.table:
-        run_table(args)
-        return
+    world_env = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world_env == 1:
+        spawn_ranks(args)
+    if world_env > 1 and world_env != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} does not match WORLD_SIZE={world_env}")
 
     import torch
     from paper_2109_10060_b200.build import build
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    world = world_env
+    if not torch.cuda.is_available() or torch.cuda.device_count() <= local_rank:
+        raise SystemExit(f"rank {rank}: no CUDA device {local_rank} (the benchmark has no CPU path)")
+    dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
@@ -533,8 +883,15 @@ def main():
     dev = torch.device(f"cuda:{local_rank}")
     ctx = dsn.Context(local_rank)
     peaks = load_peaks()
+    timer = GraphTimer(torch, use_graph=not args.no_graph)
 
-    wlk = make_workload(args.workload, dsn, torch, dev, args.batch)
+    if args.table:
+        print(TABLE_HEADER)
+        collect_rows(dsn, torch, ctx, dev, peaks, timer, args.table_filter, args.table_batch_div,
+                     emit=lambda r: print(row_markdown(r), flush=True))
+        return
+
+    wlk = make_workload(args.workload, dsn, torch, dev, args.batch, args.routing)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -543,12 +900,17 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    def status_ok():
+        code, detail = ctx.get_status()
+        if code != 0:
+            raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
+
+    t_host0 = time.perf_counter()
     for i in range(args.warmup):
         wlk.step(ctx, i)
+    host_us_per_step = (time.perf_counter() - t_host0) / args.warmup * 1e6   # enqueue time of the API calls (first call included)
     barrier()
-    code, detail = ctx.get_status()
-    if code != 0:
-        raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
+    status_ok()
     counts = wlk.histogram()
 
     # The timed steps replay a CUDA graph that holds one step per rotating buffer set, so that the
@@ -572,68 +934,62 @@ def main():
         sys.stderr.write(f"graph capture unavailable ({exc}); timing direct calls\n")
 
     def run_steps(n):
+        """n steps, n a multiple of the buffer-set count when graphed."""
         if graphed:
             for _ in range(n // wlk.copies):
                 graph.replay()
-            for i in range(n % wlk.copies):
-                wlk.step(ctx, i)
         else:
             for i in range(n):
                 wlk.step(ctx, i)
 
-    run_steps(wlk.copies * 2)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    run_steps(2 * wlk.copies)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    est_ms = max(e0.elapsed_time(e1) / (2 * wlk.copies), 1e-4)
+    # EXACTLY --steps steps are asked for; the timed region is stretched to MIN_TIMED_SECONDS where that
+    # many steps would be shorter (and to a whole number of graph replays); ms_per_step = region / timed_steps
+    timed_steps = max(args.steps, int(math.ceil(MIN_TIMED_SECONDS * 1e3 / est_ms)))
+    timed_steps = -(-timed_steps // wlk.copies) * wlk.copies
+    if world > 1:
+        tmax = torch.tensor([timed_steps], dtype=torch.int64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        timed_steps = int(tmax.item())
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record(stream)
-    run_steps(args.steps)
+    run_steps(timed_steps)
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    status_ok()
+
+    # the same steps as direct API calls (no graph): device time per step and host time to enqueue one
+    direct_n = max(wlk.copies, min(timed_steps, 50))
+    torch.cuda.synchronize()
+    t_host0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(direct_n):
+        wlk.step(ctx, i)
+    e1.record(stream)
+    host_enqueue_us = (time.perf_counter() - t_host0) / direct_n * 1e6
+    torch.cuda.synchronize()
+    direct_ms = e0.elapsed_time(e1) / direct_n
 
     # per-kernel durations: each step of the path (same kernels, one C call each) captured as its own
     # graph over the rotating buffers and replayed back to back
-    acc = {}
-    marks = []
-    wlk.decomposed_step(ctx, 0, lambda n: marks.append(n))
+    parts = wlk.parts(counts)
+    for _, call, _, _, _ in parts:          # consistent routing arrays and intermediates for every part
+        call(ctx, 0)
     torch.cuda.synchronize()
-    part_names = marks[1:]
-    for pi, pname in enumerate(part_names):
-        try:
-            if args.no_graph:
-                raise RuntimeError("disabled by --no-graph")
-            gpart = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gpart, stream=side):
-                for i in range(wlk.copies):
-                    wlk.decomposed_part(ctx, i, pi)
-            gpart.replay()
-            torch.cuda.synchronize()
-            reps = 20
-            e0.record(stream)
-            for _ in range(reps):
-                gpart.replay()
-            e1.record(stream)
-            torch.cuda.synchronize()
-            acc[pname] = [e0.elapsed_time(e1) / (reps * wlk.copies)]
-        except Exception as exc:  # noqa: BLE001
-            sys.stderr.write(f"per-kernel graph for {pname} unavailable ({exc})\n")
-    if not acc:  # no graphs: direct calls with an event after each (includes launch gaps)
-        for i in range(13):
-            evs = []
-            def mark(n):
-                ev = torch.cuda.Event(enable_timing=True)
-                ev.record(stream)
-                evs.append((n, ev))
-            wlk.decomposed_step(ctx, i, mark)
-            torch.cuda.synchronize()
-            if i >= 3:
-                for (n0, a), (n1, b) in zip(evs[:-1], evs[1:]):
-                    acc.setdefault(n1, []).append(a.elapsed_time(b))
-    wlk.decomposed_step(ctx, 0, lambda n: None)   # leave the routing arrays consistent
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
+    part_us = {}
+    for pname, call, _, _, _ in parts:
+        part_us[pname] = timer.time_us(lambda i, c=call: c(ctx, i % wlk.copies), wlk.copies, min_seconds=0.1)
+    status_ok()
 
     # end to end: batch starts and ends in pinned host memory; upload, compute and download overlap
     hx, hy = wlk.e2e_io()
@@ -644,7 +1000,7 @@ def main():
     torch.cuda.synchronize()
     wlk.e2e_pipeline(ctx, hx, hy, 2 * wlk.copies, streams, events)
     barrier()
-    e2e_steps = min(args.steps, 40)
+    e2e_steps = max(2 * wlk.copies, min(args.steps, 40))
     e0.record(stream)
     for st in streams:
         st.wait_event(e0)
@@ -656,67 +1012,93 @@ def main():
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
-    code, detail = ctx.get_status()
-    if code != 0:
-        raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
+    status_ok()
 
     from paper_2109_10060_b200.sharding import max_over_ranks
-    t = max_over_ranks(torch.tensor([ms_total], dtype=torch.float64, device=dev), dist if world > 1 else None)
-    t2 = max_over_ranks(torch.tensor([ms_e2e], dtype=torch.float64, device=dev), dist if world > 1 else None)
-    ms_step = float(t.item()) / args.steps
+    t = max_over_ranks(torch.tensor([ms_total], dtype=torch.float64, device=dev), dist)
+    t2 = max_over_ranks(torch.tensor([ms_e2e], dtype=torch.float64, device=dev), dist)
+    ms_step = float(t.item()) / timed_steps
     ms_e2e = float(t2.item())
     flops = wlk.exec_flops(counts)
     value = world * flops / (ms_step * 1e-3) / 1e12
     e2e_value = world * flops / (ms_e2e * 1e-3) / 1e12
-
-    if "route+gemm_chain" in acc and "route" in acc:
-        gemm_ms = float(np.mean(acc["route+gemm_chain"])) - float(np.mean(acc["route"]))
-        gemm_kernel = "gemm_bf16_chain_kernel (1 launch per step: conv1, conv2 and conv3 of every sample on one CTA pair)"
-    else:
-        gemm_ms = sum(float(np.mean(v)) for k, v in acc.items() if k.startswith("gemm:"))
-        gemm_kernel = "gemm_bf16_pair_kernel (3 launches per step: conv1, conv2, conv3)"
-    gemm_bytes = wlk.gemm_bytes(counts)
-    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
-    per_kernel = {k: round(float(np.mean(v)) * 1e3, 2) for k, v in acc.items()}
-    roofline = {"bound": "hbm", "kernel": gemm_kernel,
-                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "peak_source": peaks["source"] + " copy bandwidth, burst",
-                # dram__bytes_read + dram__bytes_write of one launch of this kernel on this workload (ncu capture
-                # summarised under profiles/; to be re-taken, or set to None, whenever the kernel changes)
-                "traffic": CHAIN_CFG2_DRAM_BYTES if (gemm_kernel.startswith("gemm_bf16_chain") and args.workload == "cfg2"
-                                                     and args.batch in (None, 128)) else None,
-                "algorithmic_bytes_per_step": gemm_bytes, "us_per_step": round(gemm_ms * 1e3, 2),
-                "executed_tflops": flops / (gemm_ms * 1e-3) / 1e12,
-                "frac_of_bf16_peak_burst": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
-
     if rank != 0:
         return
+
+    # roofline of the dominant grouped-GEMM launch
+    info = {p[0]: p for p in parts}
+    gemm_parts = [p for p in parts if p[4] in ("gemm", "chain")]
+    chain = [p for p in gemm_parts if p[4] == "chain"]
+    dom = chain[0] if chain else max((p for p in gemm_parts), key=lambda p: part_us[p[0]])
+    dname, _, dflops, dbytes, dkind = dom
+    dus = part_us[dname]
+    ai = dflops / dbytes
+    ridge = peaks["bf16_tflops"] * 1e3 / peaks["hbm_gbs"]
+    if ai >= ridge:
+        ach, peak, unit, bound = dflops / dus / 1e6, peaks["bf16_tflops"], "TFLOP/s", "tensor"
+        src = peaks["source"] + " cuBLAS bf16 matmul, burst"
+    else:
+        ach, peak, unit, bound = dbytes / dus / 1e3, peaks["hbm_gbs"], "GB/s", "hbm"
+        src = peaks["source"] + " copy bandwidth"
+    kernel = ("gemm_bf16_chain_kernel" if dkind == "chain" else
+              ("gemm_bf16_halo_kernel" if dname.endswith("3x3") and wlk.R > 200 and max(wlk.widths) <= 128 else "gemm_bf16_pair_kernel"))
+    traffic_key = f"{args.workload}:{dname.split(':')[-1]}" + (f":{args.routing}" if args.routing else "")
+    roofline = {"bound": bound, "kernel": kernel, "launch": dname, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                "peak_source": src, "traffic": recorded_traffic(kernel, traffic_key),
+                "algorithmic_bytes_per_launch": dbytes, "flops_per_launch": dflops, "us_per_launch": round(dus, 2),
+                "arithmetic_intensity": round(ai, 1), "ridge": round(ridge, 1),
+                "executed_tflops": dflops / dus / 1e6,
+                "frac_of_bf16_peak_sustained": dflops / dus / 1e6 / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                "timing": ("one API call (route + chained launch) per replay; the route kernel's share is inside the figure"
+                           if dkind == "chain" else "the launch alone in a CUDA graph of its own, replayed for 0.1 s")}
+    gsel = [p for p in gemm_parts if p[4] == "gemm"]
+    g_fl, g_us = sum(p[2] for p in gsel), sum(part_us[p[0]] for p in gsel)
+    gemm_layers = {"layers": [p[0] for p in gsel], "executed_tflops": g_fl / g_us / 1e6, "us": round(g_us, 1),
+                   "frac_of_bf16_peak_burst": g_fl / g_us / 1e6 / peaks["bf16_tflops"],
+                   "frac_of_bf16_peak_sustained": g_fl / g_us / 1e6 / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                   "per_layer": {p[0]: {"us": round(part_us[p[0]], 1), "tflops": round(p[2] / part_us[p[0]] / 1e6, 1),
+                                        "frac_of_bf16_peak_burst": round(p[2] / part_us[p[0]] / 1e6 / peaks["bf16_tflops"], 3)}
+                                 for p in gsel}}
+
     out = {
         "metric": "sliced_gemm_executed_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{wlk.name}: batch {wlk.B} per GPU, gate-driven routing" if wlk.gate_driven
-                   else f"{wlk.name}: batch {wlk.B} per GPU, routing {wlk.cfg['routing']}",
-                   "path": "gate -> route -> 1x1 -> 3x3 -> 1x1 -> input order (dsn_layer_forward)",
-                   "l2": f"inputs and outputs rotate over {wlk.copies} buffers (> 126 MB L2)",
+        "steps": args.steps, "timed_steps": timed_steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_title(args.workload), "name": wlk.name, "batch_per_gpu": wlk.B,
+                   "routing": wlk.routing_name, "path": wlk.path, "flops": wlk.flops_note,
+                   "l2": f"inputs and outputs rotate over {wlk.copies} buffer sets; one set's input is "
+                         f"{wlk.x_host_bits.nbytes / 1e6:.0f} MB (L2 126 MB)",
                    "launch": "CUDA graph replay of the public-API step" if graphed else "direct calls",
+                   "timed_region": f"{timed_steps} steps = max(--steps, {MIN_TIMED_SECONDS} s worth), {ms_total:.1f} ms",
                    "routing_histogram": counts.tolist(), "parallelism": f"batch shards x{world}, no collective"},
         "samples_per_s": world * wlk.B / (ms_step * 1e-3),
         "pct_bf16_peak_burst": 100 * value / world / peaks["bf16_tflops"],
+        "pct_bf16_peak_sustained": 100 * value / world / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
         "pct_bf16_peak_nominal": 100 * value / world / NOMINAL_BF16_TFLOPS,
-        "kernel_us": per_kernel,
+        "direct_calls": {"ms_per_step": direct_ms, "host_enqueue_us_per_step": round(host_enqueue_us, 1),
+                         "host_enqueue_us_per_step_first_calls": round(host_us_per_step, 1),
+                         "note": "the same steps issued as plain API calls without a graph"},
+        "kernel_us": {k: round(v, 2) for k, v in part_us.items()},
         "roofline": roofline,
+        "gemm_layers": gemm_layers,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(hx.numel() * 2),
                 "d2h_bytes_per_step": int(hy.numel() * 2), "ms_per_step": ms_e2e,
-                "how": "dsn_layer_forward per step; upload, compute and download pipelined on three streams"},
-        "gpu_launches": wlk.kernels_per_step * args.steps,
+                "how": "the public-API step per batch; upload, compute and download pipelined on three streams"},
+        "gpu_launches": wlk.kernels_per_step * timed_steps,
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        n = wlk.B
-        f_cpu, dt = wlk.oracle_sample(n)
+        n = {"cfg5": 8, "cfg3": 16}.get(args.workload, min(wlk.B, 128))
+        samples = wlk.oracle_samples(n)
+        t0 = time.perf_counter()
+        f_cpu = wlk.oracle_run(samples)
+        dt = time.perf_counter() - t0
         out["cpu_baseline"] = {"value": f_cpu / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
-                               "sample": f"{n} of {wlk.B} samples, gate + route + bottleneck chain, fp64 numpy (threaded BLAS), {dt:.1f} s wall"}
+                               "sample": f"{n} of {wlk.B} samples; {wlk.oracle_what}; {dt:.1f} s wall"}
+    if not args.no_per_config and world == 1:
+        del wlk
+        torch.cuda.empty_cache()
+        out["per_config"] = collect_rows(dsn, torch, ctx, dev, peaks, timer, args.table_filter, args.table_batch_div)
     print(json.dumps(out))
 
 

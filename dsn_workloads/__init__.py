@@ -266,3 +266,20 @@ def mobilenet_pointwise(B=256, hw=14, C=640):
         Wpw=normal(rng(config, 1 if C == 640 else 11), (C, C, 1, 1), std=C ** -0.5),
         idx=idx_quota_uniform(rng(config, 6), B, len(widths)),
     )
+
+
+def mobilenet_block(B=256, hw=14, C=640, K=3, C_mlp=128):
+    """DS-MBNet separable block (routing-space table of DS-MBNet): depthwise KxK on the c_t leading channels,
+    ReLU, then pointwise 1x1 c_t -> c_t, ReLU.  Depthwise filter in the oracle's [C][K][K] indexing."""
+    config = 6
+    widths = WIDTHS_14[C]
+    T = len(widths)
+    return dict(
+        name=f"mbnet_dwpw_{hw}x{hw}_{C}", dtype="bf16", B=B, H=hw, W=hw, C=C, K=K, T=T, widths=widths,
+        x=normal(rng(config, 20), (B, hw, hw, C), relu=True),
+        Wdw=normal(rng(config, 21), (C, K, K), std=1.0 / K),
+        Wpw=normal(rng(config, 22), (C, C, 1, 1), std=C ** -0.5),
+        gate_W1=normal(rng(config, 24), (C_mlp, C), std=C ** -0.5, bf16=False),
+        gate_W2=normal(rng(config, 25), (T, C_mlp), std=C_mlp ** -0.5, bf16=False),
+        idx=idx_quota_uniform(rng(config, 26), B, T), routing="uniform",
+    )

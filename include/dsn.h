@@ -52,7 +52,7 @@ enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1, DSN_LAYER_ATTENT
 
 #define DSN_MAX_SLICES 64   /* largest T                                               */
 #define DSN_MAX_GROUPS 4096 /* largest G of a caller-built group list                  */
-#define DSN_MAX_CHAIN 4     /* layers per dsn_layer_forward call                       */
+#define DSN_MAX_CHAIN 6     /* layers per dsn_layer_forward call (a ViT block: QKV, attention, proj, fc1, fc2) */
 
 /* Batch grouping (not in the paper, which defines only per-sample behaviour, Eq. (dyn_net):
  * every input runs the path its own gate picks).  Grouped position p holds sample perm[p];
@@ -194,6 +194,16 @@ const char* dsn_strerror(int code);
 /* Waits for `stream`, returns the first device-detected condition since the last call
  * (code = DSN_OK if none; detail = a count or position) and clears it. */
 int dsn_get_status(dsn_ctx* ctx, void* stream, int32_t* code, int32_t* detail);
+
+/* Limit of the bounded waits inside the kernels (every wait on a barrier or counter gives up after this
+ * long, records DSN_ERR_TIMEOUT with a position code and lets the kernel return; the context stays usable).
+ * microseconds = 0 restores the default of 2 s.  Synchronises `stream`.  (Failure detection; the paper has
+ * no counterpart.) */
+int dsn_set_wait_limit(dsn_ctx* ctx, uint32_t microseconds, void* stream);
+/* Self-test of that mechanism: launches one small kernel that waits, with the library's own wait routine,
+ * on a barrier nothing arrives at.  It returns after the wait limit; dsn_get_status() then reports
+ * DSN_ERR_TIMEOUT (detail 9001).  Nothing faults and later calls run normally. */
+int dsn_selftest_bounded_wait(dsn_ctx* ctx, void* stream);
 
 /* Ratio list -> channel counts (host only).  granule g = 0 picks g = min(8, C/32);
  * k = g*floor(r*C/g + 1/2) clamped to [g, C].  The paper lists channel counts, not a rounding

@@ -21,10 +21,10 @@ ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
 INPUT_ORDER, GROUPED = 0, 1
 TAIL_UNTOUCHED, TAIL_ZERO = 0, 1
 LAYER_LINEAR, LAYER_CONV, LAYER_ATTENTION = 0, 1, 2
-MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 4
+MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 6
 
 EXPORTS = [
-    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_widths_from_ratios",
+    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_set_wait_limit", "dsn_selftest_bounded_wait", "dsn_widths_from_ratios",
     "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
     "dsn_sliced_attention", "dsn_sliced_depthwise", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
@@ -101,6 +101,8 @@ def load_library():
     lib.dsn_strerror.argtypes = [C.c_int]
     lib.dsn_strerror.restype = C.c_char_p
     lib.dsn_get_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
+    lib.dsn_set_wait_limit.argtypes = [vp, C.c_uint32, vp]
+    lib.dsn_selftest_bounded_wait.argtypes = [vp, vp]
     lib.dsn_widths_from_ratios.argtypes = [i32, C.POINTER(C.c_double), i32, i32, C.POINTER(i32)]
     lib.dsn_executed_macs.argtypes = [C.POINTER(i32), i32, i32, C.POINTER(i32), C.POINTER(i32), i32]
     lib.dsn_executed_macs.restype = i64
@@ -187,6 +189,14 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def set_wait_limit(self, microseconds: int, stream=None):
+        """Limit of the kernels' bounded waits (0 = the 2 s default)."""
+        _check(self.lib.dsn_set_wait_limit(self.handle, int(microseconds), _stream_handle(stream)), "dsn_set_wait_limit")
+
+    def selftest_bounded_wait(self, stream=None):
+        """Launches the kernel that waits on a barrier nobody arrives at; it returns after the wait limit."""
+        _check(self.lib.dsn_selftest_bounded_wait(self.handle, _stream_handle(stream)), "dsn_selftest_bounded_wait")
 
     def get_status(self, stream=None):
         code, detail = C.c_int32(), C.c_int32()

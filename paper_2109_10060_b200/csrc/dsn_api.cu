@@ -23,6 +23,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Every entry point runs on the context's device: launches, attribute settings and symbol look-ups all act
+// on the calling thread's current device.
+int check_ctx(const dsn_ctx* ctx) {
+  if (!ctx) return DSN_ERR_INVALID_ARG;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) return DSN_ERR_CUDA;
+  return cur == ctx->device ? DSN_OK : DSN_ERR_INVALID_ARG;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
@@ -384,8 +393,9 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
 }
 
 int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
-  if (!ctx) return DSN_ERR_INVALID_ARG;
-  int e = validate_call(c, r, x, y);
+  int e = check_ctx(ctx);
+  if (e) return e;
+  e = validate_call(c, r, x, y);
   if (e) return e;
   if (r->B == 0) return DSN_OK;
   SliceTable st;
@@ -436,6 +446,22 @@ LayerCall from_conv(const dsn_conv_desc* d) {
   return c;
 }
 
+// Host-side checks of an attention element (pointers may be null when only the descriptor is checked).
+int check_attention(const dsn_attention_desc* d, const dsn_routing* r, const void* qkv, const void* out) {
+  if (!d || !d->heads) return DSN_ERR_INVALID_ARG;
+  if (d->dtype != DSN_BF16 || d->D_h != 64 || d->N > 256) return DSN_ERR_UNSUPPORTED;
+  if (d->N < 1 || d->H < 1 || d->H > 64 || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (d->ld_qkv < (int64_t)3 * d->H * d->D_h || d->ld_out < (int64_t)d->H * d->D_h) return DSN_ERR_INVALID_ARG;
+  if (d->order != DSN_INPUT_ORDER && d->order != DSN_GROUPED) return DSN_ERR_INVALID_ARG;
+  for (int t = 0; t < d->T; ++t)
+    if (d->heads[t] < 1 || d->heads[t] > d->H) return DSN_ERR_INVALID_ARG;
+  int e = check_routing(r, d->T);
+  if (e) return e;
+  if ((qkv && !aligned16(qkv)) || (out && !aligned16(out)) || d->ld_qkv % 8 || d->ld_out % 8) return DSN_ERR_ALIGNMENT;
+  if ((int64_t)r->B * d->N > 0x7fffffffLL) return DSN_ERR_INVALID_ARG;
+  return DSN_OK;
+}
+
 int check_gate(const dsn_gate_desc* g) {
   if (!g || !g->W1 || !g->W2) return DSN_ERR_INVALID_ARG;
   if (g->dtype != DSN_BF16 && g->dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
@@ -462,6 +488,7 @@ int layer_call_of(const dsn_layer_desc* L, int j, LayerCall& c) {
     // between two sliced layers only: it reads and writes grouped intermediates
     if (j == 0 || j + 1 == L->n_layers) return DSN_ERR_INVALID_ARG;
     const dsn_attention_desc* a = static_cast<const dsn_attention_desc*>(L->layer[j]);
+    if (!a->heads || a->T < 1 || a->T > DSN_MAX_SLICES || a->D_h < 1 || a->H < 1) return DSN_ERR_INVALID_ARG;
     memset(&c, 0, sizeof(c));
     c.att = a;
     c.dtype = a->dtype;
@@ -491,12 +518,21 @@ int plan_layer(const dsn_layer_desc* L, LayerPlan& pl) {
   if (e) return e;
   pl.elem = first.dtype == DSN_BF16 ? 2 : 4;
   int prev_out = 0, prev_R = 0;
+  int prev_k_out[DSN_MAX_SLICES] = {0};
   for (int j = 0; j < L->n_layers; ++j) {
     LayerCall c;
     e = layer_call_of(L, j, c);
     if (e) return e;
     if (c.T != L->T || c.dtype != first.dtype) return DSN_ERR_INVALID_ARG;
+    if (!c.att && (!c.k_in || !c.k_out)) return DSN_ERR_INVALID_ARG;
     if (j > 0 && (c.C_in != prev_out || c.H * c.W != prev_R)) return DSN_ERR_INVALID_ARG;
+    // every layer of the block inherits the one decision (Sec. 5): a path may read no more columns of an
+    // intermediate than the layer before wrote for that path (the columns beyond hold stale workspace bytes)
+    for (int t = 0; t < L->T; ++t) {
+      const int need_in = c.att ? 3 * c.att->heads[t] * c.att->D_h : c.k_in[t];
+      if (j > 0 && need_in > prev_k_out[t]) return DSN_ERR_INVALID_ARG;
+      prev_k_out[t] = c.att ? c.att->heads[t] * c.att->D_h : c.k_out[t];
+    }
     prev_out = c.C_out;
     prev_R = c.H * c.W;
     if (j + 1 < L->n_layers) {
@@ -578,15 +614,33 @@ int dsn_destroy(dsn_ctx* ctx) {
 }
 
 int dsn_get_status(dsn_ctx* ctx, void* stream, int32_t* code, int32_t* detail) {
-  if (!ctx) return DSN_ERR_INVALID_ARG;
-  int32_t h[DSN_STATUS_WORDS];
+  if (int e = check_ctx(ctx)) return e;
+  int32_t h[DSN_STATUS_REPORT_WORDS];
   cudaStream_t s = as_stream(stream);
   if (cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DSN_ERR_CUDA;
-  if (cudaMemsetAsync(ctx->d_status, 0, sizeof(h), s) != cudaSuccess) return DSN_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->d_status, 0, sizeof(h), s) != cudaSuccess) return DSN_ERR_CUDA;  // the report words only
   if (cudaStreamSynchronize(s) != cudaSuccess) return DSN_ERR_CUDA;
   if (code) *code = h[0];
   if (detail) *detail = h[1];
   return DSN_OK;
+}
+
+int dsn_set_wait_limit(dsn_ctx* ctx, uint32_t microseconds, void* stream) {
+  if (int e = check_ctx(ctx)) return e;
+  cudaStream_t s = as_stream(stream);
+  // the source of an asynchronous copy must stay valid until the copy has run: wait for an earlier one first
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DSN_ERR_CUDA;
+  ctx->wait_limit_us = microseconds;
+  if (cudaMemcpyAsync(ctx->d_status + DSN_STATUS_WAIT_US, &ctx->wait_limit_us, sizeof(uint32_t), cudaMemcpyHostToDevice,
+                      s) != cudaSuccess)
+    return DSN_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_selftest_bounded_wait(dsn_ctx* ctx, void* stream) {
+  if (int e = check_ctx(ctx)) return e;
+  return dsn_launch_selftest_wait(ctx->d_status, as_stream(stream)) == cudaSuccess ? DSN_OK : DSN_ERR_CUDA;
 }
 
 int dsn_widths_from_ratios(int32_t C, const double* ratios, int32_t T, int32_t granule, int32_t* widths_out) {
@@ -624,8 +678,10 @@ size_t dsn_gate_workspace_bytes(const dsn_gate_desc* g) {
 
 int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_out, float* logits_out,
              void* workspace, size_t ws_bytes, void* stream) {
-  if (!ctx || !x || !idx_out) return DSN_ERR_INVALID_ARG;
-  int e = check_gate(g);
+  if (!x || !idx_out) return DSN_ERR_INVALID_ARG;
+  int e = check_ctx(ctx);
+  if (e) return e;
+  e = check_gate(g);
   if (e) return e;
   if (g->B == 0) return DSN_OK;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
@@ -655,8 +711,9 @@ int dsn_gate_attention(dsn_ctx* ctx, const dsn_gate_desc* g, const float* W3, co
 int dsn_scale_channels(dsn_ctx* ctx, const dsn_routing* r, int32_t to_grouped, int32_t dtype, int32_t B, int32_t R,
                        int32_t c_valid, const void* x, int64_t ldx, const float* scale, void* y, int64_t ldy,
                        void* stream) {
-  if (!ctx || !x || !y || !scale || B < 0 || R < 1 || c_valid < 1 || ldx < c_valid || ldy < c_valid)
+  if (!x || !y || !scale || B < 0 || R < 1 || c_valid < 1 || ldx < c_valid || ldy < c_valid)
     return DSN_ERR_INVALID_ARG;
+  if (int e = check_ctx(ctx)) return e;
   if (dtype != DSN_BF16 && dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
   const int32_t* perm = nullptr;
   if (to_grouped) {
@@ -672,15 +729,17 @@ int dsn_scale_channels(dsn_ctx* ctx, const dsn_routing* r, int32_t to_grouped, i
 
 int dsn_resbn_fold(dsn_ctx* ctx, int32_t T, int32_t C, const float* gamma, const float* beta, const float* mu,
                    const float* sigma, float* scale_out, float* shift_out, void* stream) {
-  if (!ctx || T < 1 || T > DSN_MAX_SLICES || C < 1 || !gamma || !beta || !mu || !sigma || !scale_out || !shift_out)
+  if (T < 1 || T > DSN_MAX_SLICES || C < 1 || !gamma || !beta || !mu || !sigma || !scale_out || !shift_out)
     return DSN_ERR_INVALID_ARG;
+  if (int e = check_ctx(ctx)) return e;
   if (dsn_launch_resbn_fold(T * C, C, gamma, beta, mu, sigma, scale_out, shift_out, as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
   return DSN_OK;
 }
 
 int dsn_route(dsn_ctx* ctx, const int32_t* idx, int32_t B, int32_t T, dsn_routing* out, void* stream) {
-  if (!ctx || !idx || !out || B < 0 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (!idx || !out || B < 0 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (int e = check_ctx(ctx)) return e;
   if (!out->counts || !out->offsets || !out->perm || !out->inv_perm) return DSN_ERR_INVALID_ARG;
   out->B = B;
   out->G = T;
@@ -693,9 +752,11 @@ int dsn_route(dsn_ctx* ctx, const int32_t* idx, int32_t B, int32_t T, dsn_routin
 
 int dsn_permute_rows(dsn_ctx* ctx, const dsn_routing* r, int32_t dtype, int32_t R, int32_t T, const int32_t* k,
                      const void* src, int64_t ld_src, void* dst, int64_t ld_dst, int32_t to_grouped, void* stream) {
-  if (!ctx || !src || !dst || !k || R < 1 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (!src || !dst || !k || R < 1 || T < 1 || T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
   if (dtype != DSN_BF16 && dtype != DSN_F32) return DSN_ERR_INVALID_ARG;
-  int e = check_routing(r, T);
+  int e = check_ctx(ctx);
+  if (e) return e;
+  e = check_routing(r, T);
   if (e) return e;
   SliceTable st;
   memset(&st, 0, sizeof(st));
@@ -735,7 +796,8 @@ int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, 
 
 int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_routing* r, const void* x, void* y,
                          void* stream) {
-  if (!ctx || !d || !x || !y || !d->W || !d->c || !d->ksize) return DSN_ERR_INVALID_ARG;
+  if (!d || !x || !y || !d->W || !d->c || !d->ksize) return DSN_ERR_INVALID_ARG;
+  if (int e0 = check_ctx(ctx)) return e0;
   if (d->dtype != DSN_BF16) return DSN_ERR_UNSUPPORTED;
   if (d->H < 1 || d->W_ < 1 || d->C < 1 || d->C > 32767 || d->K < 1 || d->K > 7 || d->K % 2 == 0) return DSN_ERR_INVALID_ARG;
   if (d->stride != 1 && d->stride != 2) return DSN_ERR_UNSUPPORTED;
@@ -756,18 +818,12 @@ int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_ro
 
 int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_routing* r, const void* qkv, void* out,
                          void* stream) {
-  if (!ctx || !d || !qkv || !out || !d->heads) return DSN_ERR_INVALID_ARG;
-  if (d->dtype != DSN_BF16 || d->D_h != 64 || d->N > 256) return DSN_ERR_UNSUPPORTED;
-  if (d->N < 1 || d->H < 1 || d->H > 64 || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
-  if (d->ld_qkv < (int64_t)3 * d->H * d->D_h || d->ld_out < (int64_t)d->H * d->D_h) return DSN_ERR_INVALID_ARG;
-  if (d->order != DSN_INPUT_ORDER && d->order != DSN_GROUPED) return DSN_ERR_INVALID_ARG;
-  for (int t = 0; t < d->T; ++t)
-    if (d->heads[t] < 1 || d->heads[t] > d->H) return DSN_ERR_INVALID_ARG;
-  int e = check_routing(r, d->T);
+  if (!qkv || !out) return DSN_ERR_INVALID_ARG;
+  int e = check_ctx(ctx);
   if (e) return e;
-  if (!aligned16(qkv) || !aligned16(out) || d->ld_qkv % 8 || d->ld_out % 8) return DSN_ERR_ALIGNMENT;
+  e = check_attention(d, r, qkv, out);
+  if (e) return e;
   if (r->B == 0) return DSN_OK;
-  if ((int64_t)r->B * d->N > 0x7fffffffLL) return DSN_ERR_INVALID_ARG;
   CUtensorMap map;
   const uint64_t dims[3] = {64, (uint64_t)3 * d->H, (uint64_t)r->B * d->N};
   const uint64_t str[2] = {128, (uint64_t)d->ld_qkv * 2};
@@ -789,9 +845,11 @@ size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L) {
 
 int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, const int32_t* idx_in, void* y,
                       dsn_routing* r_out, int32_t* idx_out, void* workspace, size_t ws_bytes, void* stream) {
-  if (!ctx || !L || !x || !y) return DSN_ERR_INVALID_ARG;
+  if (!L || !x || !y) return DSN_ERR_INVALID_ARG;
+  int e = check_ctx(ctx);
+  if (e) return e;
   LayerPlan pl;
-  int e = plan_layer(L, pl);
+  e = plan_layer(L, pl);
   if (e) return e;
   if (!L->gate && !idx_in) return DSN_ERR_INVALID_ARG;
   if (L->gate && (L->gate->B != L->B || L->gate->T != L->T)) return DSN_ERR_INVALID_ARG;
@@ -824,8 +882,14 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
     if (!c.att) {
       e = validate_call(c, &r, in, out);
-      if (e) return e;
+    } else {  // the attention core between two layers: dense grouped intermediates
+      dsn_attention_desc a = *c.att;
+      a.ld_qkv = c.C_in;
+      a.ld_out = c.C_out;
+      a.order = DSN_GROUPED;
+      e = check_attention(&a, &r, in, out);
     }
+    if (e) return e;
   }
 
   const int32_t* idx = idx_in;

@@ -418,19 +418,14 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   p.out = static_cast<__nv_bfloat16*>(out); p.ld_out = ld_out;
   p.status = status;
   const size_t smem = 1024 + 3072 + kVBytes + kPBytes;  // P overlays K, Q and 16 KB more
-  static bool configured = false;
-  static int resident = 0;  // CTAs the persistent form keeps in flight: two per SM
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    int dev = 0, sms = 0;
-    if (e == cudaSuccess) e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    resident = 2 * sms;
-    configured = true;
-  }
+  static size_t configured[2][DSN_MAX_DEVICES] = {};
+  cudaError_t e = dsn_ensure_dynamic_smem(attention_kernel<false>, smem, configured[0]);
+  if (e == cudaSuccess) e = dsn_ensure_dynamic_smem(attention_kernel<true>, smem, configured[1]);
+  int dev = 0, sms = 0;
+  if (e == cudaSuccess) e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const int resident = 2 * sms;  // CTAs the persistent form keeps in flight: two per SM
   const int halves = N > 128 ? 2 : 1;
   if (G <= kAttTableGroups) {
     const long long dense = (long long)H * B * halves;

@@ -320,13 +320,12 @@ size_t dsn_gemm_smem_bytes(int BN, int stages, int G) {
 }
 
 cudaError_t dsn_launch_gemm_bf16(const GemmParams& p, int sm_count, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[2] = {0, 0};
+  static size_t configured[2][DSN_MAX_DEVICES] = {};
   const int res = p.residual ? 1 : 0;
   void (*kernel)(GemmParams) = res ? gemm_bf16_kernel<true> : gemm_bf16_kernel<false>;
-  if (smem_bytes > configured[res]) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  {
+    cudaError_t e = dsn_ensure_dynamic_smem(kernel, smem_bytes, configured[res]);
     if (e != cudaSuccess) return e;
-    configured[res] = smem_bytes;
   }
   return dsn_launch(kernel, dim3(sm_count), dim3(kThreads), smem_bytes, s, 1, p);
 }

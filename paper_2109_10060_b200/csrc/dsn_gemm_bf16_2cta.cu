@@ -301,15 +301,14 @@ int dsn_gemm_pair_max_clusters(size_t smem_bytes) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_pair(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[3] = {0, 0, 0};
+  static size_t configured[3][DSN_MAX_DEVICES] = {};
   const bool lean = !p.residual && !p.bias && !p.bn_scale && p.act != DSN_ACT_GELU;
   const int form = p.residual ? 2 : (lean ? 1 : 0);
   void (*kernel)(GemmParams) = form == 2 ? gemm_bf16_pair_kernel<true, false>
                                : form == 1 ? gemm_bf16_pair_kernel<false, true> : gemm_bf16_pair_kernel<false, false>;
-  if (smem_bytes > configured[form]) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  {
+    cudaError_t e = dsn_ensure_dynamic_smem(kernel, smem_bytes, configured[form]);
     if (e != cudaSuccess) return e;
-    configured[form] = smem_bytes;
   }
   return dsn_launch(kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, p);
 }

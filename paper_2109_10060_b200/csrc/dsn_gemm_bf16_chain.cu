@@ -51,11 +51,12 @@ __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.pr
 static __device__ __noinline__ bool wait_counter(uint32_t addr, uint32_t target, volatile uint32_t* abort_flag,
                                                  int32_t* status, int where) {
   const uint64_t t0 = globaltimer_ns();
+  const uint64_t limit = wait_limit_ns(status);
   uint32_t spins = 0;
   while ((int32_t)(ld_acquire_cluster(addr) - target) < 0) {
     if ((++spins & 31u) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit) {
         *abort_flag = 1;
         dsn_set_status(status, DSN_ERR_TIMEOUT, where);
         return false;
@@ -379,7 +380,7 @@ size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[4] = {0, 0, 0, 0};
+  static size_t configured[4][DSN_MAX_DEVICES] = {};
   int aff = 0, gelu = 0;
   for (int l = 0; l < cp.n_layers; ++l) {
     aff |= (cp.L[l].bias || cp.L[l].bn_scale) ? 1 : 0;
@@ -388,10 +389,9 @@ cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, s
   void (*kernel)(DsnChainParams) = aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
                                        : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
   const int form = 2 * aff + gelu;
-  if (smem_bytes > configured[form]) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  {
+    cudaError_t e = dsn_ensure_dynamic_smem(kernel, smem_bytes, configured[form]);
     if (e != cudaSuccess) return e;
-    configured[form] = smem_bytes;
   }
   return dsn_launch(kernel, dim3(2 * clusters), dim3(kThreads), smem_bytes, s, 2, cp);
 }

@@ -18,7 +18,7 @@ constexpr uint32_t kABytes = BM * BK * 2;  // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kStageOutBytes = kEpiWarps * 32 * 128;  // epilogue staging: 32 rows x 128 bytes per warp
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: the default limit of a bounded wait
 
 // ---------------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -27,6 +27,11 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+}
+// Limit of a bounded wait: the context's setting (microseconds, in the status block) or the default.
+__device__ __forceinline__ uint64_t wait_limit_ns(const int32_t* status) {
+  const uint32_t us = status ? *reinterpret_cast<const volatile uint32_t*>(status + DSN_STATUS_WAIT_US) : 0u;
+  return us ? (uint64_t)us * 1000ull : kWaitLimitNs;
 }
 
 // True in exactly one lane of a converged warp.  Guarding the TMA / tcgen05 issue of a warp-uniform
@@ -67,12 +72,13 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                             int32_t* status, int where) {
   const uint64_t t0 = globaltimer_ns();
+  const uint64_t limit = wait_limit_ns(status);
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 31u) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit) {
         *abort_flag = 1;
         dsn_set_status(status, DSN_ERR_TIMEOUT, where);
         return false;

@@ -9,8 +9,11 @@
 #include "dsn.h"
 
 // Device status word: [0] = first condition code, [1] = detail, [2] = count of non-finite gate
-// scores, [3] = count of out-of-range routing indices.
-#define DSN_STATUS_WORDS 4
+// scores, [3] = count of out-of-range routing indices.  These four are read and cleared by dsn_get_status();
+// word [4] holds the limit of the kernels' bounded waits in microseconds (0 = the 2 s default).
+#define DSN_STATUS_WORDS 8
+#define DSN_STATUS_REPORT_WORDS 4
+#define DSN_STATUS_WAIT_US 4
 
 struct dsn_ctx {
   int device;
@@ -21,7 +24,11 @@ struct dsn_ctx {
   int conv_halo;       // 1 = 3x3 layers stage the input tile once with its halo (default), 0 = one load per tap (DSN_CONV3X3=taps)
   int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
+  uint32_t wait_limit_us;  // staging copy of the wait limit (source of the asynchronous copy into the status block)
 };
+
+// Launches a one-CTA kernel that waits on a barrier nobody arrives at (the self-test of the bounded waits).
+cudaError_t dsn_launch_selftest_wait(int32_t* status, cudaStream_t s);
 
 // Programmatic dependent launch: a kernel may be scheduled while its predecessor in the stream is
 // still draining.  Every kernel of this library therefore calls dsn_grid_dependency_wait() before its
@@ -59,6 +66,23 @@ inline cudaError_t dsn_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.attrs = attr;
   cfg.numAttrs = (unsigned)n;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The dynamic shared-memory limit of a kernel is a per-device attribute: it is raised once per (kernel form,
+// device), with the launching thread's current device (the context's device: every entry point checks that).
+#define DSN_MAX_DEVICES 64
+template <typename K>
+inline cudaError_t dsn_ensure_dynamic_smem(K kernel, size_t bytes, size_t* per_device /* [DSN_MAX_DEVICES] */) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= DSN_MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (bytes > per_device[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    per_device[dev] = bytes;
+  }
+  return cudaSuccess;
 }
 
 __device__ __forceinline__ void dsn_set_status(int32_t* status, int code, int detail) {

@@ -17,3 +17,19 @@ def dsn():
     """The ctypes binding of the CUDA library; GPU tests fail loudly when it is missing."""
     import paper_2109_10060_b200 as pkg
     return pkg
+
+
+# Measured parity figures (worst errors per configuration) that the GPU tests want shown with the result.
+PARITY_REPORT = []
+
+
+@pytest.fixture(scope="session")
+def parity_report():
+    return PARITY_REPORT
+
+
+def pytest_terminal_summary(terminalreporter):
+    if PARITY_REPORT:
+        terminalreporter.write_line("measured parity figures (max|err| / max|ref| per group unless stated):")
+        for line in PARITY_REPORT:
+            terminalreporter.write_line("  " + line)

@@ -111,6 +111,40 @@ def test_attention_full_size_vit_small_sampled(dsn, ctx):
         assert np.all(got[i, :, :w] != SENTINEL)
 
 
+def test_attention_full_size_vit_base_sampled(dsn, ctx, parity_report):
+    """The serving-scale configuration at its full size: 1024 samples x 197 tokens, 12 heads of which a path uses
+    5..12, quota-uniform routing over the 8 paths, grouped order, row pitch 2304 (what the QKV layer of the
+    benchmark step hands over).  The batch tiles a block of 64 seeded samples; the oracle evaluates the first and
+    last sample of every group."""
+    B, N, H, Dh, blk = 1024, 197, 12, 64, 64
+    heads = [p_[1] for p_ in wl.vit_base_paths()]
+    T = len(heads)
+    idx = np.asarray(wl.idx_quota_uniform(wl.rng(5, 9), B, T), np.int32)
+    g = np.random.default_rng(55)
+    q, k, v = (wl.to_bf16_values(wl.normal(g, (blk, N, H * Dh))) for _ in range(3))
+    block = up_bf16(head_major(q, k, v, H, Dh))                 # [64][N][3*H*Dh]
+    counts, offsets, perm, inv = O.route(idx, T)
+    r = route_on_gpu(dsn, ctx, idx, T)
+    src = block[torch.from_numpy((perm % blk).astype(np.int64)).to(DEV)]      # grouped: position p holds sample perm[p]
+    out = torch.full((B, N, H * Dh), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_attention(ctx, dsn.make_attention_desc(N, H, Dh, heads, order=dsn.GROUPED), r, src, out)
+    check_status(ctx, dsn)
+    sel = sorted({int(perm[offsets[t]]) for t in range(T) if counts[t]} | {int(perm[offsets[t + 1] - 1]) for t in range(T) if counts[t]})
+    src_of = [i % blk for i in sel]
+    ref = O.attention(q[src_of], k[src_of], v[src_of], idx[sel], heads, Dh)
+    got = down(out[torch.from_numpy(inv[sel].astype(np.int64)).to(DEV)])
+    worst = 0.0
+    for j, i in enumerate(sel):
+        w = heads[idx[i]] * Dh
+        err = np.max(np.abs(got[j, :, :w] - ref[j, :, :w])) / np.max(np.abs(ref[j, :, :w]))
+        worst = max(worst, err)
+        assert err <= TOL, (int(i), int(idx[i]), err)
+        assert np.all(got[j, :, w:] == SENTINEL)
+    parity_report.append(f"cfg5 attention core alone, B=1024, 5..12 heads: worst {worst:.2e} over {len(sel)} samples (bound {TOL:.0e})")
+    written = (out[:, 0, ::Dh] != SENTINEL).sum(dim=1).cpu().numpy()          # heads written per grouped position
+    np.testing.assert_array_equal(written, np.asarray(heads)[idx[perm]])
+
+
 def test_attention_closed_forms_on_device(dsn, ctx):
     """Zero queries -> every output row is the mean of the values; a dominant key copies its value."""
     B, N, H, Dh = 2, 197, 2, 64

@@ -241,6 +241,36 @@ def test_host_side_argument_errors_launch_nothing(dsn, ctx):
     check_status(ctx, dsn)
 
 
+def test_layer_forward_rejects_a_layer_that_reads_more_than_was_written(dsn, ctx):
+    """All layers of a block inherit one decision: a path may not read more columns of an intermediate than
+    the layer before wrote for it (those columns hold stale workspace bytes).  Refused on the host."""
+    B, R, C, T = 4, 8, 64, 2
+    W = torch.zeros(C, C, dtype=torch.bfloat16, device=DEV)
+    x = torch.zeros(B, R, C, dtype=torch.bfloat16, device=DEV)
+    y = torch.full((B, R, C), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    idx = torch.zeros(B, dtype=torch.int32, device=DEV)
+
+    def code_of(k_out0, k_in1, heads=None):
+        layers = [dsn.make_linear_desc(dsn.BF16, R, C, 3 * C if heads else C, [C, C], k_out0, torch.zeros(3 * C if heads else C, C, dtype=torch.bfloat16, device=DEV))]
+        if heads:
+            layers.append(dsn.make_attention_desc(R, 1, 64, heads))
+        layers.append(dsn.make_linear_desc(dsn.BF16, R, C, C, k_in1, [C, C], W))
+        L = dsn.make_layer_desc(B, T, layers, None)
+        ws = torch.empty(max(1024, dsn.dsn_layer_workspace_bytes(L) + 4096), dtype=torch.uint8, device=DEV)
+        try:
+            dsn.dsn_layer_forward(ctx, L, x, idx, y, ws)
+        except dsn.DsnError as e:
+            return e.code
+        return 0
+
+    assert code_of([32, 64], [32, 64]) == 0
+    assert code_of([32, 64], [40, 64]) == dsn.ERR_INVALID_ARG           # path 0 reads 40 columns, 32 were written
+    assert code_of([192, 128], [64, 64], heads=[1, 1]) == dsn.ERR_INVALID_ARG   # QKV of path 1 too narrow for its head
+    assert code_of([192, 192], [64, 64], heads=[1, 2]) == dsn.ERR_INVALID_ARG   # more heads than the layer has
+    assert code_of([192, 192], [64, 64], heads=[1, 1]) == 0
+    check_status(ctx, dsn)
+
+
 @pytest.mark.parametrize("T,in_order,out_order", [(40, 0, 0), (64, 1, 1)])
 def test_bf16_linear_more_slices_than_one_launch_holds(dsn, ctx, T, in_order, out_order):
     """A launch carries tensor maps for 16 distinct slices; a layer with more (here 40, and the maximum of

@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import dsn_workloads as wl
+from oracle import dsn_oracle as O
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -33,13 +34,23 @@ def _both(dsn, ctx, cfg, B, R, C):
     dsn.dsn_gate(ctx, g, x, idx_ref, log_ref, ws)
     idx_new = torch.full((B,), -2, dtype=torch.int32, device=DEV)
     log_new = torch.full((B, T), 7.0, dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()            # the driver's own count of free device memory
     dsn.dsn_gate_static(ctx, g, x, idx_new, log_new)
     torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before                      # the call took no device memory from anyone
     assert ctx.get_status() == (0, 0)
     scale = max(1.0, float(log_ref.abs().max()))
     assert float((log_new - log_ref).abs().max()) <= 2e-5 * scale      # the gate tests' score tolerance
     assert torch.equal(idx_new, idx_ref)
     assert int(idx_ref.min()) >= 0 and int(idx_ref.max()) < T
+    # and directly against the CPU oracle: scores within the gate tolerance, choices equal outside the 1e-4 margin
+    idx_o, scores_o, margin = O.gate(cfg["x"].reshape(B, R, C), cfg["gate_W1"], cfg["gate_W2"])
+    got = log_new.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - scores_o)) <= 2e-5 * max(1.0, float(np.max(np.abs(scores_o))))
+    safe = margin >= 1e-4
+    np.testing.assert_array_equal(idx_new.cpu().numpy()[safe], idx_o[safe])
 
 
 def test_static_gate_matches_workspace_gate_on_two_calls_in_a_row(dsn):
