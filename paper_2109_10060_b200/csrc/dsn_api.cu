@@ -825,12 +825,19 @@ int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_ro
   if (e) return e;
   if (r->B == 0) return DSN_OK;
   CUtensorMap map;
-  const uint64_t dims[3] = {64, (uint64_t)3 * d->H, (uint64_t)r->B * d->N};
-  const uint64_t str[2] = {128, (uint64_t)d->ld_qkv * 2};
-  const uint32_t box[3] = {64, 1, 128};
-  e = encode_map(ctx, &map, qkv, 3, dims, str, box);
+  // samples are a dimension of their own: a box that runs past the sample's last row reads zeros there
+  const uint64_t dims[4] = {64, (uint64_t)3 * d->H, (uint64_t)d->N, (uint64_t)r->B};
+  const uint64_t str[3] = {128, (uint64_t)d->ld_qkv * 2, (uint64_t)d->ld_qkv * 2 * (uint64_t)d->N};
+  const uint32_t box[4] = {64, 1, 128, 1};
+  e = encode_map(ctx, &map, qkv, 4, dims, str, box);
   if (e) return e;
-  if (dsn_launch_attention(map, d->heads, d->T, d->N, d->H, r->B, r->G, d->order == DSN_GROUPED, r->offsets, r->perm,
+  CUtensorMap map_out;
+  const uint64_t od[3] = {(uint64_t)d->H * 64, (uint64_t)d->N, (uint64_t)r->B};
+  const uint64_t os[2] = {(uint64_t)d->ld_out * 2, (uint64_t)d->ld_out * 2 * (uint64_t)d->N};
+  const uint32_t ob[3] = {64, 32, 1};
+  e = encode_map(ctx, &map_out, out, 3, od, os, ob);
+  if (e) return e;
+  if (dsn_launch_attention(map, map_out, d->heads, d->T, d->N, d->H, r->B, r->G, d->order == DSN_GROUPED, r->offsets, r->perm,
                            r->group_slice, qkv, d->ld_qkv, out, d->ld_out, ctx->d_status, as_stream(stream)) !=
       cudaSuccess)
     return DSN_ERR_CUDA;

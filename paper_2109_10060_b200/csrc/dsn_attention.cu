@@ -24,7 +24,11 @@
 //   the row is scaled by 1 / sum, rounded to bf16 and stored (each of the two threads writes 64 bytes
 //   of the 128-byte line).
 // Waits are bounded as in the GEMM.
+#include <stdlib.h>
+#include <string.h>
+
 #include "dsn_gemm_device.cuh"
+#include "dsn_attention.cuh"
 
 namespace {
 
@@ -36,21 +40,6 @@ constexpr uint32_t kKBytes = 256 * 128;       // 256 keys x 64 bf16
 constexpr uint32_t kVBytes = 256 * 128;       // 256 keys x 64 bf16
 constexpr uint32_t kPBytes = 4 * 128 * 128;   // 4 key chunks x 128 queries x 64 keys bf16 (over K, Q and 16 KB more)
 constexpr uint32_t kAttTmemCols = 256;
-
-struct AttParams {
-  CUtensorMap map;        // qkv seen as [rows][3H][64], box 128 rows x 1 x 64
-  int8_t heads[DSN_MAX_SLICES];
-  int32_t N, H, B, G, T;
-  int32_t grouped;        // 1: position p holds its data at row block p; 0: at row block perm[p]
-  const int32_t* offsets;
-  const int32_t* perm;
-  const int32_t* group_slice;
-  const __nv_bfloat16* qkv;
-  int64_t ld_qkv;
-  __nv_bfloat16* out;
-  int64_t ld_out;
-  int32_t* status;
-};
 
 __device__ __forceinline__ int find_group_of(const int32_t* __restrict__ offsets, int G, int p) {
   int lo = 0, hi = G;
@@ -83,7 +72,6 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16])
       : "memory");
 }
 
-constexpr int kAttTableGroups = 64;  // groups the persistent form can hold in its shared-memory table
 
 // One work item = (sample position, head, half of the queries).  kPersist = false: one CTA per item of
 // the dense grid (head, position, half); items of heads the sample's path does not have return at once.
@@ -190,13 +178,12 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
   const int npad = (N + 15) & ~15;
   const int kboxes = npad > 128 ? 2 : 1;
   auto issue_loads = [&](int hd, int hf, int bk) {  // by one elected lane
-    const int r0 = bk * N;
     mbar_expect_tx(bar_load, (uint32_t)kboxes * 2u * 16384u + kQBytes);
     for (int b2 = 0; b2 < kboxes; ++b2) {
-      tma_load_3d(k_s + b2 * 16384, &p.map, 0, hd * 3 + 1, r0 + 128 * b2, bar_load);
-      tma_load_3d(v_s + b2 * 16384, &p.map, 0, hd * 3 + 2, r0 + 128 * b2, bar_load);
+      tma_load_4d(k_s + b2 * 16384, &p.map, 0, hd * 3 + 1, 128 * b2, bk, bar_load);
+      tma_load_4d(v_s + b2 * 16384, &p.map, 0, hd * 3 + 2, 128 * b2, bk, bar_load);
     }
-    tma_load_3d(q_s, &p.map, 0, hd * 3 + 0, r0 + 128 * hf, bar_load);
+    tma_load_4d(q_s, &p.map, 0, hd * 3 + 0, 128 * hf, bk, bar_load);
   };
 
   if (warp == 1) {  // not the warp that issues the loads: the allocation may have to wait for the SM's other CTA
@@ -399,11 +386,18 @@ __global__ void __launch_bounds__(kAttThreads, 2) attention_kernel(const __grid_
 
 }  // namespace
 
-struct dsn_attention_launch {
-  AttParams p;
-};
+// 0 (default): the warp-specialised form where it applies; DSN_ATTENTION=items keeps the form with one
+// (sample, head, query half) item per CTA pass everywhere (for comparisons).
+static int dsn_attention_form() {
+  static int form = -1;
+  if (form < 0) {
+    const char* e = getenv("DSN_ATTENTION");
+    form = (e && strcmp(e, "items") == 0) ? 1 : 0;
+  }
+  return form;
+}
 
-cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, int T, int N, int H, int B, int G,
+cudaError_t dsn_launch_attention(const CUtensorMap& map, const CUtensorMap& map_out, const int32_t* heads, int T, int N, int H, int B, int G,
                                  int grouped, const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                  const void* qkv, int64_t ld_qkv, void* out, int64_t ld_out, int32_t* status,
                                  cudaStream_t s) {
@@ -411,6 +405,7 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   AttParams p;
   memset(&p, 0, sizeof(p));
   p.map = map;
+  p.map_out = map_out;
   for (int t = 0; t < T; ++t) p.heads[t] = (int8_t)heads[t];
   p.N = N; p.H = H; p.B = B; p.G = G; p.T = T; p.grouped = grouped;
   p.offsets = offsets; p.perm = perm; p.group_slice = group_slice;
@@ -427,6 +422,7 @@ cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, i
   if (e != cudaSuccess) return e;
   const int resident = 2 * sms;  // CTAs the persistent form keeps in flight: two per SM
   const int halves = N > 128 ? 2 : 1;
+  if (G <= kAttTableGroups && dsn_attention_form() == 0) return dsn_launch_attention_ws(p, sms, s);
   if (G <= kAttTableGroups) {
     const long long dense = (long long)H * B * halves;
     return dsn_launch(attention_kernel<true>, dim3((unsigned)(dense < resident ? dense : resident)), dim3(kAttThreads), smem, s,

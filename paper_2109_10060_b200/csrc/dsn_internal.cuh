@@ -182,7 +182,7 @@ cudaError_t dsn_launch_resbn_fold(int n, int C, const float* gamma, const float*
 cudaError_t dsn_launch_route(const int32_t* idx, int B, int T, int32_t* counts, int32_t* offsets,
                              int32_t* perm, int32_t* inv_perm, int32_t* status, cudaStream_t s);
 
-cudaError_t dsn_launch_attention(const CUtensorMap& map, const int32_t* heads, int T, int N, int H, int B, int G,
+cudaError_t dsn_launch_attention(const CUtensorMap& map, const CUtensorMap& map_out, const int32_t* heads, int T, int N, int H, int B, int G,
                                  int grouped, const int32_t* offsets, const int32_t* perm, const int32_t* group_slice,
                                  const void* qkv, int64_t ld_qkv, void* out, int64_t ld_out, int32_t* status,
                                  cudaStream_t s);
