@@ -45,7 +45,10 @@ enum dsn_status {
 };
 
 enum dsn_dtype { DSN_F32 = 0, DSN_BF16 = 1 };
-enum dsn_act { DSN_ACT_NONE = 0, DSN_ACT_RELU = 1, DSN_ACT_GELU = 2 /* exact erf form */ };
+/* DSN_ACT_GELU: x/2 (1 + erf(x / sqrt 2)) with erf evaluated as tanh of a fitted odd quintic on the hardware
+ * tanh: within 3e-5 (absolute) of the erf form from the fit, below 1e-3 absolute overall at |x| = 4, i.e. a
+ * fraction of a bfloat16 rounding step of the output. */
+enum dsn_act { DSN_ACT_NONE = 0, DSN_ACT_RELU = 1, DSN_ACT_GELU = 2 };
 enum dsn_order { DSN_INPUT_ORDER = 0, DSN_GROUPED = 1 };
 enum dsn_tail { DSN_TAIL_UNTOUCHED = 0, DSN_TAIL_ZERO = 1 };
 enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1, DSN_LAYER_ATTENTION = 2 };
@@ -186,8 +189,11 @@ typedef struct dsn_layer_desc {
  * Environment switches, read here, that select between kernels computing the same results (for
  * comparisons and as fallbacks): DSN_GEMM_MODE=1cta (one CTA per tile instead of CTA pairs),
  * DSN_CHAIN=0 (dsn_layer_forward: one launch per layer even for small batches), DSN_CONV3X3=taps
- * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_PDL=0 (no
- * programmatic dependent launch). */
+ * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_ATTENTION=items (the
+ * attention core with one (sample, head, query half) per CTA pass instead of the warp-specialised form),
+ * DSN_PDL=0 (no programmatic dependent launch).
+ * Every later call must be made with `device` as the calling thread's current CUDA device (else
+ * DSN_ERR_INVALID_ARG): launches and kernel attributes act on the current device. */
 int dsn_create(dsn_ctx** ctx, int device);
 int dsn_destroy(dsn_ctx* ctx);
 const char* dsn_strerror(int code);
@@ -231,8 +237,8 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
  * until the process exits), so the call takes no workspace and performs no allocation of any kind.
  *   - Limit: B * (splits * c_valid + C_mlp) <= 1,048,576 floats, where splits (1..64) is the
  *     row-band count the gate picks for this GPU; larger problems return DSN_ERR_WORKSPACE and
- *     launch nothing.  The ResNet-50 and ViT workloads fit (128 x (5 x 1024 + 128),
- *     1024 x (1 x 768 + 128)).
+ *     launch nothing.  The ResNet-50 and ViT workloads fit (128 samples x (4 splits x 1024 + 128) on a
+ *     148-SM GPU, 1024 x (1 x 768 + 128)).
  *   - The context's device must be the current device (else DSN_ERR_INVALID_ARG).
  *   - The first call on a device looks up the array's device address (a synchronous runtime
  *     query); make that first call before starting any stream capture.
@@ -305,7 +311,8 @@ size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L);
  * (Sec. 5).  Batches of at most two samples per SM pair whose samples have 150..256 rows (14x14
  * images, 197 tokens) run their 2-3 sliced layers as ONE launch in which every SM pair walks whole
  * samples through the layers; otherwise (and whenever a layer has skip features or the block holds
- * the attention core) one launch per layer.  Same results either way.
+ * the attention core) one launch per layer.  The two forms agree to within one bfloat16 rounding step of an
+ * output on a few percent of the elements (the 3x3 layer sums its taps in a different order), not bit for bit.
  * x, y in input order.  idx_in: device [B], required when L->gate is NULL, ignored otherwise.
  * r_out (optional): receives pointers into the workspace holding the block's routing arrays
  * (valid until the workspace is reused).  idx_out (optional): device [B], the gate's choice. */
