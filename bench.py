@@ -493,6 +493,10 @@ class MobileNetBlock(Workload):
                                           in_order=dsn.INPUT_ORDER, out_order=dsn.GROUPED)
         self.pw = dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, C, w, w, self.Wpw, act=dsn.ACT_RELU,
                                      in_order=dsn.GROUPED, out_order=dsn.INPUT_ORDER)
+        # the step: one dsn_layer_forward call; depthwise + pointwise run as one kernel
+        self.L = dsn.make_layer_desc(B, T, [dsn.make_depthwise_desc(H, Wd, K, 1, C, w, [K] * T, self.Wdw, act=dsn.ACT_RELU),
+                                            dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, C, w, w, self.Wpw, act=dsn.ACT_RELU)], None)
+        self.ws = torch.empty(dsn.dsn_layer_workspace_bytes(self.L), dtype=torch.uint8, device=dev)
         self.gW1 = torch.from_numpy(cfg["gate_W1"]).to(dev)
         self.gW2 = torch.from_numpy(cfg["gate_W2"]).to(dev)
         self.gate = dsn.make_gate_desc(dsn.BF16, B, self.R, C, self.gW1.shape[0], T, self.gW1, self.gW2)
@@ -502,10 +506,11 @@ class MobileNetBlock(Workload):
         ints = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
         self.routing = dsn.make_routing(B, T, ints(T), ints(T + 1), ints(B), ints(B))
         self.t_dw = torch.zeros(B, H, Wd, C, dtype=torch.bfloat16, device=dev)
-        self.kernels_per_step = 3 + 1 + 2
+        self.kernels_per_step = 3 + 1 + 1
         self.name = cfg["name"]
         self.routing_name = cfg["routing"]
-        self.path = "gate -> route -> depthwise 3x3 (ReLU) -> pointwise 1x1 (ReLU) -> input order"
+        self.path = ("gate -> route -> [depthwise 3x3 (ReLU) -> pointwise 1x1 (ReLU)] as one kernel -> input order: dsn_gate, then "
+                     "one dsn_layer_forward call on the given routing")
         self.flops_note = "2 x multiply-adds of the depthwise (9 c_t per pixel) and pointwise (c_t^2 per pixel) layers"
 
     def _host(self, cfg):
@@ -521,9 +526,7 @@ class MobileNetBlock(Workload):
     def step(self, ctx, i):
         k, d = i % self.copies, self.dsn
         d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws)
-        d.dsn_route(ctx, self.idx_given, self.B, self.T, self.routing)
-        d.dsn_sliced_depthwise(ctx, self.dw, self.routing, self.xs[k], self.t_dw)
-        d.dsn_sliced_conv(ctx, self.pw, self.routing, self.t_dw, self.ys[k])
+        d.dsn_layer_forward(ctx, self.L, self.xs[k], self.idx_given, self.ys[k], self.ws)
 
     def histogram(self):
         return np.bincount(self.cfg["idx"], minlength=self.T)
@@ -541,9 +544,11 @@ class MobileNetBlock(Workload):
             ("gate", lambda ctx, k: d.dsn_gate(ctx, self.gate, self.xs[k], self.idx_out, None, self.gate_ws), 0,
              2 * self.B * self.R * self.C, "hbm"),
             ("route", lambda ctx, k: d.dsn_route(ctx, self.idx_given, self.B, self.T, r), 0, 20 * self.B, "latency"),
-            ("depthwise", lambda ctx, k: d.dsn_sliced_depthwise(ctx, self.dw, r, self.xs[k], self.t_dw), dwf, dw_bytes, "hbm"),
-            ("gemm:pointwise", lambda ctx, k: d.dsn_sliced_conv(ctx, self.pw, r, self.t_dw, self.ys[k]), pwf,
-             gemm_algorithmic_bytes(c, self.R, w, w), "gemm"),
+            ("route+gemm:dwpw_fused", lambda ctx, k: d.dsn_layer_forward(ctx, self.L, self.xs[k], self.idx_given, self.ys[k], self.ws),
+             dwf + pwf, gemm_algorithmic_bytes(c, self.R, w, w), "gemm"),
+            ("unfused:depthwise", lambda ctx, k: d.dsn_sliced_depthwise(ctx, self.dw, r, self.xs[k], self.t_dw), dwf, dw_bytes, "hbm"),
+            ("unfused:pointwise", lambda ctx, k: d.dsn_sliced_conv(ctx, self.pw, r, self.t_dw, self.ys[k]), pwf,
+             gemm_algorithmic_bytes(c, self.R, w, w), "other"),
         ]
 
     def exec_flops(self, counts):

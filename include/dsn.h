@@ -51,7 +51,7 @@ enum dsn_dtype { DSN_F32 = 0, DSN_BF16 = 1 };
 enum dsn_act { DSN_ACT_NONE = 0, DSN_ACT_RELU = 1, DSN_ACT_GELU = 2 };
 enum dsn_order { DSN_INPUT_ORDER = 0, DSN_GROUPED = 1 };
 enum dsn_tail { DSN_TAIL_UNTOUCHED = 0, DSN_TAIL_ZERO = 1 };
-enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1, DSN_LAYER_ATTENTION = 2 };
+enum dsn_layer_kind { DSN_LAYER_LINEAR = 0, DSN_LAYER_CONV = 1, DSN_LAYER_ATTENTION = 2, DSN_LAYER_DEPTHWISE = 3 };
 
 #define DSN_MAX_SLICES 64   /* largest T                                               */
 #define DSN_MAX_GROUPS 4096 /* largest G of a caller-built group list                  */
@@ -179,8 +179,14 @@ typedef struct dsn_layer_desc {
   int32_t T;
   int32_t n_layers;                 /* 1..DSN_MAX_CHAIN                                  */
   int32_t kind[DSN_MAX_CHAIN];      /* dsn_layer_kind                                    */
-  const void* layer[DSN_MAX_CHAIN]; /* dsn_linear_desc*, dsn_conv_desc* or (between two layers) dsn_attention_desc*;
-                                       order and leading-dimension fields of chained elements are ignored */
+  const void* layer[DSN_MAX_CHAIN]; /* dsn_linear_desc*, dsn_conv_desc*, dsn_depthwise_desc* (not as the last element) or
+                                       (between two layers) dsn_attention_desc*; order and leading-dimension fields of
+                                       chained elements are ignored.  A depthwise element followed by a 1x1 layer whose
+                                       k_in equals the depthwise widths (the DS-MBNet separable block, Sec. 3.3) can run
+                                       as ONE kernel in which the depthwise result feeds the tensor core from shared
+                                       memory and never reaches global memory (DSN_DWPW=fused; bf16, widths and row
+                                       pitches multiples of 8); by default the two run one after the other through the
+                                       workspace, which is the faster form on this GPU */
 } dsn_layer_desc;
 
 /* ---- context ------------------------------------------------------------------------- */
@@ -191,7 +197,7 @@ typedef struct dsn_layer_desc {
  * DSN_CHAIN=0 (dsn_layer_forward: one launch per layer even for small batches), DSN_CONV3X3=taps
  * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_ATTENTION=items (the
  * attention core with one (sample, head, query half) per CTA pass instead of the warp-specialised form),
- * DSN_PDL=0 (no programmatic dependent launch).
+ * DSN_DWPW=fused (depthwise + following 1x1 layer as one kernel), DSN_PDL=0 (no programmatic dependent launch).
  * Every later call must be made with `device` as the calling thread's current CUDA device (else
  * DSN_ERR_INVALID_ARG): launches and kernel attributes act on the current device. */
 int dsn_create(dsn_ctx** ctx, int device);
@@ -210,6 +216,13 @@ int dsn_set_wait_limit(dsn_ctx* ctx, uint32_t microseconds, void* stream);
  * on a barrier nothing arrives at.  It returns after the wait limit; dsn_get_status() then reports
  * DSN_ERR_TIMEOUT (detail 9001).  Nothing faults and later calls run normally. */
 int dsn_selftest_bounded_wait(dsn_ctx* ctx, void* stream);
+
+/* The context keeps the TMA tensor maps it has encoded (keyed by base pointer, extents, strides and box; 512 slots,
+ * host memory), so that repeated calls on the same buffers and slices skip the encoding (about a microsecond per
+ * map, up to three maps per distinct slice and layer).  A map describes addresses and geometry only, so a hit stays
+ * valid for as long as the caller's buffer does.  DSN_MAP_CACHE=0 at dsn_create turns the cache off.
+ * Returns the hit and miss counts since the context was created. */
+int dsn_map_cache_stats(dsn_ctx* ctx, uint64_t* hits, uint64_t* misses);
 
 /* Ratio list -> channel counts (host only).  granule g = 0 picks g = min(8, C/32);
  * k = g*floor(r*C/g + 1/2) clamped to [g, C].  The paper lists channel counts, not a rounding

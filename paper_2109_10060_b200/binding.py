@@ -20,11 +20,11 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
 INPUT_ORDER, GROUPED = 0, 1
 TAIL_UNTOUCHED, TAIL_ZERO = 0, 1
-LAYER_LINEAR, LAYER_CONV, LAYER_ATTENTION = 0, 1, 2
+LAYER_LINEAR, LAYER_CONV, LAYER_ATTENTION, LAYER_DEPTHWISE = 0, 1, 2, 3
 MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 6
 
 EXPORTS = [
-    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_set_wait_limit", "dsn_selftest_bounded_wait", "dsn_widths_from_ratios",
+    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_set_wait_limit", "dsn_selftest_bounded_wait", "dsn_map_cache_stats", "dsn_widths_from_ratios",
     "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
     "dsn_sliced_attention", "dsn_sliced_depthwise", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
@@ -103,6 +103,7 @@ def load_library():
     lib.dsn_get_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
     lib.dsn_set_wait_limit.argtypes = [vp, C.c_uint32, vp]
     lib.dsn_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.dsn_map_cache_stats.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.dsn_widths_from_ratios.argtypes = [i32, C.POINTER(C.c_double), i32, i32, C.POINTER(i32)]
     lib.dsn_executed_macs.argtypes = [C.POINTER(i32), i32, i32, C.POINTER(i32), C.POINTER(i32), i32]
     lib.dsn_executed_macs.restype = i64
@@ -198,6 +199,12 @@ class Context:
         """Launches the kernel that waits on a barrier nobody arrives at; it returns after the wait limit."""
         _check(self.lib.dsn_selftest_bounded_wait(self.handle, _stream_handle(stream)), "dsn_selftest_bounded_wait")
 
+    def map_cache_stats(self):
+        """(hits, misses) of the context's tensor-map cache."""
+        h, m = C.c_uint64(), C.c_uint64()
+        _check(self.lib.dsn_map_cache_stats(self.handle, C.byref(h), C.byref(m)), "dsn_map_cache_stats")
+        return h.value, m.value
+
     def get_status(self, stream=None):
         code, detail = C.c_int32(), C.c_int32()
         _check(self.lib.dsn_get_status(self.handle, _stream_handle(stream), C.byref(code), C.byref(detail)),
@@ -245,7 +252,8 @@ def make_layer_desc(B, T, layers, gate: Optional[GateDesc] = None) -> LayerDesc:
     L.gate = C.pointer(gate) if gate is not None else None
     L.B, L.T, L.n_layers = B, T, len(layers)
     for j, d in enumerate(layers):
-        L.kind[j] = LAYER_CONV if isinstance(d, ConvDesc) else (LAYER_ATTENTION if isinstance(d, AttentionDesc) else LAYER_LINEAR)
+        L.kind[j] = (LAYER_CONV if isinstance(d, ConvDesc) else LAYER_ATTENTION if isinstance(d, AttentionDesc)
+                     else LAYER_DEPTHWISE if isinstance(d, DepthwiseDesc) else LAYER_LINEAR)
         L.layer[j] = C.cast(C.pointer(d), C.c_void_p)
     L._keep = (gate, list(layers))
     return L

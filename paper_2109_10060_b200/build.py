@@ -17,7 +17,7 @@ OBJ_DIR = os.path.join(PKG_DIR, "_build")
 LIB_PATH = os.path.join(PKG_DIR, "libdsn.so")
 SOURCES = ["dsn_api.cu", "dsn_gate.cu", "dsn_route.cu", "dsn_copy.cu", "dsn_linear_f32.cu", "dsn_gemm_bf16.cu",
            "dsn_gemm_bf16_2cta.cu", "dsn_gemm_bf16_chain.cu", "dsn_conv3x3_halo.cu", "dsn_attention.cu", "dsn_attention_ws.cu",
-           "dsn_depthwise.cu", "dsn_selftest.cu"]
+           "dsn_depthwise.cu", "dsn_dwpw.cu", "dsn_selftest.cu"]
 
 
 def _headers_mtime() -> float:

@@ -37,8 +37,32 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 
 // bf16 tensor map of rank `rank` (3 or 4); dims/strides innermost first, strides[0] implied.
-int encode_map(const dsn_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+int encode_map(dsn_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                const uint64_t* strides_bytes /* rank-1 */, const uint32_t* box) {
+  dsn_map_slot* slot = nullptr;
+  dsn_map_key key;
+  if (ctx->map_cache) {
+    memset(&key, 0, sizeof(key));
+    key.base = base;
+    key.rank = (uint32_t)rank;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
+    uint64_t h = 1469598103934665603ull;  // FNV-1a over the key
+    const unsigned char* kb = reinterpret_cast<const unsigned char*>(&key);
+    for (size_t i = 0; i < sizeof(key); ++i) h = (h ^ kb[i]) * 1099511628211ull;
+    // four probes from the hashed slot; a miss takes the first free probe, else replaces the hashed slot
+    for (int probe = 0; probe < 4; ++probe) {
+      dsn_map_slot* cand = &ctx->map_cache[(h + (uint64_t)probe) % DSN_MAP_CACHE_SLOTS];
+      if (cand->used && memcmp(&cand->key, &key, sizeof(key)) == 0) {
+        *out = cand->map;
+        ++ctx->map_hits;
+        return DSN_OK;
+      }
+      if (!cand->used && !slot) slot = cand;
+    }
+    if (!slot) slot = &ctx->map_cache[h % DSN_MAP_CACHE_SLOTS];
+    ++ctx->map_misses;
+  }
   cuuint64_t gd[4], gs[3];
   cuuint32_t bx[4], es[4];
   for (int i = 0; i < rank; ++i) {
@@ -55,7 +79,13 @@ int encode_map(const dsn_ctx* ctx, CUtensorMap* out, const void* base, int rank,
       out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? DSN_OK : DSN_ERR_CUDA;
+  if (r != CUDA_SUCCESS) return DSN_ERR_CUDA;
+  if (slot) {
+    slot->key = key;
+    slot->map = *out;
+    slot->used = 1;
+  }
+  return DSN_OK;
 }
 
 // One sliced layer in the form the kernels take.
@@ -73,6 +103,8 @@ struct LayerCall {
   const void* residual;
   int act, in_order, out_order, tail;
   const dsn_attention_desc* att;  // non-null: this chain element is the attention core, not a sliced layer
+  const dsn_depthwise_desc* dw;   // non-null: this chain element is a slice-able depthwise convolution
+  int R_in;                       // rows per sample it reads (differs from H * W, the rows it writes, for a strided depthwise element)
 };
 
 int check_slices(int T, const int32_t* k_in, const int32_t* k_out, int C_in, int C_out) {
@@ -352,7 +384,7 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
   int bn_max = 64;
   for (int j = 0; j < n; ++j) {
     const LayerCall& c = calls[j];
-    if (c.att || c.dtype != DSN_BF16 || c.tail != DSN_TAIL_UNTOUCHED) return 0;
+    if (c.att || c.dw || c.dtype != DSN_BF16 || c.tail != DSN_TAIL_UNTOUCHED) return 0;
     if (c.residual) return 0;  // skip features are added by the single-layer kernels, which prefetch them
     // a sample must fill most of ONE 256-row pair tile: with more rows per sample the single-layer launches
     // (tiles across sample boundaries, halo form of the 3x3 layer) are faster (measured at 28x28 and 56x56)
@@ -392,6 +424,54 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
   return 1;
 }
 
+// Can the depthwise element `d` and the sliced layer `c` that follows it run as one kernel?
+bool dwpw_fusable(const LayerCall& d, const LayerCall& c, const void* x) {
+  if (!d.dw || c.att || c.dw || c.dtype != DSN_BF16 || c.K != 1 || c.residual || c.tail != DSN_TAIL_UNTOUCHED) return false;
+  const dsn_depthwise_desc* w = d.dw;
+  if (w->C % 8 || d.ldx % 8 || !aligned16(x) || !aligned16(w->W)) return false;
+  for (int t = 0; t < c.T; ++t)
+    if (w->c[t] % 8 || c.k_in[t] != w->c[t]) return false;
+  return true;
+}
+
+// depthwise element `d` (input x, order d.in_order) + pointwise layer `c` (output y) as one launch per 16 distinct slices
+int run_dwpw(dsn_ctx* ctx, const LayerCall& d, const LayerCall& c, const dsn_routing* r, const void* x, void* y,
+             cudaStream_t s) {
+  if (r->B == 0) return DSN_OK;
+  DwPwParams q;
+  memset(&q, 0, sizeof(q));
+  LayerCall cc = c;
+  cc.in_order = DSN_GROUPED;
+  fill_gemm_params(ctx, cc, r, y, false, q.g);
+  GemmGeom& g = q.g.g;
+  g.flat = 1;  // M rows are the group's output pixels, whatever the order of the block input
+  g.bw = DSN_GEMM_BM;
+  g.bh = g.nb = g.tiles_x = g.tiles_y = 1;
+  g.R = c.H * c.W;
+  g.a_input_order = d.in_order == DSN_INPUT_ORDER;
+  g.pair = 0;
+  g.stages = g.BN == 256 ? 4 : (g.BN == 128 ? 6 : 8);
+  while (g.stages > 2 && dsn_dwpw_smem_bytes(g.BN, g.stages, r->G) > 227 * 1024) --g.stages;
+  const dsn_depthwise_desc* w = d.dw;
+  q.x = static_cast<const __nv_bfloat16*>(x);
+  q.ldx = d.ldx;
+  q.w = static_cast<const __nv_bfloat16*>(w->W);
+  q.dw_bias = w->bias; q.dw_bn_scale = w->bn_scale; q.dw_bn_shift = w->bn_shift; q.dw_act = w->act;
+  q.H = w->H; q.W = w->W_; q.Wo = c.W; q.K = w->K; q.stride = w->stride; q.C = w->C;
+  for (int t = 0; t < w->T; ++t) q.ksize[t] = (int8_t)w->ksize[t];
+  int done[DSN_MAX_SLICES];
+  memset(done, 0, sizeof(done));
+  int remaining = c.T;
+  const size_t smem = dsn_dwpw_smem_bytes(g.BN, g.stages, r->G);
+  while (remaining > 0) {
+    const int e = fill_gemm_maps(ctx, cc, r, y /* stands in for the activation map, which this kernel does not use */, y,
+                                 q.g, done, remaining);
+    if (e) return e;
+    if (dsn_launch_dwpw(q, ctx->sm_count, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
+  }
+  return DSN_OK;
+}
+
 int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
   int e = check_ctx(ctx);
   if (e) return e;
@@ -429,6 +509,7 @@ LayerCall from_linear(const dsn_linear_desc* d) {
   c.w_row = d->ldw; c.w_tap = d->ldw;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
   c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.residual = d->residual; c.att = nullptr;
+  c.dw = nullptr; c.R_in = d->R;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
 }
@@ -442,8 +523,23 @@ LayerCall from_conv(const dsn_conv_desc* d) {
   c.w_row = (int64_t)d->K * d->K * d->C_in; c.w_tap = d->C_in;
   c.T = d->T; c.k_in = d->k_in; c.k_out = d->k_out;
   c.Wt = d->W; c.bias = d->bias; c.bn_scale = d->bn_scale; c.bn_shift = d->bn_shift; c.residual = d->residual; c.att = nullptr;
+  c.dw = nullptr; c.R_in = d->H * d->W_;
   c.act = d->act; c.in_order = d->in_order; c.out_order = d->out_order; c.tail = d->tail;
   return c;
+}
+
+int check_depthwise(const dsn_depthwise_desc* d) {
+  if (!d || !d->W || !d->c || !d->ksize) return DSN_ERR_INVALID_ARG;
+  if (d->dtype != DSN_BF16) return DSN_ERR_UNSUPPORTED;
+  if (d->H < 1 || d->W_ < 1 || d->C < 1 || d->C > 32767 || d->K < 1 || d->K > 7 || d->K % 2 == 0) return DSN_ERR_INVALID_ARG;
+  if (d->stride != 1 && d->stride != 2) return DSN_ERR_UNSUPPORTED;
+  if (d->ldx < d->C || d->ldy < d->C || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
+  if (d->act < DSN_ACT_NONE || d->act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
+  if ((d->bn_scale == nullptr) != (d->bn_shift == nullptr)) return DSN_ERR_INVALID_ARG;
+  for (int t = 0; t < d->T; ++t)
+    if (d->c[t] < 1 || d->c[t] > d->C || d->ksize[t] < 1 || d->ksize[t] > d->K || d->ksize[t] % 2 == 0)
+      return DSN_ERR_INVALID_ARG;
+  return DSN_OK;
 }
 
 // Host-side checks of an attention element (pointers may be null when only the descriptor is checked).
@@ -491,11 +587,27 @@ int layer_call_of(const dsn_layer_desc* L, int j, LayerCall& c) {
     if (!a->heads || a->T < 1 || a->T > DSN_MAX_SLICES || a->D_h < 1 || a->H < 1) return DSN_ERR_INVALID_ARG;
     memset(&c, 0, sizeof(c));
     c.att = a;
+    c.R_in = a->N;
     c.dtype = a->dtype;
     c.H = 1; c.W = a->N; c.K = 1;
     c.C_in = 3 * a->H * a->D_h;
     c.C_out = a->H * a->D_h;
     c.T = a->T;
+  } else if (L->kind[j] == DSN_LAYER_DEPTHWISE) {
+    // never the last element: the block's output comes from a sliced layer
+    if (j + 1 == L->n_layers) return DSN_ERR_INVALID_ARG;
+    const dsn_depthwise_desc* d = static_cast<const dsn_depthwise_desc*>(L->layer[j]);
+    const int e = check_depthwise(d);
+    if (e) return e;
+    memset(&c, 0, sizeof(c));
+    c.dw = d;
+    c.dtype = d->dtype;
+    c.H = (d->H - 1) / d->stride + 1; c.W = (d->W_ - 1) / d->stride + 1; c.K = 1;   // the rows it writes
+    c.R_in = d->H * d->W_;
+    c.C_in = d->C; c.C_out = d->C;
+    c.T = d->T;
+    c.k_in = d->c; c.k_out = d->c;
+    c.ldx = d->ldx; c.ldy = d->C;
   } else return DSN_ERR_INVALID_ARG;
   return DSN_OK;
 }
@@ -525,7 +637,7 @@ int plan_layer(const dsn_layer_desc* L, LayerPlan& pl) {
     if (e) return e;
     if (c.T != L->T || c.dtype != first.dtype) return DSN_ERR_INVALID_ARG;
     if (!c.att && (!c.k_in || !c.k_out)) return DSN_ERR_INVALID_ARG;
-    if (j > 0 && (c.C_in != prev_out || c.H * c.W != prev_R)) return DSN_ERR_INVALID_ARG;
+    if (j > 0 && (c.C_in != prev_out || c.R_in != prev_R)) return DSN_ERR_INVALID_ARG;
     // every layer of the block inherits the one decision (Sec. 5): a path may read no more columns of an
     // intermediate than the layer before wrote for that path (the columns beyond hold stale workspace bytes)
     for (int t = 0; t < L->T; ++t) {
@@ -543,7 +655,7 @@ int plan_layer(const dsn_layer_desc* L, LayerPlan& pl) {
   pl.off_buf[0] = take(need[0]);
   pl.off_buf[1] = take(need[1]);
   // a physical gather pays when a sample has too few rows to fill a 128-row tile on its own
-  pl.gather_first = first.dtype == DSN_BF16 && first.H * first.W <= 64;
+  pl.gather_first = first.dtype == DSN_BF16 && first.H * first.W <= 64 && !first.dw;
   pl.off_gather = take(pl.gather_first ? B * (size_t)(first.H * first.W) * (size_t)first.C_in * pl.elem : 0);
   pl.total = off;
   return DSN_OK;
@@ -588,6 +700,10 @@ int dsn_create(dsn_ctx** out, int device) {
     c->gemm_mode = (m && strcmp(m, "1cta") == 0) ? 1 : 0;
     const char* cv = getenv("DSN_CONV3X3");  // "taps": 3x3 layers load the tile once per tap (for comparisons)
     c->conv_halo = (cv && strcmp(cv, "taps") == 0) ? 0 : 1;
+    const char* mc = getenv("DSN_MAP_CACHE");  // "0": encode every tensor map anew on every call (for comparisons)
+    if (!(mc && mc[0] == '0')) c->map_cache = static_cast<dsn_map_slot*>(calloc(DSN_MAP_CACHE_SLOTS, sizeof(dsn_map_slot)));
+    const char* dp = getenv("DSN_DWPW");  // "fused": a depthwise element and the 1x1 layer after it run as one kernel
+    c->dwpw_fused = (dp && strcmp(dp, "fused") == 0) ? 1 : 0;
     const char* ch = getenv("DSN_CHAIN");  // "0": one launch per layer even for small batches (for comparisons)
     c->chain_mode = (ch && ch[0] == '0') ? 0 : 1;
   }
@@ -609,6 +725,7 @@ int dsn_create(dsn_ctx** out, int device) {
 int dsn_destroy(dsn_ctx* ctx) {
   if (!ctx) return DSN_ERR_INVALID_ARG;
   cudaFree(ctx->d_status);
+  free(ctx->map_cache);
   free(ctx);
   return DSN_OK;
 }
@@ -635,6 +752,13 @@ int dsn_set_wait_limit(dsn_ctx* ctx, uint32_t microseconds, void* stream) {
                       s) != cudaSuccess)
     return DSN_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return DSN_ERR_CUDA;
+  return DSN_OK;
+}
+
+int dsn_map_cache_stats(dsn_ctx* ctx, uint64_t* hits, uint64_t* misses) {
+  if (!ctx) return DSN_ERR_INVALID_ARG;
+  if (hits) *hits = ctx->map_hits;
+  if (misses) *misses = ctx->map_misses;
   return DSN_OK;
 }
 
@@ -796,17 +920,9 @@ int dsn_sliced_conv(dsn_ctx* ctx, const dsn_conv_desc* d, const dsn_routing* r, 
 
 int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_routing* r, const void* x, void* y,
                          void* stream) {
-  if (!d || !x || !y || !d->W || !d->c || !d->ksize) return DSN_ERR_INVALID_ARG;
+  if (!x || !y) return DSN_ERR_INVALID_ARG;
   if (int e0 = check_ctx(ctx)) return e0;
-  if (d->dtype != DSN_BF16) return DSN_ERR_UNSUPPORTED;
-  if (d->H < 1 || d->W_ < 1 || d->C < 1 || d->C > 32767 || d->K < 1 || d->K > 7 || d->K % 2 == 0) return DSN_ERR_INVALID_ARG;
-  if (d->stride != 1 && d->stride != 2) return DSN_ERR_UNSUPPORTED;
-  if (d->ldx < d->C || d->ldy < d->C || d->T < 1 || d->T > DSN_MAX_SLICES) return DSN_ERR_INVALID_ARG;
-  if (d->act < DSN_ACT_NONE || d->act > DSN_ACT_GELU) return DSN_ERR_INVALID_ARG;
-  if ((d->bn_scale == nullptr) != (d->bn_shift == nullptr)) return DSN_ERR_INVALID_ARG;
-  for (int t = 0; t < d->T; ++t)
-    if (d->c[t] < 1 || d->c[t] > d->C || d->ksize[t] < 1 || d->ksize[t] > d->K || d->ksize[t] % 2 == 0)
-      return DSN_ERR_INVALID_ARG;
+  if (int e1 = check_depthwise(d)) return e1;
   int e = check_routing(r, d->T);
   if (e) return e;
   if (dsn_launch_depthwise(d->c, d->ksize, d->T, d->H, d->W_, d->K, d->stride, d->C, r->B, r->G, r->offsets, r->perm,
@@ -887,7 +1003,9 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
                            : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
     void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
-    if (!c.att) {
+    if (c.dw) {
+      e = (!aligned16(in) || c.ldx % 8) ? DSN_ERR_ALIGNMENT : check_routing(&r, c.T);
+    } else if (!c.att) {
       e = validate_call(c, &r, in, out);
     } else {  // the attention core between two layers: dense grouped intermediates
       dsn_attention_desc a = *c.att;
@@ -937,7 +1055,21 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
     const void* in = first ? (pl.gather_first ? (const void*)(ws + pl.off_gather) : x)
                            : (const void*)(ws + pl.off_buf[(j - 1) & 1]);
     void* out = last ? y : (void*)(ws + pl.off_buf[j & 1]);
-    if (calls[j].att) {
+    if (calls[j].dw) {
+      if (L->B > 0 && ctx->dwpw_fused && dwpw_fusable(calls[j], calls[j + 1], in)) {
+        // the separable block as one kernel: the depthwise result goes from registers to the tensor core's operand tile
+        void* out2 = j + 2 == L->n_layers ? y : (void*)(ws + pl.off_buf[(j + 1) & 1]);
+        e = run_dwpw(ctx, calls[j], calls[j + 1], &r, in, out2, s);
+        ++j;
+      } else {
+        dsn_depthwise_desc d2 = *calls[j].dw;
+        d2.in_order = calls[j].in_order;
+        d2.out_order = DSN_GROUPED;
+        d2.ldx = calls[j].ldx;
+        d2.ldy = calls[j].C_out;
+        e = dsn_sliced_depthwise(ctx, &d2, &r, in, out, stream);
+      }
+    } else if (calls[j].att) {
       dsn_attention_desc a = *calls[j].att;
       a.ld_qkv = calls[j].C_in;   // dense grouped intermediates
       a.ld_out = calls[j].C_out;

@@ -15,6 +15,23 @@
 #define DSN_STATUS_REPORT_WORDS 4
 #define DSN_STATUS_WAIT_US 4
 
+// Tensor-map cache: encoding a map on the host costs about a microsecond and a layer needs up to three per distinct
+// slice, on every call.  Maps depend only on (base pointer, extents, strides, box), so a context keeps the ones it
+// has built in a small direct-mapped table; serving loops that call with the same buffers hit it every time.
+#define DSN_MAP_CACHE_SLOTS 512
+struct dsn_map_key {
+  const void* base;
+  uint64_t dims[4];
+  uint64_t strides[3];
+  uint32_t box[4];
+  uint32_t rank;
+};
+struct dsn_map_slot {
+  dsn_map_key key;
+  CUtensorMap map;
+  int used;
+};
+
 struct dsn_ctx {
   int device;
   int sm_count;
@@ -23,7 +40,11 @@ struct dsn_ctx {
   int gemm_mode;       // 0 = CTA pairs where possible (default), 1 = one CTA per tile (DSN_GEMM_MODE=1cta)
   int conv_halo;       // 1 = 3x3 layers stage the input tile once with its halo (default), 0 = one load per tap (DSN_CONV3X3=taps)
   int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
+  int dwpw_fused;      // 1 = depthwise + following 1x1 layer as one kernel (DSN_DWPW=fused); default 0: measured slower than the
+                       //     two launches, because four producer warps on plain ALUs cannot keep up with the tensor core
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
+  dsn_map_slot* map_cache;   // DSN_MAP_CACHE_SLOTS slots (host memory), or nullptr when the cache is off (DSN_MAP_CACHE=0)
+  uint64_t map_hits, map_misses;
   uint32_t wait_limit_us;  // staging copy of the wait limit (source of the asynchronous copy into the status block)
 };
 
@@ -146,6 +167,23 @@ struct GemmParams {
   int32_t act;
   int32_t* status;
 };
+
+// Depthwise k x k fused into the pointwise GEMM that follows it: `g` describes the pointwise layer (flat tiling over
+// the grouped output pixels, R = Ho * Wo rows per sample; mapA is unused), the rest the depthwise producer.
+struct DwPwParams {
+  GemmParams g;
+  const __nv_bfloat16* x;   // block input [sample][H][W][ldx], order given by g.g.a_input_order
+  int64_t ldx;
+  const __nv_bfloat16* w;   // depthwise filter [K][K][C]
+  const float* dw_bias;
+  const float* dw_bn_scale; // [T][C] or nullptr
+  const float* dw_bn_shift;
+  int32_t dw_act;
+  int32_t H, W, Wo, K, stride, C;
+  int8_t ksize[DSN_MAX_SLICES];
+};
+size_t dsn_dwpw_smem_bytes(int BN, int stages, int G);
+cudaError_t dsn_launch_dwpw(const DwPwParams& q, int sm_count, size_t smem_bytes, cudaStream_t s);
 
 // A chain of up to three sliced layers run by one launch (every layer tiled per sample, CTA pairs).
 #define DSN_CHAIN_MAX_LAYERS 3

@@ -241,6 +241,32 @@ def test_host_side_argument_errors_launch_nothing(dsn, ctx):
     check_status(ctx, dsn)
 
 
+def test_tensor_maps_are_encoded_once_per_buffer_and_slice(dsn):
+    """Repeated calls on the same buffers reuse the context's cached tensor maps (no misses after the first call) and
+    give the same bytes; another output buffer misses only for the maps that name it."""
+    c = dsn.Context(0)
+    g = np.random.default_rng(9)
+    B, R, C, T = 20, 50, 192, 4
+    k_in, k_out = [64, 128, 192, 192], [192, 64, 128, 192]
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    r = route_on_gpu(dsn, c, idx, T)
+    x, W = up_bf16(wl.normal(g, (B, R, C))), up_bf16(wl.normal(g, (C, C), std=C ** -0.5))
+    d = dsn.make_linear_desc(dsn.BF16, R, C, C, k_in, k_out, W)
+    y1 = torch.zeros((B, R, C), dtype=torch.bfloat16, device=DEV)
+    y2 = torch.zeros((B, R, C), dtype=torch.bfloat16, device=DEV)
+    dsn.dsn_sliced_linear(c, d, r, x, y1)
+    h0, m0 = c.map_cache_stats()
+    assert m0 > 0
+    dsn.dsn_sliced_linear(c, d, r, x, y1)
+    h1, m1 = c.map_cache_stats()
+    assert m1 == m0 and h1 - h0 == m0 + h0                 # every map of the second call came from the cache
+    dsn.dsn_sliced_linear(c, d, r, x, y2)
+    h2, m2 = c.map_cache_stats()
+    assert 0 < m2 - m1 < m0                                # only the output maps are new
+    check_status(c, dsn)
+    assert torch.equal(y1, y2)
+
+
 def test_layer_forward_rejects_a_layer_that_reads_more_than_was_written(dsn, ctx):
     """All layers of a block inherit one decision: a path may not read more columns of an intermediate than
     the layer before wrote for it (those columns hold stale workspace bytes).  Refused on the host."""
