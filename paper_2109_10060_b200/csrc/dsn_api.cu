@@ -280,7 +280,9 @@ int fill_gemm_maps(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const
     const uint32_t wb[3] = {DSN_GEMM_BK, 1, (uint32_t)(g.pair ? g.BN / 2 : g.BN)};
     e = encode_map(ctx, &p.mapB[m], c.Wt, 3, wd, ws, wb);
     if (e) return e;
-    const uint64_t yd[2] = {(uint64_t)map_n[m], (uint64_t)r->B * g.R};  // columns clipped at k_out
+    // columns clipped at k_out rounded down to 8 (the store clips at 16-byte granularity; the epilogue writes the 1..7
+    // columns beyond with plain stores); widths below 8 never use the map
+    const uint64_t yd[2] = {(uint64_t)(map_n[m] >= 8 ? (map_n[m] & ~7) : 8), (uint64_t)r->B * g.R};
     const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
     const uint32_t yb[2] = {64, 32};
     e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);

@@ -275,7 +275,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
-      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
 
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
       if (!ok) break;

@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(kDwThreads, 1) dwpw_kernel(const __grid_consta
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
-      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 44));
       if (!ok) break;
       tc_fence_after();

@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_kernel(const __grid_con
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
       // (a slice width that is no multiple of 8 columns = 16 bytes keeps the element-wise path: the
       // store was seen to clip the row at 16-byte granularity and would touch columns >= k_out)
-      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
 
       // every lane waits, then the warp takes one decision so that tcgen05.ld stays warp-wide
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 4));

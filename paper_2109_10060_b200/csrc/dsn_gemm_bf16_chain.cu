@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
       // TMA stores only where nobody waits for them: their completion (needed before the sample's next
       // layer may read the rows) takes several microseconds, plain stores followed by a release do not
-      const bool contig = l + 1 == cp.n_layers && __all_sync(0xffffffffu, valid && out_row == base_row + lane) && (t.ko & 7) == 0;
+      const bool contig = l + 1 == cp.n_layers && __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
       const bool any_valid = __any_sync(0xffffffffu, valid);
 
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, status, 35));

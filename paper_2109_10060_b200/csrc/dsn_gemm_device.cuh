@@ -177,6 +177,28 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Packed fp32 pairs (two lanes per 64-bit register) and the three-input maximum.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(p)); }
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 // erf(z) ~= tanh(c1 z + c3 z^3 + c5 z^5): coefficients fitted by least squares so that the GELU built
 // on it stays within 3e-5 (absolute) of the exact erf form for every x; evaluated with the hardware
 // tanh (relative error <= 2^-11), i.e. one special-function instruction per element instead of the
@@ -268,11 +290,31 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
       }
     }
     if (contig) {
+      // The store's tensor map ends at the slice width rounded DOWN to 8 columns (a TMA store clips at 16-byte
+      // granularity); a width that is no multiple of 8 leaves 1..7 columns, which every lane writes for its own row.
       fence_async_smem();
       __syncwarp();
       if (elect_one()) {
         tma_store_2d(mapY, n0 + c0, base_row, smem_u32(stage_w));
         bulk_commit();
+      }
+      const int col8 = ncols & ~7, tail_n = ncols & 7;
+      if (tail_n != 0 && col8 >= c0 && col8 < c0 + 64) {
+        const int j = (col8 - c0) >> 3;
+        const uint4 val = *reinterpret_cast<const uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4));
+        const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+        __nv_bfloat16* dst = yrow + col8;
+        if ((reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+          int off = 0;
+          if (tail_n & 4) { *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]); off = 4; }
+          if (tail_n & 2) { *reinterpret_cast<uint32_t*>(dst + off) = w[off >> 1]; off += 2; }
+          if (tail_n & 1) reinterpret_cast<uint16_t*>(dst)[off] = (uint16_t)(w[off >> 1] & 0xffffu);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (e < tail_n)
+              reinterpret_cast<uint16_t*>(dst)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
+        }
       }
       continue;
     }
@@ -292,12 +334,22 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
         const uint4 val = *reinterpret_cast<const uint4*>(stage_w + row * 128 + ((j ^ (row & 7)) << 4));
         if (col + 8 <= ncols) {
           *reinterpret_cast<uint4*>(rp[i] + col) = val;
-        } else {  // slice width not a multiple of 8: the last few columns one by one
+        } else {  // slice width not a multiple of 8: the 1..7 columns left leave as one 8-, one 4- and one 2-byte store
+          // (the piece starts on a 16-byte boundary of the row whenever the row itself does; an odd start falls back to 2-byte stores)
           const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+          const int n = ncols - col;
+          __nv_bfloat16* dst = rp[i] + col;
+          if ((reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+            int off = 0;
+            if (n & 4) { *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]); off = 4; }
+            if (n & 2) { *reinterpret_cast<uint32_t*>(dst + off) = w[off >> 1]; off += 2; }
+            if (n & 1) reinterpret_cast<uint16_t*>(dst)[off] = (uint16_t)(w[off >> 1] & 0xffffu);
+          } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (col + e < ncols)
-              reinterpret_cast<uint16_t*>(rp[i] + col)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
+            for (int e = 0; e < 8; ++e)
+              if (e < n)
+                reinterpret_cast<uint16_t*>(dst)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
+          }
         }
       }
     }
