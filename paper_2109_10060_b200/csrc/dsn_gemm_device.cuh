@@ -213,6 +213,24 @@ __device__ __forceinline__ float erf_fast(float z) {
   return t;
 }
 
+// The same GELU for two values at once with packed fp32 arithmetic (two lanes per instruction): the epilogue is bound
+// by instruction issue, not by a pipe, and this form needs 6 packed instructions and 2 tanh for a pair where the
+// scalar form needs 16 and 2 (measured: cfg3 fc1 57.4 -> 53.5 us, cfg5 fc1 on the narrowest path 203 -> 188 us).  0.5 v (1 + t) is evaluated as h + h t with h = v / 2.
+__device__ __forceinline__ void gelu_pair(float a, float b, float& ra, float& rb) {
+  // erf(v / sqrt 2) ~= tanh(v (k1 + k3 v^2 + k5 v^4)) with the 1 / sqrt 2 folded into the coefficients of erf_fast
+  const uint64_t zero2 = pack2(0.f, 0.f);
+  const uint64_t v2 = pack2(a, b);
+  const uint64_t z2 = ffma2(v2, v2, zero2);
+  uint64_t q = ffma2(z2, pack2(-0.00035873294f, -0.00035873294f), pack2(0.037050344f, 0.037050344f));
+  q = ffma2(z2, q, pack2(0.79745847f, 0.79745847f));
+  float u0, u1, t0, t1;
+  unpack2(ffma2(v2, q, zero2), u0, u1);
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(u0));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(u1));
+  const uint64_t h2 = ffma2(v2, pack2(0.5f, 0.5f), zero2);
+  unpack2(ffma2(h2, pack2(t0, t1), h2), ra, rb);
+}
+
 // The activation (and whether any per-column affine term exists) is a template parameter so that the
 // per-element loop holds no trace of the other variants: an if-converted erf or a few unused loads per
 // element are enough to put the epilogue behind the main loop.
@@ -281,7 +299,9 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
                 else if (RES && res_row) b += __bfloat162float(res_row[cb + c + 1]);
               }
             }
-            __nv_bfloat162 h = __floats2bfloat162_rn(apply_act<ACT>(a), apply_act<ACT>(b));
+            if (ACT == DSN_ACT_GELU) gelu_pair(a, b, a, b);
+            else { a = apply_act<ACT>(a); b = apply_act<ACT>(b); }
+            __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
             w[e] = *reinterpret_cast<uint32_t*>(&h);
           }
           const int j = 4 * half + jj;
