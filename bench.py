@@ -692,12 +692,35 @@ def collect_rows(dsn, torch, ctx, dev, peaks, timer, row_filter=None, batch_div=
         if emit:
             emit(row)
 
-    def gemm_row(cfgname, lname, rname, B, us, flops, byts):
+    def gemm_row(cfgname, lname, rname, B, us, flops, byts, floor_util=None):
         tf = flops / us / 1e6
         bound = min(PEAK, flops / byts * HBM / 1e3)
-        add({"config": cfgname, "layer": lname, "routing": rname, "us": round(us, 1), "tflops": round(tf, 1),
-             "pct_bf16_peak": round(100 * tf / PEAK, 1), "bound_tflops": round(bound), "pct_of_bound": round(100 * tf / bound),
-             "gbs": round(byts / us / 1e3), "samples_per_s": round(B / us * 1e6)})
+        row = {"config": cfgname, "layer": lname, "routing": rname, "us": round(us, 1), "tflops": round(tf, 1),
+               "pct_bf16_peak": round(100 * tf / PEAK, 1), "bound_tflops": round(bound), "pct_of_bound": round(100 * tf / bound),
+               "gbs": round(byts / us / 1e3), "samples_per_s": round(B / us * 1e6)}
+        if floor_util is not None and floor_util < 0.995:
+            # a tcgen05.mma of N columns occupies the tensor pipe for max(59, N / 2) cycles (measured): narrow slices
+            # cannot use more than this share of the peak, whatever the kernel does
+            fb = min(bound, PEAK * floor_util)
+            row["bound_with_mma_floor_tflops"] = round(fb)
+            row["pct_of_bound_with_mma_floor"] = round(100 * tf / fb)
+        add(row)
+
+    def mma_floor_util(counts, R, k_in, k_out, K):
+        """Share of the tensor peak the executed FLOPs can reach when every instruction of N < 118 columns still
+        occupies the pipe for 59 cycles: FLOP-weighted over the slices and their n-tiles."""
+        bn = 256 if max(k_out) > 128 else (128 if max(k_out) > 64 else 64)
+        fl = tm = 0.0
+        for t, n in enumerate(counts):
+            if not n:
+                continue
+            for n0 in range(0, k_out[t], bn):
+                cols = min(bn, k_out[t] - n0)
+                n_inst = min(bn, (cols + 31) // 32 * 32)
+                f = float(n) * R * k_in[t] * cols * K * K
+                fl += f
+                tm += f / cols * n_inst / ((n_inst / 2) / max(59.0, n_inst / 2))   # issued columns / pipe share
+        return fl / tm if tm else 1.0
 
     def routed(B, T, idx):
         r = dsn.make_routing(B, T, ints(np.zeros(T)), ints(np.zeros(T + 1)), ints(np.zeros(B)), ints(np.zeros(B)))
@@ -733,7 +756,8 @@ def collect_rows(dsn, torch, ctx, dev, peaks, timer, row_filter=None, batch_div=
         assert code == 0, code
         counts = np.bincount(idx, minlength=T)
         flops = 2 * dsn.dsn_executed_macs(counts.tolist(), R, k_in, k_out, K)
-        gemm_row(cfgname, lname, rname, B, us, flops, gemm_algorithmic_bytes(counts, R, k_in, k_out, K))
+        gemm_row(cfgname, lname, rname, B, us, flops, gemm_algorithmic_bytes(counts, R, k_in, k_out, K),
+                 mma_floor_util(counts, R, k_in, k_out, K))
         del xs, ys
 
     def gate_route(cfgname, B, R, C, T):
