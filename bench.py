@@ -952,6 +952,9 @@ def main():
         if code != 0:
             raise SystemExit(f"device status {code} ({dsn.dsn_strerror(code)}) detail {detail}")
 
+    launches0 = ctx.stats()["launches"]
+    wlk.step(ctx, 0)
+    launches_per_step = ctx.stats()["launches"] - launches0   # counted by the library itself, one direct step
     t_host0 = time.perf_counter()
     for i in range(args.warmup):
         wlk.step(ctx, i)
@@ -1141,7 +1144,9 @@ def main():
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(hx.numel() * 2),
                 "d2h_bytes_per_step": int(hy.numel() * 2), "ms_per_step": ms_e2e,
                 "how": "the public-API step per batch; upload, compute and download pipelined on three streams"},
-        "gpu_launches": wlk.kernels_per_step * timed_steps,
+        "gpu_launches": launches_per_step * timed_steps,
+        "gpu_launches_per_step": launches_per_step,
+        "library_stats": ctx.stats(),
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:

@@ -224,6 +224,27 @@ int dsn_selftest_bounded_wait(dsn_ctx* ctx, void* stream);
  * Returns the hit and miss counts since the context was created. */
 int dsn_map_cache_stats(dsn_ctx* ctx, uint64_t* hits, uint64_t* misses);
 
+/* What a context has launched since it was created (host-side counters; kernels of this library only).  With
+ * DSN_LOG=1 in the environment at dsn_create, every sliced-layer and dsn_layer_forward call also writes one line to
+ * stderr. */
+typedef struct dsn_stats {
+  uint64_t calls;                 /* sliced-layer and dsn_layer_forward calls                              */
+  uint64_t launches;              /* kernels launched, all families                                        */
+  uint64_t launches_gemm_pair;    /* grouped GEMM on CTA pairs                                             */
+  uint64_t launches_gemm_halo;    /* 3x3 layers, halo form                                                 */
+  uint64_t launches_gemm_chain;   /* a block's layers as one launch                                        */
+  uint64_t launches_gemm_one_cta; /* grouped GEMM, one CTA per tile                                        */
+  uint64_t launches_linear_f32;
+  uint64_t launches_attention;
+  uint64_t launches_depthwise;
+  uint64_t launches_dwpw;         /* depthwise + pointwise as one kernel                                   */
+  uint64_t launches_gate;         /* pooling, hidden layer, scores (3 per gate), attention head            */
+  uint64_t launches_route;
+  uint64_t launches_copy;         /* gather / scatter, zero fill, channel scaling, Re-SBN folding          */
+  uint64_t map_hits, map_misses;  /* tensor-map cache                                                      */
+} dsn_stats;
+int dsn_get_stats(dsn_ctx* ctx, dsn_stats* out);
+
 /* Ratio list -> channel counts (host only).  granule g = 0 picks g = min(8, C/32);
  * k = g*floor(r*C/g + 1/2) clamped to [g, C].  The paper lists channel counts, not a rounding
  * rule; this rule reproduces its DS-MBNet list 224..640 step 32 from ratios 0.35..1.0. */

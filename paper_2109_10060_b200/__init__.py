@@ -5,5 +5,5 @@ There is no CPU or framework fallback: calling any compute entry point without t
 CUDA library raises ImportError.
 """
 from .binding import *  # noqa: F401,F403
-from .binding import (Context, DsnError, EXPORTS, LIB_PATH, Routing, GateDesc, LinearDesc, ConvDesc, LayerDesc, AttentionDesc, DepthwiseDesc,
+from .binding import (Context, DsnError, EXPORTS, LIB_PATH, Routing, GateDesc, LinearDesc, ConvDesc, LayerDesc, AttentionDesc, DepthwiseDesc, Stats,
                       load_library)

@@ -24,7 +24,7 @@ LAYER_LINEAR, LAYER_CONV, LAYER_ATTENTION, LAYER_DEPTHWISE = 0, 1, 2, 3
 MAX_SLICES, MAX_GROUPS, MAX_CHAIN = 64, 4096, 6
 
 EXPORTS = [
-    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_set_wait_limit", "dsn_selftest_bounded_wait", "dsn_map_cache_stats", "dsn_widths_from_ratios",
+    "dsn_create", "dsn_destroy", "dsn_strerror", "dsn_get_status", "dsn_set_wait_limit", "dsn_selftest_bounded_wait", "dsn_map_cache_stats", "dsn_get_stats", "dsn_widths_from_ratios",
     "dsn_executed_macs", "dsn_gate_workspace_bytes", "dsn_gate", "dsn_gate_static", "dsn_gate_attention", "dsn_scale_channels", "dsn_resbn_fold", "dsn_route", "dsn_permute_rows",
     "dsn_sliced_attention", "dsn_sliced_depthwise", "dsn_linear_workspace_bytes", "dsn_conv_workspace_bytes", "dsn_sliced_linear", "dsn_sliced_conv",
     "dsn_layer_workspace_bytes", "dsn_layer_forward",
@@ -78,6 +78,13 @@ class DepthwiseDesc(C.Structure):
                 ("out_order", C.c_int32)]
 
 
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("calls", "launches", "launches_gemm_pair", "launches_gemm_halo", "launches_gemm_chain",
+                                          "launches_gemm_one_cta", "launches_linear_f32", "launches_attention",
+                                          "launches_depthwise", "launches_dwpw", "launches_gate", "launches_route",
+                                          "launches_copy", "map_hits", "map_misses")]
+
+
 class LayerDesc(C.Structure):
     _fields_ = [("gate", C.POINTER(GateDesc)), ("B", C.c_int32), ("T", C.c_int32), ("n_layers", C.c_int32),
                 ("kind", C.c_int32 * MAX_CHAIN), ("layer", C.c_void_p * MAX_CHAIN)]
@@ -103,6 +110,7 @@ def load_library():
     lib.dsn_get_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
     lib.dsn_set_wait_limit.argtypes = [vp, C.c_uint32, vp]
     lib.dsn_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.dsn_get_stats.argtypes = [vp, C.POINTER(Stats)]
     lib.dsn_map_cache_stats.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.dsn_widths_from_ratios.argtypes = [i32, C.POINTER(C.c_double), i32, i32, C.POINTER(i32)]
     lib.dsn_executed_macs.argtypes = [C.POINTER(i32), i32, i32, C.POINTER(i32), C.POINTER(i32), i32]
@@ -204,6 +212,12 @@ class Context:
         h, m = C.c_uint64(), C.c_uint64()
         _check(self.lib.dsn_map_cache_stats(self.handle, C.byref(h), C.byref(m)), "dsn_map_cache_stats")
         return h.value, m.value
+
+    def stats(self) -> dict:
+        """Launch counters of this context (kernels of the library, by family)."""
+        st = Stats()
+        _check(self.lib.dsn_get_stats(self.handle, C.byref(st)), "dsn_get_stats")
+        return {n: int(getattr(st, n)) for n, _ in Stats._fields_}
 
     def get_status(self, stream=None):
         code, detail = C.c_int32(), C.c_int32()

@@ -32,6 +32,15 @@ int check_ctx(const dsn_ctx* ctx) {
   return cur == ctx->device ? DSN_OK : DSN_ERR_INVALID_ARG;
 }
 
+// Launch counters and the optional call log (DSN_LOG=1: one line per launch family on stderr).
+void count_launch(dsn_ctx* ctx, uint64_t dsn_stats::*field, uint64_t n = 1) {
+  ctx->stats.*field += n;
+  ctx->stats.launches += n;
+}
+void log_call(const dsn_ctx* ctx, const char* what, long long B, long long T) {
+  if (ctx && ctx->log) fprintf(stderr, "[dsn] %s B=%lld T=%lld launches so far %llu\n", what, B, T, (unsigned long long)ctx->stats.launches);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
@@ -339,6 +348,7 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
       while (remaining_h > 0) {
         const int e = fill_gemm_maps(ctx, c, r, x, y, p, done_h, remaining_h);
         if (e) return e;
+        count_launch(ctx, &dsn_stats::launches_gemm_halo);
         if (dsn_launch_gemm_bf16_halo(p, clusters_h, smem_h, s) != cudaSuccess) return DSN_ERR_CUDA;
       }
       return DSN_OK;
@@ -367,8 +377,8 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
     const int e = fill_gemm_maps(ctx, c, r, x, y, p, done, remaining);
     if (e) return e;
     if (g.pair) {
-      if (dsn_launch_gemm_bf16_pair(p, clusters, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
-    } else if (dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) {
+      if (count_launch(ctx, &dsn_stats::launches_gemm_pair), dsn_launch_gemm_bf16_pair(p, clusters, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
+    } else if (count_launch(ctx, &dsn_stats::launches_gemm_one_cta), dsn_launch_gemm_bf16(p, ctx->sm_count, smem, s) != cudaSuccess) {
       return DSN_ERR_CUDA;
     }
   }
@@ -421,6 +431,7 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
   cp.n_layers = n;
   cp.stages = stages;
   cp.bn_max = bn_max;
+  count_launch(ctx, &dsn_stats::launches_gemm_chain);
   if (dsn_launch_gemm_bf16_chain(cp, clusters, dsn_gemm_chain_smem_bytes(bn_max, stages, r->G), s) != cudaSuccess)
     return DSN_ERR_CUDA;
   return 1;
@@ -469,6 +480,7 @@ int run_dwpw(dsn_ctx* ctx, const LayerCall& d, const LayerCall& c, const dsn_rou
     const int e = fill_gemm_maps(ctx, cc, r, y /* stands in for the activation map, which this kernel does not use */, y,
                                  q.g, done, remaining);
     if (e) return e;
+    count_launch(ctx, &dsn_stats::launches_dwpw);
     if (dsn_launch_dwpw(q, ctx->sm_count, smem, s) != cudaSuccess) return DSN_ERR_CUDA;
   }
   return DSN_OK;
@@ -477,6 +489,8 @@ int run_dwpw(dsn_ctx* ctx, const LayerCall& d, const LayerCall& c, const dsn_rou
 int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void* x, void* y, cudaStream_t s) {
   int e = check_ctx(ctx);
   if (e) return e;
+  ++ctx->stats.calls;
+  log_call(ctx, c.K == 1 ? "sliced layer (1x1 / linear)" : "sliced layer (3x3)", r ? r->B : -1, c.T);
   e = validate_call(c, r, x, y);
   if (e) return e;
   if (r->B == 0) return DSN_OK;
@@ -486,6 +500,7 @@ int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void
     e = run_bf16(ctx, c, r, x, y, s);
     if (e) return e;
   } else {
+    count_launch(ctx, &dsn_stats::launches_linear_f32);
     if (dsn_launch_linear_f32(st, c.T, c.H * c.W, static_cast<const float*>(x), c.ldx,
                               static_cast<const float*>(c.Wt), c.w_row, static_cast<float*>(y), c.ldy, c.bias, c.bn_scale, c.bn_shift,
                               c.C_out, static_cast<const float*>(c.residual), c.act,
@@ -494,6 +509,7 @@ int run_layer(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void
       return DSN_ERR_CUDA;
   }
   if (c.tail == DSN_TAIL_ZERO) {
+    count_launch(ctx, &dsn_stats::launches_copy);
     if (dsn_launch_zero_tail(st, c.dtype == DSN_BF16 ? 2 : 4, c.H * c.W, c.C_out, y, c.ldy,
                              c.out_order == DSN_INPUT_ORDER, r->B, r->G, r->offsets, r->perm, r->group_slice,
                              s) != cudaSuccess)
@@ -702,6 +718,8 @@ int dsn_create(dsn_ctx** out, int device) {
     c->gemm_mode = (m && strcmp(m, "1cta") == 0) ? 1 : 0;
     const char* cv = getenv("DSN_CONV3X3");  // "taps": 3x3 layers load the tile once per tap (for comparisons)
     c->conv_halo = (cv && strcmp(cv, "taps") == 0) ? 0 : 1;
+    const char* lg = getenv("DSN_LOG");  // "1": one line per entry-point call on stderr
+    c->log = (lg && lg[0] == '1') ? 1 : 0;
     const char* mc = getenv("DSN_MAP_CACHE");  // "0": encode every tensor map anew on every call (for comparisons)
     if (!(mc && mc[0] == '0')) c->map_cache = static_cast<dsn_map_slot*>(calloc(DSN_MAP_CACHE_SLOTS, sizeof(dsn_map_slot)));
     const char* dp = getenv("DSN_DWPW");  // "fused": a depthwise element and the 1x1 layer after it run as one kernel
@@ -764,6 +782,14 @@ int dsn_map_cache_stats(dsn_ctx* ctx, uint64_t* hits, uint64_t* misses) {
   return DSN_OK;
 }
 
+int dsn_get_stats(dsn_ctx* ctx, dsn_stats* out) {
+  if (!ctx || !out) return DSN_ERR_INVALID_ARG;
+  ctx->stats.map_hits = ctx->map_hits;
+  ctx->stats.map_misses = ctx->map_misses;
+  *out = ctx->stats;
+  return DSN_OK;
+}
+
 int dsn_selftest_bounded_wait(dsn_ctx* ctx, void* stream) {
   if (int e = check_ctx(ctx)) return e;
   return dsn_launch_selftest_wait(ctx->d_status, as_stream(stream)) == cudaSuccess ? DSN_OK : DSN_ERR_CUDA;
@@ -814,6 +840,7 @@ int dsn_gate(dsn_ctx* ctx, const dsn_gate_desc* g, const void* x, int32_t* idx_o
   const size_t need = ((size_t)g->B * splits * g->c_valid + (size_t)g->B * g->C_mlp) * sizeof(float);
   if (!workspace || ws_bytes < need) return DSN_ERR_WORKSPACE;
   if (!aligned16(workspace)) return DSN_ERR_ALIGNMENT;
+  count_launch(ctx, &dsn_stats::launches_gate, 3);  // pool, hidden layer, scores
   if (dsn_launch_gate(*g, x, idx_out, logits_out, static_cast<float*>(workspace), splits, ctx->d_status,
                       as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
@@ -830,6 +857,7 @@ int dsn_gate_attention(dsn_ctx* ctx, const dsn_gate_desc* g, const float* W3, co
   if ((size_t)4 * 4 * g->C_mlp > 48 * 1024) return DSN_ERR_UNSUPPORTED;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
   const float* hid = static_cast<const float*>(workspace) + (size_t)g->B * splits * g->c_valid;
+  count_launch(ctx, &dsn_stats::launches_gate);
   if (dsn_launch_gate_attention(*g, hid, W3, b3, scale_out, as_stream(stream)) != cudaSuccess) return DSN_ERR_CUDA;
   return DSN_OK;
 }
@@ -847,6 +875,7 @@ int dsn_scale_channels(dsn_ctx* ctx, const dsn_routing* r, int32_t to_grouped, i
     if (x == y) return DSN_ERR_INVALID_ARG;  // a permutation cannot run in place
     perm = r->perm;
   }
+  count_launch(ctx, &dsn_stats::launches_copy);
   if (dsn_launch_scale_channels(dtype == DSN_BF16 ? 2 : 4, B, R, c_valid, x, ldx, scale, y, ldy, perm,
                                 as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
@@ -858,6 +887,7 @@ int dsn_resbn_fold(dsn_ctx* ctx, int32_t T, int32_t C, const float* gamma, const
   if (T < 1 || T > DSN_MAX_SLICES || C < 1 || !gamma || !beta || !mu || !sigma || !scale_out || !shift_out)
     return DSN_ERR_INVALID_ARG;
   if (int e = check_ctx(ctx)) return e;
+  count_launch(ctx, &dsn_stats::launches_copy);
   if (dsn_launch_resbn_fold(T * C, C, gamma, beta, mu, sigma, scale_out, shift_out, as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
   return DSN_OK;
@@ -870,6 +900,7 @@ int dsn_route(dsn_ctx* ctx, const int32_t* idx, int32_t B, int32_t T, dsn_routin
   out->B = B;
   out->G = T;
   out->group_slice = nullptr;
+  count_launch(ctx, &dsn_stats::launches_route);
   if (dsn_launch_route(idx, B, T, out->counts, out->offsets, out->perm, out->inv_perm, ctx->d_status,
                        as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
@@ -890,6 +921,7 @@ int dsn_permute_rows(dsn_ctx* ctx, const dsn_routing* r, int32_t dtype, int32_t 
     if (k[t] < 1 || k[t] > ld_src || k[t] > ld_dst) return DSN_ERR_INVALID_ARG;
     st.k_in[t] = k[t];
   }
+  count_launch(ctx, &dsn_stats::launches_copy);
   if (dsn_launch_permute_rows(st, dtype == DSN_BF16 ? 2 : 4, R, src, ld_src, dst, ld_dst, to_grouped ? 1 : 0, r->B,
                               r->G, r->offsets, r->perm, r->group_slice, as_stream(stream)) != cudaSuccess)
     return DSN_ERR_CUDA;
@@ -927,6 +959,7 @@ int dsn_sliced_depthwise(dsn_ctx* ctx, const dsn_depthwise_desc* d, const dsn_ro
   if (int e1 = check_depthwise(d)) return e1;
   int e = check_routing(r, d->T);
   if (e) return e;
+  count_launch(ctx, &dsn_stats::launches_depthwise);
   if (dsn_launch_depthwise(d->c, d->ksize, d->T, d->H, d->W_, d->K, d->stride, d->C, r->B, r->G, r->offsets, r->perm,
                            r->group_slice, d->in_order == DSN_INPUT_ORDER, d->out_order == DSN_INPUT_ORDER, x, d->ldx,
                            d->W, d->bias, d->bn_scale, d->bn_shift, d->act, y, d->ldy, as_stream(stream)) != cudaSuccess)
@@ -955,6 +988,7 @@ int dsn_sliced_attention(dsn_ctx* ctx, const dsn_attention_desc* d, const dsn_ro
   const uint32_t ob[3] = {64, 32, 1};
   e = encode_map(ctx, &map_out, out, 3, od, os, ob);
   if (e) return e;
+  count_launch(ctx, &dsn_stats::launches_attention);
   if (dsn_launch_attention(map, map_out, d->heads, d->T, d->N, d->H, r->B, r->G, d->order == DSN_GROUPED, r->offsets, r->perm,
                            r->group_slice, qkv, d->ld_qkv, out, d->ld_out, ctx->d_status, as_stream(stream)) !=
       cudaSuccess)
@@ -973,6 +1007,8 @@ int dsn_layer_forward(dsn_ctx* ctx, const dsn_layer_desc* L, const void* x, cons
   if (!L || !x || !y) return DSN_ERR_INVALID_ARG;
   int e = check_ctx(ctx);
   if (e) return e;
+  ++ctx->stats.calls;
+  log_call(ctx, "dsn_layer_forward", L->B, L->T);
   LayerPlan pl;
   e = plan_layer(L, pl);
   if (e) return e;

@@ -45,6 +45,8 @@ struct dsn_ctx {
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
   dsn_map_slot* map_cache;   // DSN_MAP_CACHE_SLOTS slots (host memory), or nullptr when the cache is off (DSN_MAP_CACHE=0)
   uint64_t map_hits, map_misses;
+  dsn_stats stats;           // launch counters (dsn_get_stats)
+  int log;                   // 1: DSN_LOG=1
   uint32_t wait_limit_us;  // staging copy of the wait limit (source of the asynchronous copy into the status block)
 };
 

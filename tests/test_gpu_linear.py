@@ -265,6 +265,9 @@ def test_tensor_maps_are_encoded_once_per_buffer_and_slice(dsn):
     assert 0 < m2 - m1 < m0                                # only the output maps are new
     check_status(c, dsn)
     assert torch.equal(y1, y2)
+    st = c.stats()                                          # the library's own launch counters
+    assert st["calls"] == 3 and st["launches_route"] == 1 and st["launches_gemm_pair"] + st["launches_gemm_one_cta"] == 3
+    assert st["launches"] == 4 and st["map_hits"] == h2 and st["map_misses"] == m2
 
 
 def test_layer_forward_rejects_a_layer_that_reads_more_than_was_written(dsn, ctx):

@@ -35,7 +35,7 @@ def test_struct_layouts_match_header_sizes(lib, tmp_path):
     import subprocess
     names = {"dsn_routing": lib.Routing, "dsn_gate_desc": lib.GateDesc, "dsn_linear_desc": lib.LinearDesc,
              "dsn_conv_desc": lib.ConvDesc, "dsn_layer_desc": lib.LayerDesc,
-             "dsn_attention_desc": lib.AttentionDesc, "dsn_depthwise_desc": lib.DepthwiseDesc}
+             "dsn_attention_desc": lib.AttentionDesc, "dsn_depthwise_desc": lib.DepthwiseDesc, "dsn_stats": lib.Stats}
     src = tmp_path / "sizes.c"
     body = "".join(f'printf("{n} %zu\\n", sizeof({n}));' for n in names)
     src.write_text('#include <stdio.h>\n#include "dsn.h"\nint main(void){' + body + "return 0;}\n")
