@@ -244,7 +244,13 @@ def test_host_side_argument_errors_launch_nothing(dsn, ctx):
 def test_tensor_maps_are_encoded_once_per_buffer_and_slice(dsn):
     """Repeated calls on the same buffers reuse the context's cached tensor maps (no misses after the first call) and
     give the same bytes; another output buffer misses only for the maps that name it."""
-    c = dsn.Context(0)
+    import os
+    saved = os.environ.pop("DSN_MAP_CACHE", None)          # the switch is read when the context is created
+    try:
+        c = dsn.Context(0)
+    finally:
+        if saved is not None:
+            os.environ["DSN_MAP_CACHE"] = saved
     g = np.random.default_rng(9)
     B, R, C, T = 20, 50, 192, 4
     k_in, k_out = [64, 128, 192, 192], [192, 64, 128, 192]
