@@ -344,8 +344,8 @@ size_t dsn_layer_workspace_bytes(const dsn_layer_desc* L);
 /* Gate (or the given indices) -> routing -> the block's layers, all layers under the one decision
  * (Sec. 5).  Batches of at most two samples per SM pair whose samples have 150..256 rows (14x14
  * images, 197 tokens) run their 2-3 sliced layers as ONE launch in which every SM pair walks whole
- * samples through the layers; otherwise (and whenever a layer has skip features or the block holds
- * the attention core) one launch per layer.  The two forms agree to within one bfloat16 rounding step of an
+ * samples through the layers (skip features included); otherwise (and whenever the block holds the attention core
+ * or a depthwise element) one launch per layer.  The two forms agree to within one bfloat16 rounding step of an
  * output on a few percent of the elements (the 3x3 layer sums its taps in a different order), not bit for bit.
  * x, y in input order.  idx_in: device [B], required when L->gate is NULL, ignored otherwise.
  * r_out (optional): receives pointers into the workspace holding the block's routing arrays

@@ -397,7 +397,6 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
   for (int j = 0; j < n; ++j) {
     const LayerCall& c = calls[j];
     if (c.att || c.dw || c.dtype != DSN_BF16 || c.tail != DSN_TAIL_UNTOUCHED) return 0;
-    if (c.residual) return 0;  // skip features are added by the single-layer kernels, which prefetch them
     // a sample must fill most of ONE 256-row pair tile: with more rows per sample the single-layer launches
     // (tiles across sample boundaries, halo form of the 3x3 layer) are faster (measured at 28x28 and 56x56)
     if (c.H * c.W < 150 || c.H * c.W > 256) return 0;

@@ -129,7 +129,7 @@ __device__ __forceinline__ void chain_walk(const DsnChainParams& cp, const int32
 // kAff: some layer of the block has a bias or a per-path affine; kGelu: some layer ends in GELU.  A form
 // without one of them holds none of that code: the kernel is sensitive to its own size (each of the two cuts
 // took about 1 us off the bottleneck step).
-template <bool kAff, bool kGelu>
+template <bool kAff, bool kGelu, bool kRes = false>
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __grid_constant__ DsnChainParams cp) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -326,7 +326,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       const float* brow = (kAff && P.bias) ? P.bias + t.n0 : nullptr;
       const float* sc_row = (kAff && P.bn_scale) ? P.bn_scale + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
       const float* sh_row = (kAff && P.bn_scale) ? P.bn_shift + (int64_t)t.slice * P.bn_ld + t.n0 : nullptr;
-      const __nv_bfloat16* res_row = nullptr;  // layers with skip features do not run chained
+      // skip features (only the forms compiled for them carry the code): laid out like the layer's own output
+      const __nv_bfloat16* res_row = (kRes && P.residual && valid) ? P.residual + out_row * P.ldy + t.n0 : nullptr;
       int ncols = t.ko - t.n0;
       ncols = ncols > g.BN ? g.BN : ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
@@ -340,7 +341,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * cp.bn_max);
       const CUtensorMap* mY = &P.mapY[t.map];
-      const int variant = any_valid ? P.act * 2 + ((brow || sc_row) ? 1 : 0) : -1;
+      int variant = any_valid ? P.act * 2 + ((brow || sc_row) ? 1 : 0) : -1;
+      if (kRes && any_valid && P.residual) variant = 6 + P.act;
       switch (variant) {
         case -1: break;  // none of this warp's 32 rows belongs to the sample
         case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
@@ -349,6 +351,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
         case 3: if constexpr (kAff) epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         case 4: if constexpr (kGelu) epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         case 5: if constexpr (kAff && kGelu) epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 6: if constexpr (kRes) epilogue_tile<DSN_ACT_NONE, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 7: if constexpr (kRes) epilogue_tile<DSN_ACT_RELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+        case 8: if constexpr (kRes && kGelu) epilogue_tile<DSN_ACT_GELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
         default: break;
       }
       tc_fence_before();
@@ -380,15 +385,19 @@ size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[4][DSN_MAX_DEVICES] = {};
-  int aff = 0, gelu = 0;
+  static size_t configured[6][DSN_MAX_DEVICES] = {};
+  int aff = 0, gelu = 0, res = 0;
   for (int l = 0; l < cp.n_layers; ++l) {
     aff |= (cp.L[l].bias || cp.L[l].bn_scale) ? 1 : 0;
     gelu |= cp.L[l].act == DSN_ACT_GELU ? 1 : 0;
+    res |= cp.L[l].residual ? 1 : 0;
   }
-  void (*kernel)(DsnChainParams) = aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
-                                       : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
-  const int form = 2 * aff + gelu;
+  // a block with skip features (the residual tail of a DS-ResNet block, Sec. 5) takes the forms that carry that code
+  void (*kernel)(DsnChainParams) =
+      res ? (gelu ? gemm_bf16_chain_kernel<true, true, true> : gemm_bf16_chain_kernel<true, false, true>)
+          : aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
+                : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
+  const int form = res ? 4 + gelu : 2 * aff + gelu;
   {
     cudaError_t e = dsn_ensure_dynamic_smem(kernel, smem_bytes, configured[form]);
     if (e != cudaSuccess) return e;

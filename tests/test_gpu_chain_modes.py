@@ -127,3 +127,48 @@ def test_chained_bottleneck_edge_batches(dsn, B, routing):
     _, _, ref = O.bottleneck(cfg["x"][sel], cfg["W1"], cfg["W2"], cfg["W3"], idx[sel], cfg["widths"], mirror_bf16=True)
     errs = group_errors(got[sel], ref, idx[sel], [cfg["C_outer"]] * T, T)
     assert max(errs.values()) <= 1e-2, errs
+
+
+@pytest.mark.parametrize("B,chained", [(37, True), (37, False), (160, True)], ids=["chained", "per-layer", "large-batch"])
+def test_bottleneck_with_identity_shortcut(dsn, B, chained, parity_report):
+    """The residual tail of a DS-ResNet block (Sec. 5) inside dsn_layer_forward: out = ReLU(conv3(h) + x) with the block
+    input itself as skip features.  Small batches run the three layers as one chained launch, which adds the skip
+    features in its last layer's epilogue; with DSN_CHAIN=0, and for batches beyond two samples per CTA pair, one
+    launch per layer.  All three against the oracle's chain (each stored tensor rounded to bf16)."""
+    saved = os.environ.get("DSN_CHAIN")
+    os.environ["DSN_CHAIN"] = "1" if chained else "0"       # read when the context is created
+    try:
+        ctx = dsn.Context(0)
+    finally:
+        if saved is None:
+            del os.environ["DSN_CHAIN"]
+        else:
+            os.environ["DSN_CHAIN"] = saved
+    cfg = wl.bottleneck(78, B, 14, 14, 256, 64, routing="uniform", with_gate=False)
+    H, Wd, C, Ci, T, widths, idx = cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"], cfg["widths"], cfg["idx"]
+    full = [C] * T
+    x = up_bf16(cfg["x"])
+    W2 = np.ascontiguousarray(np.transpose(cfg["W2"], (0, 2, 3, 1)))
+    layers = [dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, Ci, full, widths, up_bf16(cfg["W1"].reshape(Ci, C)), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 3, 1, Ci, Ci, widths, widths, up_bf16(W2), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, Ci, C, widths, full, up_bf16(cfg["W3"].reshape(C, Ci)), act=dsn.ACT_RELU,
+                                 residual=x)]
+    L = dsn.make_layer_desc(B, T, layers, None)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, H, Wd, C), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    before = ctx.stats()
+    dsn.dsn_layer_forward(ctx, L, x, up_i32(idx), y, ws)
+    code, detail = ctx.get_status()
+    assert code == 0, (code, detail)
+    after = ctx.stats()
+    if chained and B <= 148:
+        assert after["launches_gemm_chain"] - before["launches_gemm_chain"] == 1     # the block ran as one launch
+    else:
+        assert after["launches_gemm_chain"] == before["launches_gemm_chain"]
+    y1 = O.round_bf16(O.sliced_conv(cfg["x"], cfg["W1"], idx, full, widths, 0, act=O.ACT_RELU, fill=0.0))
+    y2 = O.round_bf16(O.sliced_conv(y1, cfg["W2"], idx, widths, widths, 1, act=O.ACT_RELU, fill=0.0))
+    ref = O.sliced_conv(y2, cfg["W3"], idx, widths, full, 0, act=O.ACT_RELU, residual=cfg["x"])
+    errs = group_errors(down(y), ref, idx, full, T)
+    assert max(errs.values()) <= 1e-2, errs
+    parity_report.append(f"bottleneck with identity shortcut, B={B} ({'chained launch' if chained and B <= 148 else 'one launch per layer'}): "
+                         f"worst {max(errs.values()):.2e} (chain bound 1e-02)")
