@@ -34,26 +34,118 @@ __device__ __forceinline__ float act_apply(float v, int act) {
   return v;
 }
 
-__global__ void __launch_bounds__(kThreads) depthwise_kernel(const __grid_constant__ DwParams p) {
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+// eight bf16 (16 bytes) -> four packed fp32 pairs
+__device__ __forceinline__ void widen8(const uint4& v, uint64_t (&o)[4]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) o[j] = pack2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
+}
+
+// 3 x 3 fast path: a thread owns 8 channels of FOUR neighbouring output pixels of one output row.  Per filter row it
+// requests the 3 + 3 * STRIDE input vectors the four windows cover and the row's three filter vectors in one round,
+// widens each once and feeds every window it belongs to (a sliding window in registers): a third of the loads and of
+// the widening work of one pixel per thread, and packed fp32 FMAs (two channels per instruction).
+template <int STRIDE>
+__device__ __forceinline__ void depthwise3x3_rows(const DwParams& p, const __nv_bfloat16* xs, __nv_bfloat16* ys, int ct,
+                                                  const float* sc, const float* sh, int row0, int row1) {
+  constexpr int NCOL = 3 + 3 * STRIDE;
+  const int nvec = ct >> 3, quads = (p.Wo + 3) >> 2;
+  const int k0 = (p.K - 3) >> 1;
+  const int64_t total = (int64_t)(row1 - row0) * quads * nvec;
+  for (int64_t e = threadIdx.x; e < total; e += kThreads) {
+    const int v = (int)(e % nvec);
+    const int qi = (int)(e / nvec);
+    const int oy = row0 + qi / quads, ox0 = 4 * (qi % quads);
+    const int c0 = 8 * v;
+    const int npx = p.Wo - ox0 < 4 ? p.Wo - ox0 : 4;
+    uint64_t acc[4][4];
+#pragma unroll
+    for (int px = 0; px < 4; ++px)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[px][j] = 0ull;
+    const int ix0 = ox0 * STRIDE - 1;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const int iy = oy * STRIDE - 1 + r;
+      if (iy < 0 || iy >= p.H) continue;   // the padding rows contribute nothing
+      uint4 xv[NCOL], wv[3];
+#pragma unroll
+      for (int j = 0; j < NCOL; ++j) {
+        const int ix = ix0 + j;
+        const bool need = ix >= 0 && ix < p.W && j <= (npx - 1) * STRIDE + 2;
+        xv[j] = need ? __ldg(reinterpret_cast<const uint4*>(xs + ((int64_t)iy * p.W + ix) * p.ldx + c0)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int t = 0; t < 3; ++t)
+        wv[t] = __ldg(reinterpret_cast<const uint4*>(p.w + ((int64_t)(k0 + r) * p.K + (k0 + t)) * p.C + c0));
+      uint64_t wf[3][4];
+#pragma unroll
+      for (int t = 0; t < 3; ++t) widen8(wv[t], wf[t]);
+#pragma unroll
+      for (int j = 0; j < NCOL; ++j) {
+        uint64_t xf[4];
+        widen8(xv[j], xf);
+#pragma unroll
+        for (int px = 0; px < 4; ++px) {
+          const int t = j - px * STRIDE;   // which tap of window px this input column is
+          if (t >= 0 && t < 3) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[px][q] = ffma2(xf[q], wf[t][q], acc[px][q]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int px = 0; px < 4; ++px) {
+      if (px < npx) {
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float a, b;
+          unpack2(acc[px][j], a, b);
+          const int ca = c0 + 2 * j, cb = ca + 1;
+          if (p.bias) { a += p.bias[ca]; b += p.bias[cb]; }
+          if (sc) { a = fmaf(a, sc[ca], sh[ca]); b = fmaf(b, sc[cb], sh[cb]); }
+          __nv_bfloat162 h = __floats2bfloat162_rn(act_apply(a, p.act), act_apply(b, p.act));
+          o[j] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(ys + ((int64_t)oy * p.Wo + ox0 + px) * p.ldy + c0) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 2) depthwise_kernel(const __grid_constant__ DwParams p) {
   __shared__ int s_info[3];  // slice, sample, valid
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
   const int pos = blockIdx.y, band = blockIdx.x;
-  if (threadIdx.x == 0) {
-    int valid = pos < p.offsets[p.G], sl = 0, smp = 0;
-    if (valid) {
-      int lo = 0, hi = p.G;
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (p.offsets[mid] <= pos) lo = mid; else hi = mid;
-      }
-      sl = p.group_slice ? p.group_slice[lo] : lo;
-      smp = p.perm[pos];
-      if (smp < 0 || sl < 0 || sl >= p.T) valid = 0;
-    }
-    s_info[0] = sl; s_info[1] = smp; s_info[2] = valid;
-  }
+  // The group of this position: thread g tests group g (one round of loads instead of a binary search's chain of
+  // dependent ones), another thread fetches the sample index at the same time.
+  if (threadIdx.x < 3) s_info[threadIdx.x] = 0;
   __syncthreads();
+  for (int g = threadIdx.x; g < p.G; g += kThreads) {
+    const int lo = p.offsets[g], hi = p.offsets[g + 1];
+    if (lo <= pos && pos < hi) {
+      const int sl = p.group_slice ? p.group_slice[g] : g;
+      s_info[0] = sl;
+      s_info[2] = (sl >= 0 && sl < p.T) ? 1 : 0;
+    }
+  }
+  if (threadIdx.x == kThreads - 1) s_info[1] = p.perm[pos];
+  __syncthreads();
+  if (s_info[1] < 0) return;
   if (!s_info[2]) return;
   const int sl = s_info[0], smp = s_info[1];
   const int ct = p.c[sl], k = p.ksize[sl];
@@ -66,6 +158,12 @@ __global__ void __launch_bounds__(kThreads) depthwise_kernel(const __grid_consta
   const int pix0 = (int)(((int64_t)p.Ho * p.Wo * band) / p.bands), pix1 = (int)(((int64_t)p.Ho * p.Wo * (band + 1)) / p.bands);
   const bool vec_ok = (p.ldx % 8 == 0) && (p.ldy % 8 == 0) && (p.C % 8 == 0) &&
                       ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.w)) & 15) == 0;
+  if (k == 3 && vec_ok && (ct & 7) == 0) {   // whole output rows per band
+    const int row0 = (int)(((int64_t)p.Ho * band) / p.bands), row1 = (int)(((int64_t)p.Ho * (band + 1)) / p.bands);
+    if (p.stride == 1) depthwise3x3_rows<1>(p, xs, ys, ct, sc, sh, row0, row1);
+    else depthwise3x3_rows<2>(p, xs, ys, ct, sc, sh, row0, row1);
+    return;
+  }
   for (int64_t e = threadIdx.x; e < (int64_t)(pix1 - pix0) * nvec; e += kThreads) {
     const int pix = pix0 + (int)(e / nvec), v = (int)(e % nvec);
     const int yy = pix / p.Wo, xx = pix - yy * p.Wo;
@@ -156,7 +254,7 @@ cudaError_t dsn_launch_depthwise(const int32_t* c, const int32_t* ksize, int T, 
   // the SMs more evenly than few long-running ones (measured on 14 x 14 x 640, 256 samples: 91 us with 3 bands)
   int bands = (int)(((int64_t)p.Ho * p.Wo * ((C + 7) / 8)) / (4 * kThreads));
   if (bands < 1) bands = 1;
-  if (bands > p.Ho * p.Wo) bands = p.Ho * p.Wo;
+  if (bands > p.Ho) bands = p.Ho;   // bands are whole output rows on the 3 x 3 fast path
   if (bands > 64) bands = 64;
   p.bands = bands;
   p.x_input_order = x_input_order; p.y_input_order = y_input_order; p.act = act;
