@@ -291,10 +291,20 @@ int fill_gemm_maps(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const
     if (e) return e;
     // columns clipped at k_out rounded down to 8 (the store clips at 16-byte granularity; the epilogue writes the 1..7
     // columns beyond with plain stores); widths below 8 never use the map
-    const uint64_t yd[2] = {(uint64_t)(map_n[m] >= 8 ? (map_n[m] & ~7) : 8), (uint64_t)r->B * g.R};
-    const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
-    const uint32_t yb[2] = {64, 32};
-    e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
+    const uint64_t yn = (uint64_t)(map_n[m] >= 8 ? (map_n[m] & ~7) : 8);
+    if (g.halo) {
+      // the staged-tile kernel stores a CTA's whole block at once: (channel, x, y, sample) with the block's padded
+      // extent as the box; what lies beyond the image's width and height is clipped by the store
+      const uint64_t yd[4] = {yn, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)r->B};
+      const uint64_t ys[3] = {(uint64_t)c.ldy * 2, (uint64_t)c.ldy * 2 * g.W, (uint64_t)c.ldy * 2 * g.W * g.H};
+      const uint32_t yb[4] = {64, (uint32_t)g.bw, (uint32_t)g.bh, 1};
+      e = encode_map(ctx, &p.mapY[m], y, 4, yd, ys, yb);
+    } else {
+      const uint64_t yd[2] = {yn, (uint64_t)r->B * g.R};
+      const uint64_t ys[1] = {(uint64_t)c.ldy * 2};
+      const uint32_t yb[2] = {64, 32};
+      e = encode_map(ctx, &p.mapY[m], y, 2, yd, ys, yb);
+    }
     if (e) return e;
   }
   return DSN_OK;

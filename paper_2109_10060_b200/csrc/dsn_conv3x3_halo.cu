@@ -13,9 +13,17 @@
 // x >= W compute nothing that is stored.  Weights stream through a ring of (tap, chunk) boxes as
 // before; the activation blocks have a ring of their own (2 to 6 slots, as many as fit).
 //
-// Same contract, roles, accumulators and epilogue as dsn_gemm_bf16_2cta.cu.  Added barriers:
+// Same contract, roles and accumulators as dsn_gemm_bf16_2cta.cu.  Added barriers:
 //   afull[a]   even CTA only: the activation boxes of both CTAs have landed
 //   aempty[a]  both CTAs: the MMAs of all nine taps that read the slot are done (multicast commit)
+//
+// Epilogue.  With rows numbered over the padded width a warp's 32 rows are not 32 consecutive output rows (two
+// padding positions per image row), so a store per warp cannot be one box.  The four warps of a column group
+// therefore stage the CTA's 128 rows of a 64-column chunk in one shared block, and one TMA store over
+// (channel, x, y, sample) writes it: the padding positions and the rows below the image lie outside the tensor
+// and are clipped by the store.  Per group:
+//   swritten   4 arrivals: each warp has written its 32 rows of the block
+//   sfree      1 arrival: the store of the chunk before has finished reading the block
 #include <cuda_runtime.h>
 
 #include "dsn_gemm_pair_device.cuh"
@@ -23,6 +31,72 @@
 namespace {
 
 using namespace dsn_gemm;
+
+// What a thread of the epilogue knows about the tile at hand.
+struct HaloEpi {
+  uint32_t taddr;              // this thread's TMEM lane, first column of the accumulator
+  int ncols, n0, ko;           // columns of this n-tile, its first column, the slice's width
+  const float *brow, *sc_row, *sh_row;
+  const __nv_bfloat16* res_row;
+  __nv_bfloat16* yrow;         // this thread's output row (nullptr: padding position, not stored)
+  const CUtensorMap* mapY;     // (channel, x, y, sample), box 64 x (W + 2) x bh x 1
+  int y0, smp;                 // first image row of the tile, output sample (-1: none)
+};
+
+// One tile through the epilogue of a column group (`first`): chunks first, first + 2, ... of 64 columns.
+// `cn` counts the chunks this group has staged (barrier phases), `pending` says that the issuing warp still has to
+// hand the block back.  Returns false when the CTA is aborting.
+template <int ACT, bool AFF, bool RES>
+__device__ __forceinline__ bool halo_epilogue_tile(const HaloEpi& e, int first, int q, int lane, uint8_t* stage_g,
+                                                   uint32_t bar_sw, uint32_t bar_sf, uint32_t& cn, bool& pending,
+                                                   volatile uint32_t* abort_flag, int32_t* status) {
+  const int m = q * 32 + lane;
+  uint8_t* stage_row = stage_g + m * 128;
+  for (int c0 = 64 * first; c0 < e.ncols; c0 += 16 * kEpiWarps, ++cn) {
+    if (q == 0 && pending) {  // the issuing warp: the store of the chunk before has read the block
+      if (lane == 0) {
+        bulk_wait_read0();
+        mbar_arrive(bar_sf);
+      }
+      pending = false;
+      __syncwarp();
+    }
+    if (cn > 0 && !__all_sync(0xffffffffu, mbar_wait(bar_sf, (cn - 1u) & 1u, abort_flag, status, 44))) return false;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      if (c0 + 32 * half < e.ncols) {  // warp-uniform
+        uint32_t w[16];
+        epilogue_half<ACT, AFF, RES>(e.taddr + c0 + 32 * half, c0 + 32 * half, e.ncols, e.brow, e.sc_row, e.sh_row, e.res_row, w);
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const int j = 4 * half + jj;
+          *reinterpret_cast<uint4*>(stage_row + ((j ^ (lane & 7)) << 4)) = make_uint4(w[4 * jj], w[4 * jj + 1], w[4 * jj + 2], w[4 * jj + 3]);
+        }
+      }
+    }
+    // the store's tensor ends at the slice width rounded down to 8 columns: the 1..7 columns beyond leave here
+    const int col8 = e.ncols & ~7, tail_n = e.ncols & 7;
+    if (tail_n != 0 && col8 >= c0 && col8 < c0 + 64 && e.yrow) {
+      const int j = (col8 - c0) >> 3;
+      const uint4 val = *reinterpret_cast<const uint4*>(stage_row + ((j ^ (lane & 7)) << 4));
+      const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+      store_row_tail(e.yrow + col8, w, tail_n);
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_sw);
+    if (q == 0) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sw, cn & 1u, abort_flag, status, 45))) return false;
+      if (lane == 0) {
+        if (e.ko >= 8 && e.smp >= 0) tma_store_4d(e.mapY, e.n0 + c0, 0, e.y0, e.smp, smem_u32(stage_g));
+        bulk_commit();
+      }
+      pending = true;
+      __syncwarp();
+    }
+  }
+  return true;
+}
 
 // kRes: the layer has skip features (residual add before the activation).  The form without them holds no
 // trace of that code: its registers and code size weighed on every other epilogue variant.
@@ -50,6 +124,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
 
   const uint32_t bar_afull = base + 16 * kMaxStages + 48;   // [kMaxStages]
   const uint32_t bar_aempty = bar_afull + 8 * kMaxStages;  // [kMaxStages]
+  const uint32_t bar_stage = base + kCtrlBytes - 16 * (kEpiWarps / 4);  // per column group: swritten, sfree
   const int aslots = g.a_slots;                            // depth of the activation ring
   const int stages = g.stages;                             // depth of the weight ring
   const uint32_t bh_bytes = (uint32_t)(g.BN / 2) * BK * 2;  // this CTA's half of the weight tile of one tap
@@ -81,6 +156,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     for (int a = 0; a < aslots; ++a) {
       mbar_init(bar_afull + 8 * a, 1);
       mbar_init(bar_aempty + 8 * a, 1);
+    }
+    for (int f = 0; f < kEpiWarps / 4; ++f) {
+      mbar_init(bar_stage + 16 * f, 4);      // swritten
+      mbar_init(bar_stage + 16 * f + 8, 1);  // sfree
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -236,75 +315,68 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     const int q = warp & 3;
     const int first = (warp - 2) >> 2;
     const int m = q * 32 + lane;
+    uint8_t* stage_g = out_stage + first * (4 * 32 * 128);  // this column group's block: 128 rows of 128 bytes
+    const uint32_t bar_sw = bar_stage + 16 * first, bar_sf = bar_sw + 8;
+    uint32_t cn = 0;
+    bool pending = false;
     int it = 0;
     bool ok = true;
-    const int box_rows = g.bw * g.bh * g.nb, img_rows = g.bw * g.bh;
-    // this thread's place in a per-image tile does not change from tile to tile
-    const int row_bi = g.flat ? 0 : m / img_rows, row_rem = g.flat ? 0 : m - row_bi * img_rows;
-    const int row_j = g.flat ? 0 : row_rem / g.bw, row_x = g.flat ? 0 : row_rem - row_j * g.bw;
+    // this thread's place in the tile (rows run over the padded width) does not change from tile to tile
+    const int row_j = m / g.bw, row_x = m - row_j * g.bw;
     for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
       const PairTile t = decode_pair_tile(p, s_prefix, tile, rank, cursor);
       const int acc = it & (nacc - 1);
       const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
 
-      bool valid;
-      int64_t out_row;
-      if (g.flat) {
-        const int gr = t.row0 + m;
-        valid = gr < t.rows_end;
-        out_row = gr;
-        if (valid && g.y_input_order) {
-          const int pp = gr / g.R;
-          out_row = (int64_t)p.perm[pp] * g.R + (gr - pp * g.R);
-        }
-      } else {
-        const int yy = t.y0 + row_j, xx = t.x0 + row_x;
-        const int pp = t.b0 + row_bi;
-        valid = m < box_rows && yy < g.H && xx < g.W && pp < t.p_end;
-        out_row = 0;
-        if (valid) {
-          const int smp = g.y_input_order ? p.perm[pp] : pp;
-          out_row = (int64_t)smp * g.R + yy * g.W + xx;
-        }
-      }
-      __nv_bfloat16* yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
-      const float* brow = p.bias ? p.bias + t.n0 : nullptr;
-      const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
-      const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
-      const __nv_bfloat16* res_row = (kRes && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
-      int ncols = t.ko - t.n0;
-      ncols = ncols > g.BN ? g.BN : ncols;
-      const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
-      const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
+      const int yy = t.y0 + row_j;
+      const bool in_group = t.b0 < t.p_end;
+      const int smp = in_group ? (g.y_input_order ? p.perm[t.b0] : t.b0) : -1;
+      const bool valid = in_group && row_j < g.bh && yy < g.H && row_x < g.W;
+      const int64_t out_row = valid ? (int64_t)smp * g.R + yy * g.W + row_x : 0;
+      HaloEpi e;
+      e.ncols = t.ko - t.n0;
+      e.ncols = e.ncols > g.BN ? g.BN : e.ncols;
+      e.n0 = t.n0;
+      e.ko = t.ko;
+      e.brow = p.bias ? p.bias + t.n0 : nullptr;
+      e.sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      e.sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
+      e.res_row = (kRes && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
+      e.yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
+      e.mapY = &p.mapY[t.map];
+      e.y0 = t.y0;
+      e.smp = smp;
 
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
       if (!ok) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
-      uint8_t* stage_w = out_stage + (warp - 2) * (32 * 128);
-      const CUtensorMap* mY = &p.mapY[t.map];
+      e.taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
+#define DSN_HALO_EPI(ACT, AFF, RES) \
+  ok = halo_epilogue_tile<ACT, AFF, RES>(e, first, q, lane, stage_g, bar_sw, bar_sf, cn, pending, abort_flag, p.status)
       if constexpr (kRes) {
         switch (p.act) {
-          case DSN_ACT_NONE: epilogue_tile<DSN_ACT_NONE, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case DSN_ACT_RELU: epilogue_tile<DSN_ACT_RELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          default: epilogue_tile<DSN_ACT_GELU, true, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case DSN_ACT_NONE: DSN_HALO_EPI(DSN_ACT_NONE, true, true); break;
+          case DSN_ACT_RELU: DSN_HALO_EPI(DSN_ACT_RELU, true, true); break;
+          default: DSN_HALO_EPI(DSN_ACT_GELU, true, true); break;
         }
       } else {
-        const int variant = p.act * 2 + ((brow || sc_row) ? 1 : 0);
+        const int variant = p.act * 2 + ((e.brow || e.sc_row) ? 1 : 0);
         switch (variant) {
-          case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 1: if constexpr (!kLean) epilogue_tile<DSN_ACT_NONE, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 2: epilogue_tile<DSN_ACT_RELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 3: if constexpr (!kLean) epilogue_tile<DSN_ACT_RELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          case 4: if constexpr (!kLean) epilogue_tile<DSN_ACT_GELU, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
-          default: if constexpr (!kLean) epilogue_tile<DSN_ACT_GELU, true>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
+          case 0: DSN_HALO_EPI(DSN_ACT_NONE, false, false); break;
+          case 1: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_NONE, true, false); break;
+          case 2: DSN_HALO_EPI(DSN_ACT_RELU, false, false); break;
+          case 3: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_RELU, true, false); break;
+          case 4: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, false, false); break;
+          default: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, true, false); break;
         }
       }
+#undef DSN_HALO_EPI
+      if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it
     }
-    if (elect_one()) bulk_wait0();  // the lane that issued this warp's TMA stores
+    if (q == 0 && lane == 0) bulk_wait0();  // the lane that issued this group's TMA stores
   }
 
   // ------------------------------------------------------------------ teardown

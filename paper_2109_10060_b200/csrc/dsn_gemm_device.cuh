@@ -112,6 +112,11 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src)
                : "memory");
 }
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -241,6 +246,71 @@ __device__ __forceinline__ float apply_act(float v) {
   return v;
 }
 
+// The 1..7 last columns of a row whose width is no multiple of 8 (packed bf16 pairs in `w`): one 8-, one 4- and one
+// 2-byte store when the piece starts on an 8-byte boundary (it does whenever the row does), else 2-byte stores.
+__device__ __forceinline__ void store_row_tail(__nv_bfloat16* dst, const uint32_t (&w)[4], int n) {
+  if ((reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+    int off = 0;
+    if (n & 4) { *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]); off = 4; }
+    if (n & 2) { *reinterpret_cast<uint32_t*>(dst + off) = w[off >> 1]; off += 2; }
+    if (n & 1) reinterpret_cast<uint16_t*>(dst)[off] = (uint16_t)(w[off >> 1] & 0xffffu);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (e < n) reinterpret_cast<uint16_t*>(dst)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
+  }
+}
+
+// 32 accumulator columns of this thread's row (TMEM address `taddr`; columns cb .. cb + 31 of the tile) ->
+// bias, per-path Re-SBN, skip features, activation -> 16 packed bf16 pairs.
+template <int ACT, bool AFF, bool RES>
+__device__ __forceinline__ void epilogue_half(uint32_t taddr, int cb, int ncols, const float* brow, const float* sc_row,
+                                              const float* sh_row, const __nv_bfloat16* res_row, uint32_t (&out)[16]) {
+  // the skip features of this row's 32 columns: four 16-byte loads in flight at once, issued ahead of
+  // the TMEM load (a ragged or unaligned piece takes scalar loads)
+  uint4 rres[4];
+  bool rvec = false;
+  if (RES && res_row) {
+    const __nv_bfloat16* rp = res_row + cb;
+    rvec = cb + 32 <= ncols && (reinterpret_cast<uintptr_t>(rp) & 15u) == 0;
+    if (rvec) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) rres[i] = __ldg(reinterpret_cast<const uint4*>(rp) + i);
+    }
+  }
+  uint32_t v[32];
+  tmem_ld_32x32(taddr, v);
+  tmem_ld_wait();
+#pragma unroll
+  for (int jj = 0; jj < 4; ++jj) {
+    const uint4 rv = rvec ? rres[jj] : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int c = 8 * jj + 2 * e;
+      float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
+      if (AFF) {  // bias, the per-path Re-SBN scale and shift of this tile's columns, the skip features of this row
+        if (cb + c < ncols) {
+          if (brow) a += __ldg(brow + cb + c);
+          if (sc_row) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
+          if (RES && rvec) a += __uint_as_float(rw[e] << 16);
+          else if (RES && res_row) a += __bfloat162float(res_row[cb + c]);
+        }
+        if (cb + c + 1 < ncols) {
+          if (brow) b += __ldg(brow + cb + c + 1);
+          if (sc_row) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
+          if (RES && rvec) b += __uint_as_float(rw[e] & 0xffff0000u);
+          else if (RES && res_row) b += __bfloat162float(res_row[cb + c + 1]);
+        }
+      }
+      if (ACT == DSN_ACT_GELU) gelu_pair(a, b, a, b);
+      else { a = apply_act<ACT>(a); b = apply_act<ACT>(b); }
+      __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+      out[4 * jj + e] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  }
+}
+
 // Epilogue of one tile for one warp: accumulator rows (one per lane) -> bias, activation, bf16 ->
 // 32 x 128-byte swizzled staging tile -> global memory.  The warp takes the 64-column chunks
 // `first`, `first + kEpiWarps / 4`, ...  `yrow` is this lane's output row (nullptr when the row is not part of the
@@ -260,52 +330,13 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       if (c0 + 32 * half < ncols) {  // warp-uniform
-        // the skip features of this row's 32 columns: four 16-byte loads in flight at once, issued ahead of
-        // the TMEM load (a ragged or unaligned piece takes scalar loads)
-        uint4 rres[4];
-        bool rvec = false;
-        if (RES && res_row) {
-          const __nv_bfloat16* rp = res_row + c0 + 32 * half;
-          rvec = c0 + 32 * half + 32 <= ncols && (reinterpret_cast<uintptr_t>(rp) & 15u) == 0;
-          if (rvec) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) rres[i] = __ldg(reinterpret_cast<const uint4*>(rp) + i);
-          }
-        }
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + c0 + 32 * half, v);
-        tmem_ld_wait();
-        const int cb = c0 + 32 * half;
+        uint32_t w[16];
+        epilogue_half<ACT, AFF, RES>(taddr + c0 + 32 * half, c0 + 32 * half, ncols, brow, sc_row, sh_row, res_row, w);
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj) {
-          uint32_t w[4];
-          const uint4 rv = rvec ? rres[jj] : make_uint4(0u, 0u, 0u, 0u);
-          const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = 8 * jj + 2 * e;
-            float a = __uint_as_float(v[c]), b = __uint_as_float(v[c + 1]);
-            if (AFF) {  // bias, the per-path Re-SBN scale and shift of this tile's columns, the skip features of this row
-              if (cb + c < ncols) {
-                if (brow) a += __ldg(brow + cb + c);
-                if (sc_row) a = fmaf(a, __ldg(sc_row + cb + c), __ldg(sh_row + cb + c));
-                if (RES && rvec) a += __uint_as_float(rw[e] << 16);
-                else if (RES && res_row) a += __bfloat162float(res_row[cb + c]);
-              }
-              if (cb + c + 1 < ncols) {
-                if (brow) b += __ldg(brow + cb + c + 1);
-                if (sc_row) b = fmaf(b, __ldg(sc_row + cb + c + 1), __ldg(sh_row + cb + c + 1));
-                if (RES && rvec) b += __uint_as_float(rw[e] & 0xffff0000u);
-                else if (RES && res_row) b += __bfloat162float(res_row[cb + c + 1]);
-              }
-            }
-            if (ACT == DSN_ACT_GELU) gelu_pair(a, b, a, b);
-            else { a = apply_act<ACT>(a); b = apply_act<ACT>(b); }
-            __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-            w[e] = *reinterpret_cast<uint32_t*>(&h);
-          }
           const int j = 4 * half + jj;
-          *reinterpret_cast<uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+              make_uint4(w[4 * jj], w[4 * jj + 1], w[4 * jj + 2], w[4 * jj + 3]);
         }
       }
     }
@@ -323,18 +354,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
         const int j = (col8 - c0) >> 3;
         const uint4 val = *reinterpret_cast<const uint4*>(stage_w + lane * 128 + ((j ^ (lane & 7)) << 4));
         const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-        __nv_bfloat16* dst = yrow + col8;
-        if ((reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
-          int off = 0;
-          if (tail_n & 4) { *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]); off = 4; }
-          if (tail_n & 2) { *reinterpret_cast<uint32_t*>(dst + off) = w[off >> 1]; off += 2; }
-          if (tail_n & 1) reinterpret_cast<uint16_t*>(dst)[off] = (uint16_t)(w[off >> 1] & 0xffffu);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (e < tail_n)
-              reinterpret_cast<uint16_t*>(dst)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
-        }
+        store_row_tail(yrow + col8, w, tail_n);
       }
       continue;
     }
@@ -357,19 +377,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int ncols, int n0,
         } else {  // slice width not a multiple of 8: the 1..7 columns left leave as one 8-, one 4- and one 2-byte store
           // (the piece starts on a 16-byte boundary of the row whenever the row itself does; an odd start falls back to 2-byte stores)
           const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-          const int n = ncols - col;
-          __nv_bfloat16* dst = rp[i] + col;
-          if ((reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
-            int off = 0;
-            if (n & 4) { *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]); off = 4; }
-            if (n & 2) { *reinterpret_cast<uint32_t*>(dst + off) = w[off >> 1]; off += 2; }
-            if (n & 1) reinterpret_cast<uint16_t*>(dst)[off] = (uint16_t)(w[off >> 1] & 0xffffu);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              if (e < n)
-                reinterpret_cast<uint16_t*>(dst)[e] = (e & 1) ? (uint16_t)(w[e >> 1] >> 16) : (uint16_t)(w[e >> 1] & 0xffffu);
-          }
+          store_row_tail(rp[i] + col, w, ncols - col);
         }
       }
     }

@@ -150,7 +150,7 @@ __host__ __device__ inline uint32_t dsn_halo_slot_bytes(int wp, int bh) {
 struct GemmParams {
   CUtensorMap mapA[DSN_GEMM_MAX_MAPS];
   CUtensorMap mapB[DSN_GEMM_MAX_MAPS];
-  CUtensorMap mapY[DSN_GEMM_MAX_MAPS];  // output rows x k_out columns, 64 x 32 box, for the epilogue's TMA stores
+  CUtensorMap mapY[DSN_GEMM_MAX_MAPS];  // output rows x k_out columns, 64 x 32 box, for the epilogue's TMA stores (staged 3x3 tiles: channel, x, y, sample)
   int16_t k_in[DSN_MAX_SLICES];
   int16_t k_out[DSN_MAX_SLICES];
   uint8_t map_id[DSN_MAX_SLICES];
