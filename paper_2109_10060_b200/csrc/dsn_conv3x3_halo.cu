@@ -17,6 +17,12 @@
 //   afull[a]   even CTA only: the activation boxes of both CTAs have landed
 //   aempty[a]  both CTAs: the MMAs of all nine taps that read the slot are done (multicast commit)
 //
+// Schedule.  A pair works on ONE contiguous range of the tile sequence (groups from the widest path down), the
+// ranges cut so that every pair gets the same estimated tensor time (tensor instructions of a tile x their cycles,
+// plus a fixed amount per tile).  Consecutive tiles of a range mostly share their slice, and when the weights of a
+// (slice, n-tile) fit the ring whole they are loaded once and stay until a tile needs others: the issuing warp
+// hands their slots back (commit on `empty`) only then.
+//
 // Epilogue.  With rows numbered over the padded width a warp's 32 rows are not 32 consecutive output rows (two
 // padding positions per image row), so a store per warp cannot be one box.  The four warps of a column group
 // therefore stage the CTA's 128 rows of a 64-column chunk in one shared block, and one TMA store over
@@ -32,6 +38,42 @@ namespace {
 
 using namespace dsn_gemm;
 
+// A run: the tiles of one group, which share everything but their place (sample, image rows).  The roles walk
+// their tiles run by run: what depends on the slice is worked out once per run, and the place of a tile follows
+// from the place of the tile before by adding a fixed step (no division per tile).
+struct HaloRun {
+  int lo, hi;              // tiles [lo, hi) of the schedule
+  int slice, map, ki, ko;  // the group's slice, its tensor maps, its widths
+  int p0, p_end;           // the group's positions of the grouped order
+};
+__device__ __forceinline__ HaloRun halo_find_run(const GemmParams& p, const int32_t* s_prefix, int tile) {
+  HaloRun r;
+  const int j = dsn_find_tile_slot(s_prefix, p.G, tile);
+  const int grp = p.G - 1 - j;
+  r.lo = s_prefix[j];
+  r.hi = s_prefix[j + 1];
+  r.slice = s_prefix[2 * p.G + 2 + grp];
+  r.map = p.map_id[r.slice];
+  r.ki = p.k_in[r.slice];
+  r.ko = p.k_out[r.slice];
+  r.p0 = s_prefix[p.G + 1 + grp];
+  r.p_end = s_prefix[p.G + 2 + grp];
+  return r;
+}
+// Place of an m-tile inside its group: image `ib` of the group, band `ty` of the image (bands per image: nty).
+struct HaloPos { int ib, ty; };
+__device__ __forceinline__ HaloPos halo_pos(int mt, int nty) {
+  HaloPos q;
+  q.ib = mt / nty;
+  q.ty = mt - q.ib * nty;
+  return q;
+}
+__device__ __forceinline__ void halo_advance(HaloPos& q, const HaloPos& step, int nty) {
+  q.ib += step.ib;
+  q.ty += step.ty;
+  if (q.ty >= nty) { q.ty -= nty; ++q.ib; }
+}
+
 // What a thread of the epilogue knows about the tile at hand.
 struct HaloEpi {
   uint32_t taddr;              // this thread's TMEM lane, first column of the accumulator
@@ -43,16 +85,16 @@ struct HaloEpi {
   int y0, smp;                 // first image row of the tile, output sample (-1: none)
 };
 
-// One tile through the epilogue of a column group (`first`): chunks first, first + 2, ... of 64 columns.
+// One tile through the epilogue of a column group: chunks chunk0, chunk0 + chunk_step, ... of 64 columns.
 // `cn` counts the chunks this group has staged (barrier phases), `pending` says that the issuing warp still has to
 // hand the block back.  Returns false when the CTA is aborting.
 template <int ACT, bool AFF, bool RES>
-__device__ __forceinline__ bool halo_epilogue_tile(const HaloEpi& e, int first, int q, int lane, uint8_t* stage_g,
+__device__ __forceinline__ bool halo_epilogue_tile(const HaloEpi& e, int chunk0, int chunk_step, int q, int lane, uint8_t* stage_g,
                                                    uint32_t bar_sw, uint32_t bar_sf, uint32_t& cn, bool& pending,
                                                    volatile uint32_t* abort_flag, int32_t* status) {
   const int m = q * 32 + lane;
   uint8_t* stage_row = stage_g + m * 128;
-  for (int c0 = 64 * first; c0 < e.ncols; c0 += 16 * kEpiWarps, ++cn) {
+  for (int c0 = 64 * chunk0; c0 < e.ncols; c0 += 64 * chunk_step, ++cn) {
     if (q == 0 && pending) {  // the issuing warp: the store of the chunk before has read the block
       if (lane == 0) {
         bulk_wait_read0();
@@ -151,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     }
     for (int a = 0; a < nacc; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 2 * kEpiWarps);
+      mbar_init(bar_tempty + 8 * a, g.BN == 64 ? kEpiWarps : 2 * kEpiWarps);  // one column group per tile when a tile is one chunk
     }
     for (int a = 0; a < aslots; ++a) {
       mbar_init(bar_afull + 8 * a, 1);
@@ -180,20 +222,45 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
   // barriers and TMEM are set up; everything below reads what earlier kernels wrote
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
-  // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group
+  // s_prefix[0..G]: tile prefix; [G+1 .. 2G+1]: group offsets; [2G+2 .. 3G+1]: slice of each group; [3G+3 .. 4G+3]: cost prefix
   for (int j = threadIdx.x; j <= p.G; j += blockDim.x) s_prefix[p.G + 1 + j] = p.offsets[j];
   for (int j = threadIdx.x; j < p.G; j += blockDim.x) {
     const int sl = p.group_slice ? p.group_slice[j] : j;
     s_prefix[2 * p.G + 2 + j] = (sl >= 0 && sl < p.T) ? sl : 0;
   }
   dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);
+  // estimated tensor time of a group's tiles, in units of 16 cycles: the instructions of a tile at N / 2 cycles each
+  // (never below the 59 cycles an instruction occupies the pipe) plus about 300 cycles of fixed work
+  int32_t* s_cost = s_prefix + 3 * p.G + 3;
+  auto tile_cost = [&](int sl) {
+    const int nw = p.k_out[sl] < g.BN ? p.k_out[sl] : g.BN;
+    const int n_inst = (nw + 31) & ~31;
+    const int cyc = n_inst / 2 > 59 ? n_inst / 2 : 59;
+    return (9 * ((p.k_in[sl] + 15) >> 4) * cyc + 300) >> 4;
+  };
+  auto cost_of = [&](int grp) {
+    const int n = ntiles_of(grp);
+    return n ? n * tile_cost(p.group_slice ? p.group_slice[grp] : grp) : 0;
+  };
+  dsn_build_tile_prefix(p.G, s_cost, cost_of);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // the peer's barriers are initialised before anything can arrive on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = s_prefix[p.G];
-  PairCursor cursor;  // every role walks its own tile sequence
+  // first tile of pair k: where the running cost reaches k / npairs of the whole
+  auto range_start = [&](int k) {
+    if (k <= 0 || total == 0) return 0;
+    if (k >= npairs) return total;
+    const int32_t target = (int32_t)(((int64_t)s_cost[p.G] * k) / npairs);
+    const int j = dsn_find_tile_slot(s_cost, p.G, target);
+    const int n = s_prefix[j + 1] - s_prefix[j];
+    return s_prefix[j] + (int)(((int64_t)(target - s_cost[j]) * n) / (s_cost[j + 1] - s_cost[j]));
+  };
+  // g.ranges: a contiguous range per pair; otherwise tile pair, pair + npairs, ... (every pair sees every group)
+  const int tile_begin = g.ranges ? range_start(pair) : pair, tile_end = g.ranges ? range_start(pair + 1) : total;
+  const int sched = g.ranges ? 1 : npairs;  // distance between two tiles of this pair
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -202,38 +269,58 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     int stage = 0, aslot = 0;
     uint32_t phase = 0, aphase = 0;
     const uint32_t a_box_bytes = (uint32_t)(g.bw * (g.bh + 2)) * BK * 2;  // (W + 2) x (bh + 2) pixels
+    int res_key = -1;  // the slice whose weights the ring holds whole (-1: none)
     bool ok = true;
-    for (int tile = pair; ok && tile < total; tile += npairs) {
-      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank, cursor);
-      const CUtensorMap* mA = &p.mapA[t.map];
-      const CUtensorMap* mB = &p.mapB[t.map];
-      const int nkc = (t.ki + BK - 1) / BK;
-      int ncols = t.ko - t.n0;
-      ncols = ncols > g.BN ? g.BN : ncols;
-      const int n_inst = (ncols + 31) & ~31;
-      const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
-      int bsel = t.b0;
-      if (g.a_input_order) bsel = t.b0 < t.p_end ? p.perm[t.b0] : p.B;  // past the group: out of range, zeros
-      for (int kc = 0; ok && kc < nkc; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * aslot, aphase ^ 1u, abort_flag, p.status, 41));
-        if (!ok) break;
-        if (elect_one()) {
-          const uint32_t lead = leader_addr(bar_afull + 8 * aslot);
-          if (rank == 0) mbar_expect_tx(bar_afull + 8 * aslot, 2u * a_box_bytes);
-          tma_load_4d_pair(a_base + aslot * a_slot, mA, kc * BK, -1, t.y0 - 1, bsel, lead);  // halo: starts one pixel out
-        }
-        if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
-        for (int tap0 = 0; tap0 < 9; tap0 += tps) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 42));
+    const HaloPos step = halo_pos(2 * sched, g.tiles_y);
+    int tile = tile_begin;
+    while (ok && tile < tile_end) {
+      const HaloRun r = halo_find_run(p, s_prefix, tile);
+      const int run_end = r.hi < tile_end ? r.hi : tile_end;
+      const CUtensorMap* mA = &p.mapA[r.map];
+      const CUtensorMap* mB = &p.mapB[r.map];
+      const int nkc = (r.ki + BK - 1) / BK;
+      const int n_inst = ((r.ko < g.BN ? r.ko : g.BN) + 31) & ~31;
+      const int brow0 = rank * (n_inst >> 1);  // first weight row of this CTA's half (a slice is one n-tile here)
+      bool reuse = r.slice == res_key;         // the weights are in the ring already
+      if (!reuse) res_key = nkc * (9 / tps) <= stages ? r.slice : -1;
+      const bool keep = res_key >= 0;
+      // the sample a tile reads: looked up (a global load) one tile ahead
+      auto sample_of = [&](const HaloPos& q) {
+        const int b0 = r.p0 + q.ib;
+        if (!g.a_input_order) return b0;
+        return b0 < r.p_end ? __ldg(p.perm + b0) : p.B;  // past the group: out of range, zeros
+      };
+      HaloPos pos = halo_pos(2 * (tile - r.lo) + rank, g.tiles_y);
+      int bsel = sample_of(pos);
+      for (; ok && tile < run_end; tile += sched) {
+        HaloPos pos_next = pos;
+        halo_advance(pos_next, step, g.tiles_y);
+        const int bsel_next = tile + sched < run_end ? sample_of(pos_next) : 0;
+        const int y0 = pos.ty * g.bh;
+        for (int kc = 0; ok && kc < nkc; ++kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * aslot, aphase ^ 1u, abort_flag, p.status, 41));
           if (!ok) break;
           if (elect_one()) {
-            const uint32_t lead = leader_addr(bar_full + 8 * stage);
-            if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * slot_b);
-            for (int u = 0; u < tps; ++u)
-              tma_load_3d_pair(b_base + stage * slot_b + u * bh_bytes, mB, kc * BK, tap0 + u, brow0, lead);
+            const uint32_t lead = leader_addr(bar_afull + 8 * aslot);
+            if (rank == 0) mbar_expect_tx(bar_afull + 8 * aslot, 2u * a_box_bytes);
+            tma_load_4d_pair(a_base + aslot * a_slot, mA, kc * BK, -1, y0 - 1, bsel, lead);  // halo: starts one pixel out
           }
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
+          if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
+          for (int tap0 = 0; !reuse && tap0 < 9; tap0 += tps) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 42));
+            if (!ok) break;
+            if (elect_one()) {
+              const uint32_t lead = leader_addr(bar_full + 8 * stage);
+              if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * slot_b);
+              for (int u = 0; u < tps; ++u)
+                tma_load_3d_pair(b_base + stage * slot_b + u * bh_bytes, mB, kc * BK, tap0 + u, brow0, lead);
+            }
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
+          }
         }
+        reuse = keep;  // kept weights serve the rest of the run
+        pos = pos_next;
+        bsel = bsel_next;
       }
     }
   } else if (warp == 1) {
@@ -250,64 +337,84 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
       const uint64_t db0 = make_smem_desc(b_base);
       const uint64_t dbstep = (uint64_t)(slot_b >> 4), dbtap = (uint64_t)(bh_bytes >> 4);
       const uint64_t darow = (uint64_t)(g.bw * 8);  // one image row of the padded block, in 16-byte units
-      uint64_t db = db0;
-      for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
-        const PairTile t = decode_pair_tile(p, s_prefix, tile, 0, cursor);
-        const int acc = it & (nacc - 1);
-        const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
-        if (!ok) break;
-        tc_fence_after();
-        int ncols = t.ko - t.n0;
-        ncols = ncols > g.BN ? g.BN : ncols;
-        const int n_inst = (ncols + 31) & ~31;
+      int res_key = -1, res_stage = 0, res_n = 0;  // weights kept in the ring: their slice, first slot, slots
+      int tile = tile_begin;
+      while (ok && tile < tile_end) {
+        const HaloRun r = halo_find_run(p, s_prefix, tile);
+        const int run_end = r.hi < tile_end ? r.hi : tile_end;
+        const int n_inst = ((r.ko < g.BN ? r.ko : g.BN) + 31) & ~31;
         const uint32_t idesc = make_idesc(2 * BM, n_inst);
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
-        const int nkc = (t.ki + BK - 1) / BK;
-        const int tail_ks = ((t.ki & (BK - 1)) + 15) >> 4;  // K steps of a partial last chunk (0: none)
-        uint32_t accumulate = 0;
-        for (int kc = nkc; ok && kc > 0; --kc) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * aslot, aphase, abort_flag, p.status, 43));
-          if (!ok) break;
-          const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
-          const uint32_t a_addr = a_base + aslot * a_slot;
-          const uint64_t da0 = make_smem_desc(a_addr);
-          for (int tap0 = 0; tap0 < 9; tap0 += tps) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13));
-            if (!ok) break;
-            tc_fence_after();
-            // a tap's view of the block: same rows, start moved by whole 128-byte rows (8 descriptor units each)
-            if (tps == 9) {
-              if (elect_one()) {
-#pragma unroll
-                for (int u = 0; u < 9; ++u) {
-                  const uint64_t da = da0 + (uint64_t)(u / 3) * darow + (uint64_t)(8 * (u % 3)), dbt = db + (uint64_t)u * dbtap;
-                  umma_bf16_pair(d_tmem, da, dbt, idesc, u == 0 ? accumulate : 1u);  // +32 bytes per K step
-                  if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, dbt + 2u, idesc, 1u);
-                  if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, dbt + 4u, idesc, 1u);
-                  if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, dbt + 6u, idesc, 1u);
-                }
-                umma_commit_pair(bar_empty + 8 * stage);
-              }
-            } else {
-              const int r = tap0 / 3, sx = tap0 - 3 * r;
-              const uint64_t da = da0 + (uint64_t)r * darow + (uint64_t)(8 * sx);
-              if (elect_one()) {
-                umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
-                if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, db + 2u, idesc, 1u);
-                if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, db + 4u, idesc, 1u);
-                if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, db + 6u, idesc, 1u);
-                umma_commit_pair(bar_empty + 8 * stage);
-              }
+        const int nkc = (r.ki + BK - 1) / BK;
+        const int tail_ks = ((r.ki & (BK - 1)) + 15) >> 4;  // K steps of a partial last chunk (0: none)
+        bool reuse = r.slice == res_key;
+        if (!reuse) {
+          if (res_key >= 0 && elect_one()) {  // other weights are needed: the kept slots go back to the producer
+            for (int k = 0; k < res_n; ++k) {
+              const int sl = res_stage + k;
+              umma_commit_pair(bar_empty + 8 * (sl >= stages ? sl - stages : sl));
             }
-            accumulate = 1;
-            db += dbstep;
-            if (++stage == stages) { stage = 0; phase ^= 1u; db = db0; }
           }
-          if (ok && elect_one()) umma_commit_pair(bar_aempty + 8 * aslot);  // all nine taps have read the block
-          if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
+          res_n = nkc * (9 / tps);
+          res_key = res_n <= stages ? r.slice : -1;
+          res_stage = stage;
         }
-        if (ok && elect_one()) umma_commit_pair(bar_tfull + 8 * acc);
+        const bool keep = res_key >= 0;
+        for (; ok && tile < run_end; tile += sched, ++it) {
+          const int acc = it & (nacc - 1);
+          const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
+          int ws = reuse ? res_stage : stage;  // the slot read next
+          uint32_t accumulate = 0;
+          for (int kc = nkc; ok && kc > 0; --kc) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * aslot, aphase, abort_flag, p.status, 43));
+            if (!ok) break;
+            const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
+            const uint32_t a_addr = a_base + aslot * a_slot;
+            const uint64_t da0 = make_smem_desc(a_addr);
+            for (int tap0 = 0; tap0 < 9; tap0 += tps) {
+              if (!reuse) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 13));
+                if (!ok) break;
+                tc_fence_after();
+              }
+              const uint64_t db = db0 + (uint64_t)ws * dbstep;
+              // a tap's view of the block: same rows, start moved by whole 128-byte rows (8 descriptor units each)
+              if (tps == 9) {
+                if (elect_one()) {
+  #pragma unroll
+                  for (int u = 0; u < 9; ++u) {
+                    const uint64_t da = da0 + (uint64_t)(u / 3) * darow + (uint64_t)(8 * (u % 3)), dbt = db + (uint64_t)u * dbtap;
+                    umma_bf16_pair(d_tmem, da, dbt, idesc, u == 0 ? accumulate : 1u);  // +32 bytes per K step
+                    if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, dbt + 2u, idesc, 1u);
+                    if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, dbt + 4u, idesc, 1u);
+                    if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, dbt + 6u, idesc, 1u);
+                  }
+                  if (!keep) umma_commit_pair(bar_empty + 8 * stage);
+                }
+              } else {
+                const int tr = tap0 / 3, sx = tap0 - 3 * tr;
+                const uint64_t da = da0 + (uint64_t)tr * darow + (uint64_t)(8 * sx);
+                if (elect_one()) {
+                  umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                  if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, db + 2u, idesc, 1u);
+                  if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, db + 4u, idesc, 1u);
+                  if (nks > 3) umma_bf16_pair(d_tmem, da + 6u, db + 6u, idesc, 1u);
+                  if (!keep) umma_commit_pair(bar_empty + 8 * stage);
+                }
+              }
+              accumulate = 1;
+              if (++ws == stages) ws = 0;
+              if (!reuse && ++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok && elect_one()) umma_commit_pair(bar_aempty + 8 * aslot);  // all nine taps have read the block
+            if (++aslot == aslots) { aslot = 0; aphase ^= 1u; }
+          }
+          if (ok && elect_one()) umma_commit_pair(bar_tfull + 8 * acc);
+          reuse = keep;  // kept weights serve the rest of the run
+        }
       }
     }
   } else {
@@ -319,62 +426,79 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     const uint32_t bar_sw = bar_stage + 16 * first, bar_sf = bar_sw + 8;
     uint32_t cn = 0;
     bool pending = false;
-    int it = 0;
     bool ok = true;
     // this thread's place in the tile (rows run over the padded width) does not change from tile to tile
     const int row_j = m / g.bw, row_x = m - row_j * g.bw;
-    for (int tile = pair; ok && tile < total; tile += npairs, ++it) {
-      const PairTile t = decode_pair_tile(p, s_prefix, tile, rank, cursor);
-      const int acc = it & (nacc - 1);
-      const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
-
-      const int yy = t.y0 + row_j;
-      const bool in_group = t.b0 < t.p_end;
-      const int smp = in_group ? (g.y_input_order ? p.perm[t.b0] : t.b0) : -1;
-      const bool valid = in_group && row_j < g.bh && yy < g.H && row_x < g.W;
-      const int64_t out_row = valid ? (int64_t)smp * g.R + yy * g.W + row_x : 0;
+    // 64-wide n-tiles are a single chunk: the two column groups take every other tile instead of every other chunk
+    const bool alternate = g.BN == 64;
+    const int chunk0 = alternate ? 0 : first, chunk_step = alternate ? 1 : kEpiWarps / 4;
+    const int it_step = alternate ? kEpiWarps / 4 : 1, tile_step = it_step * sched;
+    const HaloPos step = halo_pos(2 * tile_step, g.tiles_y);
+    int tile = tile_begin + (alternate ? first * sched : 0), it = alternate ? first : 0;
+    while (ok && tile < tile_end) {
+      const HaloRun r = halo_find_run(p, s_prefix, tile);
+      const int run_end = r.hi < tile_end ? r.hi : tile_end;
       HaloEpi e;
-      e.ncols = t.ko - t.n0;
-      e.ncols = e.ncols > g.BN ? g.BN : e.ncols;
-      e.n0 = t.n0;
-      e.ko = t.ko;
-      e.brow = p.bias ? p.bias + t.n0 : nullptr;
-      e.sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
-      e.sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
-      e.res_row = (kRes && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
-      e.yrow = valid ? p.y + out_row * p.ldy + t.n0 : nullptr;
-      e.mapY = &p.mapY[t.map];
-      e.y0 = t.y0;
-      e.smp = smp;
+      e.ncols = r.ko < g.BN ? r.ko : g.BN;  // a slice is one n-tile here
+      e.n0 = 0;
+      e.ko = r.ko;
+      e.brow = p.bias;
+      e.sc_row = p.bn_scale ? p.bn_scale + (int64_t)r.slice * p.bn_ld : nullptr;
+      e.sh_row = p.bn_scale ? p.bn_shift + (int64_t)r.slice * p.bn_ld : nullptr;
+      e.mapY = &p.mapY[r.map];
+      // the sample a tile writes: looked up (a global load) one tile ahead
+      auto sample_of = [&](const HaloPos& q) {
+        const int b0 = r.p0 + q.ib;
+        if (b0 >= r.p_end) return -1;
+        return g.y_input_order ? __ldg(p.perm + b0) : b0;
+      };
+      HaloPos pos = halo_pos(2 * (tile - r.lo) + rank, g.tiles_y);
+      int smp = sample_of(pos);
+      for (; ok && tile < run_end; tile += tile_step, it += it_step) {
+        HaloPos pos_next = pos;
+        halo_advance(pos_next, step, g.tiles_y);
+        const int smp_next = tile + tile_step < run_end ? sample_of(pos_next) : -1;
+        const int acc = it & (nacc - 1);
+        const uint32_t acc_phase = (uint32_t)(it >> acc_log2) & 1u;
+        e.y0 = pos.ty * g.bh;
+        e.smp = smp;
+        const int yy = e.y0 + row_j;
+        const bool valid = smp >= 0 && row_j < g.bh && yy < g.H && row_x < g.W;
+        const int64_t out_row = valid ? (int64_t)smp * g.R + yy * g.W + row_x : 0;
+        e.res_row = (kRes && valid) ? p.residual + out_row * p.ldy : nullptr;
+        e.yrow = valid ? p.y + out_row * p.ldy : nullptr;
 
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
-      if (!ok) break;
-      tc_fence_after();
-      e.taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, p.status, 14));
+        if (!ok) break;
+        tc_fence_after();
+        e.taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * g.BN);
 #define DSN_HALO_EPI(ACT, AFF, RES) \
-  ok = halo_epilogue_tile<ACT, AFF, RES>(e, first, q, lane, stage_g, bar_sw, bar_sf, cn, pending, abort_flag, p.status)
-      if constexpr (kRes) {
-        switch (p.act) {
-          case DSN_ACT_NONE: DSN_HALO_EPI(DSN_ACT_NONE, true, true); break;
-          case DSN_ACT_RELU: DSN_HALO_EPI(DSN_ACT_RELU, true, true); break;
-          default: DSN_HALO_EPI(DSN_ACT_GELU, true, true); break;
+  ok = halo_epilogue_tile<ACT, AFF, RES>(e, chunk0, chunk_step, q, lane, stage_g, bar_sw, bar_sf, cn, pending, abort_flag, p.status)
+        if constexpr (kRes) {
+          switch (p.act) {
+            case DSN_ACT_NONE: DSN_HALO_EPI(DSN_ACT_NONE, true, true); break;
+            case DSN_ACT_RELU: DSN_HALO_EPI(DSN_ACT_RELU, true, true); break;
+            default: DSN_HALO_EPI(DSN_ACT_GELU, true, true); break;
+          }
+        } else {
+          const int variant = p.act * 2 + ((e.brow || e.sc_row) ? 1 : 0);
+          switch (variant) {
+            case 0: DSN_HALO_EPI(DSN_ACT_NONE, false, false); break;
+            case 1: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_NONE, true, false); break;
+            case 2: DSN_HALO_EPI(DSN_ACT_RELU, false, false); break;
+            case 3: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_RELU, true, false); break;
+            case 4: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, false, false); break;
+            default: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, true, false); break;
+          }
         }
-      } else {
-        const int variant = p.act * 2 + ((e.brow || e.sc_row) ? 1 : 0);
-        switch (variant) {
-          case 0: DSN_HALO_EPI(DSN_ACT_NONE, false, false); break;
-          case 1: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_NONE, true, false); break;
-          case 2: DSN_HALO_EPI(DSN_ACT_RELU, false, false); break;
-          case 3: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_RELU, true, false); break;
-          case 4: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, false, false); break;
-          default: if constexpr (!kLean) DSN_HALO_EPI(DSN_ACT_GELU, true, false); break;
-        }
-      }
 #undef DSN_HALO_EPI
-      if (!ok) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the even CTA's MMA thread waits on it
+        pos = pos_next;
+        smp = smp_next;
+      }
     }
     if (q == 0 && lane == 0) bulk_wait0();  // the lane that issued this group's TMA stores
   }
@@ -394,7 +518,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
 
 size_t dsn_gemm_halo_smem_bytes(int BN, int stages, int tps, int a_slots, int G, int wp, int bh) {
   return 1024 + kCtrlBytes + (size_t)a_slots * dsn_halo_slot_bytes(wp, bh) + (size_t)stages * tps * ((size_t)(BN / 2) * BK * 2) +
-         kStageOutBytes + sizeof(int32_t) * (3 * (size_t)G + 3);
+         kStageOutBytes + sizeof(int32_t) * (4 * (size_t)G + 4);
 }
 
 cudaError_t dsn_launch_gemm_bf16_halo(const GemmParams& p, int clusters, size_t smem_bytes, cudaStream_t s) {
