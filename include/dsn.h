@@ -195,8 +195,8 @@ typedef struct dsn_layer_desc {
  * Environment switches, read here, that select between kernels computing the same results (for
  * comparisons and as fallbacks): DSN_GEMM_MODE=1cta (one CTA per tile instead of CTA pairs),
  * DSN_CHAIN=0 (dsn_layer_forward: one launch per layer even for small batches), DSN_CONV3X3=taps
- * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_HALO_SCHED=strided|ranges
- * (tile order of the staged 3x3 kernel; chosen per layer by default), DSN_ATTENTION=items (the
+ * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_HALO_SCHED=strided
+ * (staged 3x3 kernel: tiles dealt out round-robin instead of one time-balanced range per CTA pair), DSN_ATTENTION=items (the
  * attention core with one (sample, head, query half) per CTA pass instead of the warp-specialised form),
  * DSN_DWPW=fused (depthwise + following 1x1 layer as one kernel), DSN_PDL=0 (no programmatic dependent launch).
  * Every later call must be made with `device` as the calling thread's current CUDA device (else

@@ -352,14 +352,9 @@ int run_bf16(dsn_ctx* ctx, const LayerCall& c, const dsn_routing* r, const void*
         if (tps == 1) break;
       }
       if (!fits) return DSN_ERR_UNSUPPORTED;  // cannot happen for W + 2 <= 128: two blocks and two boxes always fit
-      // Schedule: when the weights of the widest slice fill the ring, a change of slice drains it, so every pair gets
-      // one contiguous range (few changes); with room left the next slice's weights load beside the current ones and
-      // the strided order, which balances by itself, is the faster one (measured on the 56x56 and 28x28 stages).
-      int max_ki = 1;
-      for (int t = 0; t < c.T; ++t) max_ki = c.k_in[t] > max_ki ? c.k_in[t] : max_ki;
-      const int chunks = (max_ki + DSN_GEMM_BK - 1) / DSN_GEMM_BK;
-      const bool ring_full = g.tps == 9 && chunks >= g.stages;
-      p.g.ranges = ctx->halo_sched == 2 || (ctx->halo_sched == 0 && ring_full);
+      // Schedule: every pair gets one contiguous range of the tile sequence, cut by estimated time (few changes of
+      // slice per pair, so the weights stay in the ring); the strided order is kept for comparisons.
+      p.g.ranges = ctx->halo_sched != 1;
       const size_t smem_h = dsn_gemm_halo_smem_bytes(g.BN, g.stages, g.tps, g.a_slots, r->G, g.bw, g.bh);
       int done_h[DSN_MAX_SLICES];
       memset(done_h, 0, sizeof(done_h));

@@ -229,14 +229,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     s_prefix[2 * p.G + 2 + j] = (sl >= 0 && sl < p.T) ? sl : 0;
   }
   dsn_build_tile_prefix(p.G, s_prefix, ntiles_of);
-  // estimated tensor time of a group's tiles, in units of 16 cycles: the instructions of a tile at N / 2 cycles each
-  // (never below the 59 cycles an instruction occupies the pipe) plus about 300 cycles of fixed work
+  // estimated time of a group's tiles, in units of 16 cycles.  Measured on this kernel: about 1000 cycles of fixed
+  // work per tile in the issuing warp, and per tensor instruction N / 2 cycles but never less than about 40
   int32_t* s_cost = s_prefix + 3 * p.G + 3;
   auto tile_cost = [&](int sl) {
     const int nw = p.k_out[sl] < g.BN ? p.k_out[sl] : g.BN;
     const int n_inst = (nw + 31) & ~31;
-    const int cyc = n_inst / 2 > 59 ? n_inst / 2 : 59;
-    return (9 * ((p.k_in[sl] + 15) >> 4) * cyc + 300) >> 4;
+    const int cyc = n_inst / 2 > 40 ? n_inst / 2 : 40;
+    // a tile of several chunks fills the activation ring alone: part of the next tile's load is then exposed
+    const int exposed = (p.k_in[sl] > BK && aslots < 4) ? 1200 : 0;
+    return (9 * ((p.k_in[sl] + 15) >> 4) * cyc + 1000 + exposed) >> 4;
   };
   auto cost_of = [&](int grp) {
     const int n = ntiles_of(grp);
@@ -384,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
               // a tap's view of the block: same rows, start moved by whole 128-byte rows (8 descriptor units each)
               if (tps == 9) {
                 if (elect_one()) {
-  #pragma unroll
+#pragma unroll
                   for (int u = 0; u < 9; ++u) {
                     const uint64_t da = da0 + (uint64_t)(u / 3) * darow + (uint64_t)(8 * (u % 3)), dbt = db + (uint64_t)u * dbtap;
                     umma_bf16_pair(d_tmem, da, dbt, idesc, u == 0 ? accumulate : 1u);  // +32 bytes per K step

@@ -38,7 +38,7 @@ struct dsn_ctx {
   int32_t* d_status;   // DSN_STATUS_WORDS ints
   void* encode_tiled;  // cuTensorMapEncodeTiled entry point
   int gemm_mode;       // 0 = CTA pairs where possible (default), 1 = one CTA per tile (DSN_GEMM_MODE=1cta)
-  int halo_sched;      // staged 3x3 tiles: 0 = chosen per layer, 1 = strided, 2 = contiguous ranges (DSN_HALO_SCHED=strided|ranges)
+  int halo_sched;      // staged 3x3 tiles: 1 = dealt out round-robin (DSN_HALO_SCHED=strided), else one time-balanced range per pair
   int conv_halo;       // 1 = 3x3 layers stage the input tile once with its halo (default), 0 = one load per tap (DSN_CONV3X3=taps)
   int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
   int dwpw_fused;      // 1 = depthwise + following 1x1 layer as one kernel (DSN_DWPW=fused); default 0: measured slower than the
