@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_halo_kernel(const __gri
     }
     for (int a = 0; a < nacc; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, g.BN == 64 ? kEpiWarps : 2 * kEpiWarps);  // one column group per tile when a tile is one chunk
+      mbar_init(bar_tempty + 8 * a, g.BN == 64 ? 2 * 4 : 2 * kEpiWarps);  // 64-wide n-tiles: one column group (four warps in each CTA) per tile
     }
     for (int a = 0; a < aslots; ++a) {
       mbar_init(bar_afull + 8 * a, 1);
