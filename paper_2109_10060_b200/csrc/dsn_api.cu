@@ -595,7 +595,7 @@ int check_gate(const dsn_gate_desc* g) {
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 1) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
+  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 32) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
     return DSN_ERR_UNSUPPORTED;  // score kernel stages W2 in shared memory
   return DSN_OK;
 }

@@ -6,17 +6,19 @@
 // different rows, four loads are in flight per thread; fp32 accumulation in registers, one
 // shared-memory reduction across the row groups, column sums to partial[b][split][c].  No atomics,
 // so sums are reproducible run to run.
-// Kernel 2 (latency-bound, plain FMA): grid (B/4, C_mlp/16).  A CTA folds the partial sums of 4
+// Kernel 2 (latency-bound, plain FMA): grid (B/4 or B/8, C_mlp/16).  A CTA folds the partial sums of its
 // samples (scaled by 1/R) into shared memory and computes 16 hidden units for them, one warp per
-// two units, all weight loads of a 1024-channel panel in flight at once; ReLU; hid[b][j] to scratch.
-// Kernel 3 (tiny): one warp per sample, lane t owns the score of path t; arg-max by a strict '>'
-// scan in ascending path order (ties keep the lowest index).
+// two units, all weight loads of a 512-channel panel in flight at once; ReLU; hid[b][j] to scratch.
+// Kernel 3 (tiny): one warp per sample, 32 / T lanes per path; arg-max by a strict '>' scan in
+// ascending path order (ties keep the lowest index).
+// Kernels 2 and 3 load their weights before they wait for the kernel ahead of them in the stream.
 #include "dsn_internal.cuh"
 
 namespace {
 
 constexpr int kSBSmall = 4;        // samples per CTA in the hidden-layer kernel
 constexpr int kSBLarge = 8;        // ... for large batches, where re-reading W1 per CTA would bound the kernel
+constexpr int kSBLargeMinBatch = 512;  // batches from this size on take kSBLarge (measured: at B = 256 the larger form is slower)
 constexpr int kJB = 16;            // hidden units per CTA in the hidden-layer kernel
 constexpr int kPoolThreads = 512;
 constexpr int kMlpThreads = 256;
@@ -118,58 +120,80 @@ __device__ __forceinline__ float4 ld_ordered16(const float4* p) {
   return v;
 }
 
-// Hidden layer for kSB samples x kJB units per CTA.  The loop over the input channels runs in
-// panels of 1024: a warp first issues the 16-byte loads of its two weight rows for the panel
-// (16 per lane, all in flight), then the CTA folds the pooling partial sums of the panel into
-// shared memory (their loads overlap the weight loads), then the FMAs run out of registers and
-// shared memory.  Every global load of a panel is therefore issued in one round.
+// Hidden layer for kSB samples x kJB units per CTA.  The kernel is a chain of load latencies, so every
+// load that can be issued early is: the loop over the input channels runs in panels of 512; a warp
+// issues the 16-byte loads of its two weight rows for a panel (4 + 4 per lane) in one round, and those of
+// the first panel BEFORE the wait for the pooling kernel (the weights are parameters, nothing in the stream
+// writes them); the CTA then folds the pooling partial sums of the panel into shared memory (thread t owns
+// 16-byte column t % 128 of every other sample; the loads of two samples x four splits are in flight
+// together and nothing is divided); the FMAs run out of registers and shared memory.
+constexpr int kPanel = 512;
 template <int kSB>
-__global__ void __launch_bounds__(kMlpThreads)
+__global__ void __launch_bounds__(kMlpThreads, 2)
 gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, int C_full, int c_valid, int C_mlp,
                    const float* __restrict__ W1, const float* __restrict__ b1, float* __restrict__ hid) {
-  __shared__ __align__(16) float pooled[kSB][1024];
-  dsn_grid_dependency_wait();
-  dsn_grid_launch_dependents();
+  __shared__ __align__(16) float pooled[kSB][kPanel];
   const int b0 = blockIdx.x * kSB, j0 = blockIdx.y * kJB;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_r = 1.0f / (float)R;
   const bool vec = (c_valid % 4 == 0) && (C_full % 4 == 0) && ((reinterpret_cast<uintptr_t>(W1) & 15) == 0);
   const int ja = j0 + 2 * warp, jb = ja + 1;
+  float4 wa[4], wb[4];
+  auto load_weights = [&](int cbase, int cw) {
+    const float4* pa = reinterpret_cast<const float4*>(W1 + (int64_t)(ja < C_mlp ? ja : 0) * C_full + cbase);
+    const float4* pb = reinterpret_cast<const float4*>(W1 + (int64_t)(jb < C_mlp ? jb : 0) * C_full + cbase);
+    const int n4 = cw >> 2;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = lane + 32 * i;
+      wa[i] = c < n4 ? ld_ordered16(pa + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      wb[i] = c < n4 ? ld_ordered16(pb + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  if (vec) load_weights(0, c_valid < kPanel ? c_valid : kPanel);
+  dsn_grid_dependency_wait();
+  dsn_grid_launch_dependents();
   float acc[2][kSB];
 #pragma unroll
   for (int u = 0; u < 2; ++u)
 #pragma unroll
     for (int s = 0; s < kSB; ++s) acc[u][s] = 0.f;
 
-  for (int cbase = 0; cbase < c_valid; cbase += 1024) {
-    const int cw = c_valid - cbase < 1024 ? c_valid - cbase : 1024;  // panel width
-    float4 wa[8], wb[8];
-    if (vec) {
-      const float4* pa = reinterpret_cast<const float4*>(W1 + (int64_t)(ja < C_mlp ? ja : 0) * C_full + cbase);
-      const float4* pb = reinterpret_cast<const float4*>(W1 + (int64_t)(jb < C_mlp ? jb : 0) * C_full + cbase);
-      const int n4 = cw >> 2;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int c = lane + 32 * i;
-        wa[i] = c < n4 ? ld_ordered16(pa + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-        wb[i] = c < n4 ? ld_ordered16(pb + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    }
+  for (int cbase = 0; cbase < c_valid; cbase += kPanel) {
+    const int cw = c_valid - cbase < kPanel ? c_valid - cbase : kPanel;  // panel width
+    if (vec && cbase > 0) load_weights(cbase, cw);
     // fold the partial sums of this panel
     if (c_valid % 4 == 0) {
       const int n4 = cw >> 2, row4 = c_valid >> 2;
-      for (int e = tid; e < kSB * n4; e += kMlpThreads) {
-        const int s = e / n4, c4 = e - s * n4;
-        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (b0 + s < B) {
-          const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)(b0 + s) * splits) * c_valid + cbase) + c4;
-#pragma unroll 4
-          for (int sp = 0; sp < splits; ++sp) {
-            const float4 t = __ldg(p + (int64_t)sp * row4);
-            sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+      const int c4 = tid & (kPanel / 4 - 1), s0 = tid / (kPanel / 4);  // kMlpThreads / (kPanel / 4) = 2 samples per round
+      if (c4 < n4) {
+#pragma unroll
+        for (int u0 = 0; u0 < kSB / 2; u0 += 2) {  // two samples of this thread per round
+          const int smp0 = b0 + s0 + 2 * u0, smp1 = smp0 + 2;
+          const bool in0 = smp0 < B, in1 = smp1 < B;
+          const float4* p0 = reinterpret_cast<const float4*>(partial + ((int64_t)(in0 ? smp0 : 0) * splits) * c_valid + cbase) + c4;
+          const float4* p1 = reinterpret_cast<const float4*>(partial + ((int64_t)(in1 ? smp1 : 0) * splits) * c_valid + cbase) + c4;
+          float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
+          int sp = 0;
+          for (; sp + 4 <= splits; sp += 4) {  // eight independent loads in flight
+            float4 ta[4], tb[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { ta[q] = __ldg(p0 + (int64_t)(sp + q) * row4); tb[q] = __ldg(p1 + (int64_t)(sp + q) * row4); }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              sa.x += ta[q].x; sa.y += ta[q].y; sa.z += ta[q].z; sa.w += ta[q].w;
+              sb.x += tb[q].x; sb.y += tb[q].y; sb.z += tb[q].z; sb.w += tb[q].w;
+            }
           }
+          for (; sp < splits; ++sp) {
+            const float4 ta = __ldg(p0 + (int64_t)sp * row4), tb = __ldg(p1 + (int64_t)sp * row4);
+            sa.x += ta.x; sa.y += ta.y; sa.z += ta.z; sa.w += ta.w;
+            sb.x += tb.x; sb.y += tb.y; sb.z += tb.z; sb.w += tb.w;
+          }
+          const float fa = in0 ? inv_r : 0.f, fb = in1 ? inv_r : 0.f;  // samples past the batch: zeros
+          reinterpret_cast<float4*>(pooled[s0 + 2 * u0])[c4] = make_float4(sa.x * fa, sa.y * fa, sa.z * fa, sa.w * fa);
+          reinterpret_cast<float4*>(pooled[s0 + 2 * u0 + 2])[c4] = make_float4(sb.x * fb, sb.y * fb, sb.z * fb, sb.w * fb);
         }
-        reinterpret_cast<float4*>(pooled[s])[c4] = make_float4(sum.x * inv_r, sum.y * inv_r, sum.z * inv_r, sum.w * inv_r);
       }
     } else {
       for (int e = tid; e < kSB * cw; e += kMlpThreads) {
@@ -185,7 +209,7 @@ gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, 
     __syncthreads();
     if (vec) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 4; ++i) {
         const int c = lane + 32 * i;
         if (c < (cw >> 2)) {
 #pragma unroll
@@ -224,44 +248,52 @@ gate_hidden_kernel(const float* __restrict__ partial, int splits, int B, int R, 
   }
 }
 
-// Scores and arg-max: one warp per sample.  W2 ([T][C_mlp], row pitch padded by one float) and the
-// sample's hidden vector are staged in shared memory with one round of loads; lane t (and t + 32)
-// accumulates the whole dot product of path t; lane 0 then scans the T scores in ascending order
-// with a strict '>' so that ties keep the lowest index.
+// Scores and arg-max: one warp per sample.  W2 ([T][C_mlp]) is staged in shared memory BEFORE the wait for
+// the hidden-layer kernel (a parameter, written by nothing in the stream), the sample's hidden vector after
+// it.  P = 32 / T (rounded down to a power of two, at least 1) lanes share the dot product of one path, each
+// over every P-th hidden unit, and add their parts up in a fixed butterfly; the row pitch of W2 in shared
+// memory is chosen so that the 32 lanes of a step hit 32 different banks.  Lane 0 then scans the T scores in
+// ascending order with a strict '>' so that ties keep the lowest index.
 __global__ void __launch_bounds__(kMlpThreads)
 gate_score_kernel(const float* __restrict__ hid, int B, int C_mlp, int T, const float* __restrict__ W2,
                   const float* __restrict__ b2, int32_t* __restrict__ idx_out, float* __restrict__ logits_out,
                   int32_t* status) {
   extern __shared__ __align__(16) float sm[];
-  const int pitch = C_mlp + 1;
+  int P = 1;
+  while (2 * P * T <= 32) P <<= 1;
+  const int pitch = C_mlp + ((P - C_mlp) & 31);      // pitch % 32 == P % 32: path t, part q -> bank (t P + q) % 32
   float* w2s = sm;                                   // [T][pitch]
   float* hs = w2s + (size_t)T * pitch;               // [warps][C_mlp]
   float* sc = hs + (size_t)(kMlpThreads / 32) * C_mlp;  // [warps][DSN_MAX_SLICES]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int b = blockIdx.x * (kMlpThreads / 32) + warp;
+  for (int t = warp; t < T; t += kMlpThreads / 32)
+    for (int j = lane; j < C_mlp; j += 32) w2s[t * pitch + j] = __ldg(W2 + (int64_t)t * C_mlp + j);
   dsn_grid_dependency_wait();
   dsn_grid_launch_dependents();
-  for (int e = threadIdx.x; e < T * C_mlp; e += kMlpThreads) {
-    const int t = e / C_mlp, j = e - t * C_mlp;
-    w2s[t * pitch + j] = __ldg(W2 + e);
-  }
   if (b < B)
     for (int j = lane; j < C_mlp; j += 32) hs[warp * C_mlp + j] = hid[(int64_t)b * C_mlp + j];
   __syncthreads();
   if (b >= B) return;
   const float* h = hs + warp * C_mlp;
-  for (int t = lane; t < T; t += 32) {
-    const float* w = w2s + t * pitch;
+  const int part = lane & (P - 1), per_round = 32 / P;
+  for (int t0 = 0; t0 < T; t0 += per_round) {
+    const int t = t0 + lane / P;
+    const float* w = w2s + (t < T ? t : 0) * pitch;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    int j = 0;
-    for (; j + 4 <= C_mlp; j += 4) {
-      a0 = fmaf(w[j], h[j], a0); a1 = fmaf(w[j + 1], h[j + 1], a1);
-      a2 = fmaf(w[j + 2], h[j + 2], a2); a3 = fmaf(w[j + 3], h[j + 3], a3);
+    int j = part;
+    for (; j + 3 * P < C_mlp; j += 4 * P) {
+      a0 = fmaf(w[j], h[j], a0); a1 = fmaf(w[j + P], h[j + P], a1);
+      a2 = fmaf(w[j + 2 * P], h[j + 2 * P], a2); a3 = fmaf(w[j + 3 * P], h[j + 3 * P], a3);
     }
-    for (; j < C_mlp; ++j) a0 = fmaf(w[j], h[j], a0);
-    const float v = (a0 + a1) + (a2 + a3) + (b2 ? b2[t] : 0.f);
-    sc[warp * DSN_MAX_SLICES + t] = v;
-    if (logits_out) logits_out[(int64_t)b * T + t] = v;
+    for (; j < C_mlp; j += P) a0 = fmaf(w[j], h[j], a0);
+    float v = (a0 + a1) + (a2 + a3);
+    for (int o = P >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (part == 0 && t < T) {
+      v += b2 ? b2[t] : 0.f;
+      sc[warp * DSN_MAX_SLICES + t] = v;
+      if (logits_out) logits_out[(int64_t)b * T + t] = v;
+    }
   }
   __syncwarp();
   if (lane == 0) {
@@ -433,7 +465,7 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (g.B >= 512) {
+  if (g.B >= kSBLargeMinBatch) {
     dim3 hgrid((g.B + kSBLarge - 1) / kSBLarge, (g.C_mlp + kJB - 1) / kJB);
     dsn_launch(gate_hidden_kernel<kSBLarge>, hgrid, dim3(kMlpThreads), 0, s, 1, (const float*)partial, splits, g.B, g.R,
                g.C_full, g.c_valid, g.C_mlp, g.W1, g.b1, hid);
@@ -445,7 +477,7 @@ cudaError_t dsn_launch_gate(const dsn_gate_desc& g, const void* x, int32_t* idx_
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int per_cta = kMlpThreads / 32;
-  const size_t smem = sizeof(float) * ((size_t)g.T * (g.C_mlp + 1) + (size_t)per_cta * g.C_mlp +
+  const size_t smem = sizeof(float) * ((size_t)g.T * (g.C_mlp + 32) + (size_t)per_cta * g.C_mlp +
                                        (size_t)per_cta * DSN_MAX_SLICES);
   if (smem > 48 * 1024) {
     e = cudaFuncSetAttribute(gate_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -499,7 +531,7 @@ extern "C" int dsn_gate_static(dsn_ctx* ctx, const dsn_gate_desc* g, const void*
   if (g->B < 0 || g->R < 1 || g->C_full < 1 || g->c_valid < 1 || g->c_valid > g->C_full || g->C_mlp < 1 ||
       g->T < 1 || g->T > DSN_MAX_SLICES || g->ldx < g->c_valid)
     return DSN_ERR_INVALID_ARG;
-  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 1) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
+  if ((size_t)4 * ((size_t)g->T * (g->C_mlp + 32) + 8 * (size_t)g->C_mlp + 8 * DSN_MAX_SLICES) > 200 * 1024)
     return DSN_ERR_UNSUPPORTED;
   if (g->B == 0) return DSN_OK;
   const int splits = dsn_gate_splits(*g, ctx->sm_count);
