@@ -111,8 +111,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
       const CUtensorMap* mA = &p.mapA[t.map];
       const CUtensorMap* mB = &p.mapB[t.map];
       const int nkc = (t.ki + BK - 1) / BK;
-      int ncols = t.ko - t.n0;
-      ncols = ncols > g.BN ? g.BN : ncols;
+      const int ncols = t.ncols;
       const int n_inst = (ncols + 31) & ~31;
       const int brow0 = t.n0 + rank * (n_inst >> 1);  // first weight row of this CTA's half
       int bsel = t.b0;
@@ -155,8 +154,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, p.status, 12));
         if (!ok) break;
         tc_fence_after();
-        int ncols = t.ko - t.n0;
-        ncols = ncols > g.BN ? g.BN : ncols;
+        const int ncols = t.ncols;
         const int n_inst = (ncols + 31) & ~31;
         const uint32_t idesc = make_idesc(2 * BM, n_inst);
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * g.BN);
@@ -226,8 +224,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_pair_kernel(const __gri
       const float* sc_row = p.bn_scale ? p.bn_scale + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       const float* sh_row = p.bn_scale ? p.bn_shift + (int64_t)t.slice * p.bn_ld + t.n0 : nullptr;
       const __nv_bfloat16* res_row = (kRes && valid) ? p.residual + out_row * p.ldy + t.n0 : nullptr;
-      int ncols = t.ko - t.n0;
-      ncols = ncols > g.BN ? g.BN : ncols;
+      const int ncols = t.ncols;
       const long long base_row = __shfl_sync(0xffffffffu, (long long)out_row, 0);
       const bool contig = __all_sync(0xffffffffu, valid && out_row == base_row + lane) && t.ko >= 8;
 

@@ -68,7 +68,7 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 
 struct PairTile {
-  int map, ki, ko, n0, slice;
+  int map, ki, ko, n0, ncols, slice;   // the tile's columns: n0 .. n0 + ncols - 1 of the slice
   int p_end;
   int row0, rows_end;
   int b0, x0, y0;
@@ -79,6 +79,7 @@ struct PairTile {
 struct PairCursor {
   int lo = 0, hi = 0;   // tiles [lo, hi) belong to the cached group (hi = 0: nothing cached)
   int slice, map, ki, ko, p0, p_end, ntn;
+  int nq, nr;           // n-tile widths in units of 64 columns: the first nr n-tiles hold nq + 1 units, the others nq
 };
 
 // Tile `tile` of the pair schedule as seen by CTA `rank`: the pair owns m-tiles 2*mtp and 2*mtp+1 of
@@ -99,6 +100,12 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const 
     c.p0 = s_prefix[p.G + 1 + grp];         // group offsets, cached in shared memory
     c.p_end = s_prefix[p.G + 2 + grp];
     c.ntn = (c.ko + g.BN - 1) / g.BN;
+    // The slice's columns are dealt out evenly over its n-tiles in units of 64, the epilogue's store width (256 + 64
+    // columns would otherwise end in a tile whose tensor instructions run at the 59-cycle floor and that loads
+    // its activations all the same); only a slice's last tile can end inside a unit, where the store's map clips
+    const int units = (c.ko + 63) >> 6;
+    c.nq = units / c.ntn;
+    c.nr = units - c.nq * c.ntn;
   }
   t.slice = c.slice;
   t.map = c.map;
@@ -112,7 +119,9 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmParams& p, const 
     nt = local - mtp * c.ntn;
   }
   const int mt = 2 * mtp + rank;
-  t.n0 = nt * g.BN;
+  t.n0 = 64 * (nt * c.nq + (nt < c.nr ? nt : c.nr));
+  t.ncols = 64 * (c.nq + (nt < c.nr ? 1 : 0));
+  if (t.ncols > t.ko - t.n0) t.ncols = t.ko - t.n0;
   if (g.flat) {
     t.row0 = c.p0 * g.R + mt * BM;
     t.rows_end = c.p_end * g.R;
