@@ -198,7 +198,9 @@ typedef struct dsn_layer_desc {
  * (3x3 layers: one activation load per tap instead of one tile with its halo), DSN_HALO_SCHED=strided
  * (staged 3x3 kernel: tiles dealt out round-robin instead of one time-balanced range per CTA pair), DSN_ATTENTION=items (the
  * attention core with one (sample, head, query half) per CTA pass instead of the warp-specialised form),
- * DSN_DWPW=fused (depthwise + following 1x1 layer as one kernel), DSN_PDL=0 (no programmatic dependent launch).
+ * DSN_DWPW=fused (depthwise + following 1x1 layer as one kernel), DSN_CHAIN_FUSE=1 (chained launch: the last 1x1 layer
+ * takes the output of the layer before from tensor memory instead of global memory), DSN_PDL=0 (no programmatic
+ * dependent launch).
  * Every later call must be made with `device` as the calling thread's current CUDA device (else
  * DSN_ERR_INVALID_ARG): launches and kernel attributes act on the current device. */
 int dsn_create(dsn_ctx** ctx, int device);
@@ -243,6 +245,7 @@ typedef struct dsn_stats {
   uint64_t launches_route;
   uint64_t launches_copy;         /* gather / scatter, zero fill, channel scaling, Re-SBN folding          */
   uint64_t map_hits, map_misses;  /* tensor-map cache                                                      */
+  uint64_t launches_gemm_chain_tmem; /* of launches_gemm_chain: last layer fed from tensor memory          */
 } dsn_stats;
 int dsn_get_stats(dsn_ctx* ctx, dsn_stats* out);
 

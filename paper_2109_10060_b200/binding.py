@@ -82,7 +82,7 @@ class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("calls", "launches", "launches_gemm_pair", "launches_gemm_halo", "launches_gemm_chain",
                                           "launches_gemm_one_cta", "launches_linear_f32", "launches_attention",
                                           "launches_depthwise", "launches_dwpw", "launches_gate", "launches_route",
-                                          "launches_copy", "map_hits", "map_misses")]
+                                          "launches_copy", "map_hits", "map_misses", "launches_gemm_chain_tmem")]
 
 
 class LayerDesc(C.Structure):

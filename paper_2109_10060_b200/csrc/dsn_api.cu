@@ -428,6 +428,32 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
     cp.L[j].g.pair = 1;
     if (cp.L[j].g.BN > bn_max) bn_max = cp.L[j].g.BN;
   }
+  // The last layer can take its activations from tensor memory when it is a 1x1 / linear layer, the layer before
+  // produces a sample in ONE pair tile (so a tile of that layer is all the last layer needs of the sample) and at
+  // most 256 channels (128 tensor-memory columns of packed pairs beside two 128-column accumulators per region).
+  // The last layer then walks the tiles of the layer before (same pixel rectangles, same rows) with 128-wide n-tiles.
+  cp.fuse_tail = 0;
+  if (ctx->chain_fuse) {
+    const LayerCall& last = calls[n - 1];
+    const GemmGeom& gp = cp.L[n - 2].g;
+    bool ok = last.K == 1 && gp.tiles_x * gp.tiles_y <= 2 && gp.nb == 1 && !gp.flat;
+    for (int t = 0; ok && t < last.T; ++t) ok = calls[n - 2].k_out[t] <= 256 && last.k_in[t] <= calls[n - 2].k_out[t];
+    if (ok) {
+      GemmGeom& gl = cp.L[n - 1].g;
+      const int y_order = gl.y_input_order;
+      int max_ko = 1;
+      for (int t = 0; t < last.T; ++t) max_ko = last.k_out[t] > max_ko ? last.k_out[t] : max_ko;
+      gl = gp;
+      gl.taps = 1;
+      gl.KW = 1;
+      gl.pad = 0;
+      gl.a_input_order = 0;
+      gl.y_input_order = y_order;
+      gl.BN = max_ko > 64 ? 128 : 64;
+      cp.fuse_tail = 1;
+      bn_max = 256;  // two regions of 256 columns: rows of a sample below, an accumulator of the last layer above
+    }
+  }
   const int clusters = pair_clusters_for(ctx, bn_max);
   if (clusters <= 0 || r->B > 2 * clusters) return 0;
   int stages = bn_max == 256 ? 6 : 8;
@@ -445,6 +471,7 @@ int try_run_chain(dsn_ctx* ctx, const LayerCall* calls, int n, const dsn_routing
   cp.stages = stages;
   cp.bn_max = bn_max;
   count_launch(ctx, &dsn_stats::launches_gemm_chain);
+  if (cp.fuse_tail) ++ctx->stats.launches_gemm_chain_tmem;
   if (dsn_launch_gemm_bf16_chain(cp, clusters, dsn_gemm_chain_smem_bytes(bn_max, stages, r->G), s) != cudaSuccess)
     return DSN_ERR_CUDA;
   return 1;
@@ -741,6 +768,10 @@ int dsn_create(dsn_ctx** out, int device) {
     c->dwpw_fused = (dp && strcmp(dp, "fused") == 0) ? 1 : 0;
     const char* ch = getenv("DSN_CHAIN");  // "0": one launch per layer even for small batches (for comparisons)
     c->chain_mode = (ch && ch[0] == '0') ? 0 : 1;
+    // "1": in a chained launch the last 1x1 layer reads the layer before from tensor memory (measured slower on the
+    // bottleneck block: the last layer then runs on 128-wide n-tiles; off by default)
+    const char* cf = getenv("DSN_CHAIN_FUSE");
+    c->chain_fuse = (cf && cf[0] == '1') ? 1 : 0;
   }
   cudaDriverEntryPointQueryResult q;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||

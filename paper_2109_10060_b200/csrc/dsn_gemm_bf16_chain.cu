@@ -19,6 +19,15 @@
 // BOTH CTAs bump (release, cluster scope) once the stores of a tile of a non-final layer are
 // complete; the producers read it (acquire) before the first load of the sample's next layer.
 // All waits are bounded.
+//
+// Last layer fed from tensor memory (kFuse forms).  When the last layer is a 1x1 / linear layer whose input is the
+// whole output tile of the layer before (one pair tile per sample, at most 256 channels), that output never leaves
+// the SM: the epilogue of the layer before converts its accumulator rows to bf16 (bias, affine, activation as
+// usual) and writes them, two values per 32-bit column, over the first columns of the SAME accumulator region
+// (tcgen05.st; a thread only overwrites columns it has read), and the last layer's products take their A operand
+// from there (tcgen05.mma with A in tensor memory), so only its weights are loaded.  Its own accumulators are 128
+// columns wide and live in the upper halves of the two regions, which the epilogue of the layer before has read
+// by then.  ares[slot]: the 2 x 4 converting warps -> the issuing warp, the sample's rows are in place.
 #include "dsn_gemm_pair_device.cuh"
 
 namespace {
@@ -46,6 +55,40 @@ __device__ __forceinline__ uint32_t cta_addr_in_cluster(uint32_t local_addr, uin
 }
 // orders accesses to global memory through the generic proxy (plain loads / stores) and through the async proxy (TMA)
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
+// D[tmem] (+)= A[tmem] * B[smem]^T over the pair: every CTA supplies its 128 rows of A from its own tensor memory
+__device__ __forceinline__ void umma_bf16_pair_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// One warp converts its 32 accumulator rows of a whole tile (n_inst columns at `taddr`) and writes them back as
+// packed bf16 pairs over columns 0 .. n_inst / 2 - 1 of the same region: block c (32 columns) is read before the 16
+// columns at 16 c are written, which lie inside blocks this warp has already read.
+template <int ACT, bool AFF, bool RES>
+__device__ __forceinline__ void convert_tile_in_tmem(uint32_t taddr, int n_inst, int ko, const float* brow,
+                                                     const float* sc_row, const float* sh_row,
+                                                     const __nv_bfloat16* res_row) {
+  for (int c0 = 0; c0 < n_inst; c0 += 32) {
+    uint32_t w[16];
+    epilogue_half<ACT, AFF, RES>(taddr + c0, c0, ko, brow, sc_row, sh_row, res_row, w);
+    tmem_st_32x16(taddr + (c0 >> 1), w);
+  }
+  tmem_st_wait();
+}
 
 // Bounded wait until the counter reaches `target`.
 static __device__ __noinline__ bool wait_counter(uint32_t addr, uint32_t target, volatile uint32_t* abort_flag,
@@ -129,7 +172,7 @@ __device__ __forceinline__ void chain_walk(const DsnChainParams& cp, const int32
 // kAff: some layer of the block has a bias or a per-path affine; kGelu: some layer ends in GELU.  A form
 // without one of them holds none of that code: the kernel is sensitive to its own size (each of the two cuts
 // took about 1 us off the bottleneck step).
-template <bool kAff, bool kGelu, bool kRes = false>
+template <bool kAff, bool kGelu, bool kRes = false, bool kFuse = false>
 __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __grid_constant__ DsnChainParams cp) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -144,6 +187,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxStages + 36);
   uint32_t* done_cnt = reinterpret_cast<uint32_t*>(smem + 16 * kMaxStages + 40);  // [2]
   const uint32_t done_addr = base + 16 * kMaxStages + 40;
+  const uint32_t bar_ares = base + 16 * kMaxStages + 48;  // [2]
+  const int fuse_from = kFuse ? cp.n_layers - 2 : -2;     // the layer whose output stays in tensor memory
 
   const int stages = cp.stages;
   const uint32_t bh_bytes = (uint32_t)(cp.bn_max / 2) * BK * 2;  // this CTA's half of the widest weight tile
@@ -167,6 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
       mbar_init(bar_tempty + 8 * a, 2 * kEpiWarps);
+      mbar_init(bar_ares + 8 * a, 2 * 4);  // one converting warp per lane quarter in each CTA
     }
     *abort_flag = 0;
     done_cnt[0] = done_cnt[1] = 0;
@@ -196,18 +242,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
                [&](int l, int slot, const ChainTile& t, int, bool first_of_layer, int ntiles) {
       const GemmParams& P = cp.L[l];
       const GemmGeom& g = P.g;
+      const bool a_in_tmem = kFuse && l == fuse_from + 1;  // this layer's activations are not loaded
       if (first_of_layer) {
-        if (l > 0) {
+        if (l > 0 && !a_in_tmem) {
           // every tile of the layer before, of this sample, has been stored by both CTAs
           ok = __all_sync(0xffffffffu, wait_counter(done_addr + 4 * slot, target[slot], abort_flag, status, 31));
           if (!ok) return false;
           fence_proxy_async_all();  // the loads below read through the async proxy
         }
-        if (l + 1 < cp.n_layers) target[slot] += 2u * kEpiWarps * (uint32_t)ntiles;
+        if (l + 1 < cp.n_layers && l != fuse_from) target[slot] += 2u * kEpiWarps * (uint32_t)ntiles;
       }
       const CUtensorMap* mA = &P.mapA[t.map];
       const CUtensorMap* mB = &P.mapB[t.map];
-      const uint32_t a_box_bytes = (uint32_t)(g.bw * g.bh) * BK * 2;
+      const uint32_t a_box_bytes = a_in_tmem ? 0u : (uint32_t)(g.bw * g.bh) * BK * 2;
       const uint32_t tx_bytes = 2u * (a_box_bytes + (uint32_t)(g.BN / 2) * BK * 2);
       const int nkc = (t.ki + BK - 1) / BK;
       int ncols = t.ko - t.n0;
@@ -226,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
             const uint32_t full_lead = leader_addr(bar_full + 8 * stage);
             if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, tx_bytes);
             const uint32_t sa = tiles_base + stage * stage_bytes;
-            tma_load_4d_pair(sa, mA, kc * BK, cx, cy, bsel, full_lead);
+            if (!a_in_tmem) tma_load_4d_pair(sa, mA, kc * BK, cx, cy, bsel, full_lead);
             tma_load_3d_pair(sa + kABytes, mB, kc * BK, tap, brow0, full_lead);
           }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -243,18 +290,30 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       const uint64_t da0 = make_smem_desc(tiles_base), db0 = make_smem_desc(tiles_base + kABytes);
       const uint64_t dstep = (uint64_t)(stage_bytes >> 4);
       uint64_t da = da0, db = db0;
-      chain_walk(cp, s_off, pair, npairs, 0, [&](int l, int, const ChainTile& t, int it, bool, int) {
+      uint32_t ares_t0 = 0u, ares_t1 = 0u;   // where the rows of the sample of slot 0 / 1 sit in tensor memory
+      uint32_t ares_ph0 = 0u, ares_ph1 = 0u;
+      chain_walk(cp, s_off, pair, npairs, 0, [&](int l, int slot, const ChainTile& t, int it, bool first_of_layer, int) {
         const GemmGeom& g = cp.L[l].g;
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        const bool a_in_tmem = kFuse && l == fuse_from + 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, status, 33));
         if (!ok) return false;
+        if (kFuse && l == fuse_from) {
+          if (slot) ares_t1 = tmem_base + (uint32_t)(acc * cp.bn_max); else ares_t0 = tmem_base + (uint32_t)(acc * cp.bn_max);
+        }
+        if (a_in_tmem && first_of_layer) {  // the converted rows of the layer before are in place in both CTAs
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_ares + 8 * slot, slot ? ares_ph1 : ares_ph0, abort_flag, status, 36));
+          if (!ok) return false;
+          if (slot) ares_ph1 ^= 1u; else ares_ph0 ^= 1u;
+        }
         tc_fence_after();
         int ncols = t.ko - t.n0;
         ncols = ncols > g.BN ? g.BN : ncols;
         const int n_inst = (ncols + 31) & ~31;
         const uint32_t idesc = make_idesc(2 * BM, n_inst);
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * cp.bn_max);
+        // accumulators of a layer fed from tensor memory: the upper half of the region (the lower holds a sample's rows)
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * cp.bn_max) + (a_in_tmem ? (uint32_t)(cp.bn_max >> 1) : 0u);
         const int nkc = (t.ki + BK - 1) / BK;
         const int tail_ks = ((t.ki & (BK - 1)) + 15) >> 4;
         uint32_t accumulate = 0;
@@ -264,7 +323,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
             if (!ok) return false;
             tc_fence_after();
             const int nks = (kc == 1 && tail_ks != 0) ? tail_ks : BK / 16;
-            if (elect_one()) {
+            if (a_in_tmem) {
+              if (elect_one()) {
+                const uint32_t a0 = (slot ? ares_t1 : ares_t0) + (uint32_t)(32 * (nkc - kc));  // 64 bf16 = 32 columns per chunk
+                umma_bf16_pair_a_tmem(d_tmem, a0, db, idesc, accumulate);
+                if (nks > 1) umma_bf16_pair_a_tmem(d_tmem, a0 + 8u, db + 2u, idesc, 1u);
+                if (nks > 2) umma_bf16_pair_a_tmem(d_tmem, a0 + 16u, db + 4u, idesc, 1u);
+                if (nks > 3) umma_bf16_pair_a_tmem(d_tmem, a0 + 24u, db + 6u, idesc, 1u);
+                umma_commit_pair(bar_empty + 8 * stage);
+              }
+            } else if (elect_one()) {
               umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
               if (nks > 1) umma_bf16_pair(d_tmem, da + 2u, db + 2u, idesc, 1u);
               if (nks > 2) umma_bf16_pair(d_tmem, da + 4u, db + 4u, idesc, 1u);
@@ -339,10 +407,33 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, status, 35));
       if (!ok) return false;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * cp.bn_max);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * cp.bn_max) +
+                             ((kFuse && l == fuse_from + 1) ? (uint32_t)(cp.bn_max >> 1) : 0u);
       const CUtensorMap* mY = &P.mapY[t.map];
       int variant = any_valid ? P.act * 2 + ((brow || sc_row) ? 1 : 0) : -1;
       if (kRes && any_valid && P.residual) variant = 6 + P.act;
+      if (kFuse && l == fuse_from) {
+        // The rows stay on the SM as the next layer's A operand: the first warp of each lane quarter converts the whole
+        // tile in place (nothing is stored to global memory), then tells the issuing warp.
+        if (first == 0) {
+          const int n_inst = (ncols + 31) & ~31;
+          switch (variant) {
+            case 0: convert_tile_in_tmem<DSN_ACT_NONE, false, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 1: if constexpr (kAff) convert_tile_in_tmem<DSN_ACT_NONE, true, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 2: convert_tile_in_tmem<DSN_ACT_RELU, false, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 3: if constexpr (kAff) convert_tile_in_tmem<DSN_ACT_RELU, true, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 4: if constexpr (kGelu) convert_tile_in_tmem<DSN_ACT_GELU, false, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 5: if constexpr (kAff && kGelu) convert_tile_in_tmem<DSN_ACT_GELU, true, false>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 6: if constexpr (kRes) convert_tile_in_tmem<DSN_ACT_NONE, true, true>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 7: if constexpr (kRes) convert_tile_in_tmem<DSN_ACT_RELU, true, true>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            case 8: if constexpr (kRes && kGelu) convert_tile_in_tmem<DSN_ACT_GELU, true, true>(taddr, n_inst, ncols, brow, sc_row, sh_row, res_row); break;
+            default: break;  // none of this warp's rows belongs to the sample: its rows of the operand are never used
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_addr(bar_ares + 8 * slot));
+        }
+      } else
       switch (variant) {
         case -1: break;  // none of this warp's 32 rows belongs to the sample
         case 0: epilogue_tile<DSN_ACT_NONE, false>(taddr, ncols, t.n0, first, brow, sc_row, sh_row, res_row, stage_w, yrow, lane, contig, mY, (int)base_row); break;
@@ -359,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_bf16_chain_kernel(const __gr
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_addr(bar_tempty + 8 * acc));  // the accumulator is free again
-      if (l + 1 < cp.n_layers) pending_slot = slot;
+      if (l + 1 < cp.n_layers && l != fuse_from) pending_slot = slot;
       return true;
     });
     signal_pending();
@@ -385,19 +476,26 @@ size_t dsn_gemm_chain_smem_bytes(int bn_max, int stages, int G) {
 }
 
 cudaError_t dsn_launch_gemm_bf16_chain(const DsnChainParams& cp, int clusters, size_t smem_bytes, cudaStream_t s) {
-  static size_t configured[6][DSN_MAX_DEVICES] = {};
+  static size_t configured[12][DSN_MAX_DEVICES] = {};
   int aff = 0, gelu = 0, res = 0;
   for (int l = 0; l < cp.n_layers; ++l) {
     aff |= (cp.L[l].bias || cp.L[l].bn_scale) ? 1 : 0;
     gelu |= cp.L[l].act == DSN_ACT_GELU ? 1 : 0;
     res |= cp.L[l].residual ? 1 : 0;
   }
-  // a block with skip features (the residual tail of a DS-ResNet block, Sec. 5) takes the forms that carry that code
-  void (*kernel)(DsnChainParams) =
-      res ? (gelu ? gemm_bf16_chain_kernel<true, true, true> : gemm_bf16_chain_kernel<true, false, true>)
-          : aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
-                : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
-  const int form = res ? 4 + gelu : 2 * aff + gelu;
+  // a block with skip features (the residual tail of a DS-ResNet block, Sec. 5) takes the forms that carry that code;
+  // fuse_tail: the forms whose last layer reads its activations from tensor memory
+  void (*kernel)(DsnChainParams);
+  if (cp.fuse_tail) {
+    kernel = res ? (gelu ? gemm_bf16_chain_kernel<true, true, true, true> : gemm_bf16_chain_kernel<true, false, true, true>)
+             : aff ? (gelu ? gemm_bf16_chain_kernel<true, true, false, true> : gemm_bf16_chain_kernel<true, false, false, true>)
+                   : (gelu ? gemm_bf16_chain_kernel<false, true, false, true> : gemm_bf16_chain_kernel<false, false, false, true>);
+  } else {
+    kernel = res ? (gelu ? gemm_bf16_chain_kernel<true, true, true> : gemm_bf16_chain_kernel<true, false, true>)
+             : aff ? (gelu ? gemm_bf16_chain_kernel<true, true> : gemm_bf16_chain_kernel<true, false>)
+                   : (gelu ? gemm_bf16_chain_kernel<false, true> : gemm_bf16_chain_kernel<false, false>);
+  }
+  const int form = (res ? 4 + gelu : 2 * aff + gelu) + (cp.fuse_tail ? 6 : 0);
   {
     cudaError_t e = dsn_ensure_dynamic_smem(kernel, smem_bytes, configured[form]);
     if (e != cudaSuccess) return e;

@@ -41,6 +41,7 @@ struct dsn_ctx {
   int halo_sched;      // staged 3x3 tiles: 1 = dealt out round-robin (DSN_HALO_SCHED=strided), else one time-balanced range per pair
   int conv_halo;       // 1 = 3x3 layers stage the input tile once with its halo (default), 0 = one load per tap (DSN_CONV3X3=taps)
   int chain_mode;      // 1 = small-batch chains of sliced layers run as one launch (default), 0 = one launch per layer (DSN_CHAIN=0)
+  int chain_fuse;      // 1 = in a chained launch the last 1x1 layer reads the layer before from tensor memory (DSN_CHAIN_FUSE=1; default 0: measured slower)
   int dwpw_fused;      // 1 = depthwise + following 1x1 layer as one kernel (DSN_DWPW=fused); default 0: measured slower than the
                        //     two launches, because four producer warps on plain ALUs cannot keep up with the tensor core
   int pair_clusters[3];  // resident CTA pairs for BN = 64, 128, 256 (-1 = not queried yet)
@@ -196,6 +197,7 @@ struct DsnChainParams {
   int32_t n_layers;
   int32_t stages;   // depth of the operand ring
   int32_t bn_max;   // widest n-tile of the layers: accumulator stride in TMEM, weight half-box of a ring slot
+  int32_t fuse_tail;  // 1: the output of layer n_layers - 2 stays in tensor memory as the A operand of the last layer
 };
 
 // launchers implemented in the .cu files

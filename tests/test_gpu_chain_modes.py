@@ -129,6 +129,56 @@ def test_chained_bottleneck_edge_batches(dsn, B, routing):
     assert max(errs.values()) <= 1e-2, errs
 
 
+def _context_with(dsn, **switches):
+    """A context created while the given environment switches hold (they are read at creation only)."""
+    saved = {k: os.environ.get(k) for k in switches}
+    os.environ.update(switches)
+    try:
+        return dsn.Context(0)
+    finally:
+        for k, v in saved.items():
+            if v is None:
+                del os.environ[k]
+            else:
+                os.environ[k] = v
+
+
+@pytest.mark.parametrize("B,with_skip,C_outer,C_inner", [(37, False, 256, 64), (37, True, 256, 64), (148, False, 256, 64),
+                                                         (3, True, 256, 64), (21, False, 1024, 256)],
+                         ids=["plain", "skip-features", "two-per-pair", "tiny", "wide"])
+def test_bottleneck_last_layer_fed_from_tensor_memory(dsn, B, with_skip, C_outer, C_inner, parity_report):
+    """DSN_CHAIN_FUSE=1: in the chained launch the 3x3 layer's output tile is converted in place in tensor memory and the
+    last 1x1 layer takes it from there as its A operand (nothing of it is stored or loaded).  Same bottleneck, same
+    oracle chain and same bound as the default form; the launch counter shows that the form ran."""
+    ctx = _context_with(dsn, DSN_CHAIN="1", DSN_CHAIN_FUSE="1")
+    cfg = wl.bottleneck(79, B, 14, 14, C_outer, C_inner, routing="uniform", with_gate=False)
+    H, Wd, C, Ci, T, widths, idx = cfg["H"], cfg["W"], cfg["C_outer"], cfg["C_inner"], cfg["T"], cfg["widths"], cfg["idx"]
+    full = [C] * T
+    x = up_bf16(cfg["x"])
+    W2 = np.ascontiguousarray(np.transpose(cfg["W2"], (0, 2, 3, 1)))
+    layers = [dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, C, Ci, full, widths, up_bf16(cfg["W1"].reshape(Ci, C)), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 3, 1, Ci, Ci, widths, widths, up_bf16(W2), act=dsn.ACT_RELU),
+              dsn.make_conv_desc(dsn.BF16, H, Wd, 1, 0, Ci, C, widths, full, up_bf16(cfg["W3"].reshape(C, Ci)),
+                                 act=dsn.ACT_RELU if with_skip else dsn.ACT_NONE, residual=x if with_skip else None)]
+    L = dsn.make_layer_desc(B, T, layers, None)
+    ws = torch.empty(dsn.dsn_layer_workspace_bytes(L), dtype=torch.uint8, device=DEV)
+    y = torch.full((B, H, Wd, C), SENTINEL, dtype=torch.bfloat16, device=DEV)
+    before = ctx.stats()
+    dsn.dsn_layer_forward(ctx, L, x, up_i32(idx), y, ws)
+    code, detail = ctx.get_status()
+    assert code == 0, (code, detail)
+    after = ctx.stats()
+    assert after["launches_gemm_chain_tmem"] - before["launches_gemm_chain_tmem"] == 1
+    y1 = O.round_bf16(O.sliced_conv(cfg["x"], cfg["W1"], idx, full, widths, 0, act=O.ACT_RELU, fill=0.0))
+    y2 = O.round_bf16(O.sliced_conv(y1, cfg["W2"], idx, widths, widths, 1, act=O.ACT_RELU, fill=0.0))
+    ref = O.sliced_conv(y2, cfg["W3"], idx, widths, full, 0, act=O.ACT_RELU if with_skip else O.ACT_NONE,
+                        residual=cfg["x"] if with_skip else None)
+    errs = group_errors(down(y), ref, idx, full, T)
+    assert max(errs.values()) <= 1e-2, errs
+    parity_report.append(f"bottleneck, last layer fed from tensor memory, B={B}{' with skip features' if with_skip else ''}: "
+                         f"worst {max(errs.values()):.2e} (chain bound 1e-02)")
+
+
 @pytest.mark.parametrize("B,chained", [(37, True), (37, False), (160, True)], ids=["chained", "per-layer", "large-batch"])
 def test_bottleneck_with_identity_shortcut(dsn, B, chained, parity_report):
     """The residual tail of a DS-ResNet block (Sec. 5) inside dsn_layer_forward: out = ReLU(conv3(h) + x) with the block
