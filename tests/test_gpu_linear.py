@@ -137,6 +137,25 @@ def test_bf16_linear_ragged_widths_strided_and_zero_tail(dsn, ctx, R):
         assert np.all(got[i][:, Co:] == SENTINEL)                  # padding beyond C_out untouched
 
 
+@pytest.mark.parametrize("in_order,out_order", [(1, 1), (0, 0)])
+def test_bf16_linear_wide_slices_split_into_even_n_tiles(dsn, ctx, in_order, out_order):
+    """Slices wider than one 256-column tile are dealt out over their n-tiles in 64-column units (320 = 192 + 128,
+    576 = 3 x 192, 840 = 256 + 3 x 192 + a ragged end, 1344 = 6 x 224 rounded to units): every column of every tile
+    boundary must come out right, with bias and ReLU, and the columns beyond a slice stay untouched."""
+    g = np.random.default_rng(320)
+    B, R, Ci, Co, T = 23, 70, 96, 1344, 6
+    k_in, k_out = [96, 64, 96, 40, 96, 96], [320, 576, 840, 331, 1344, 264]
+    idx = g.integers(0, T, size=B).astype(np.int32)
+    x = wl.normal(g, (B, R, Ci))
+    W = wl.normal(g, (Co, Ci), std=Ci ** -0.5)
+    bias = g.standard_normal(Co).astype(np.float32) * 0.5
+    got = _run_bf16_linear(dsn, ctx, x, W, idx, k_in, k_out, R, in_order, out_order, bias=bias, act=dsn.ACT_RELU)
+    ref = O.round_bf16(O.sliced_linear(x, W, idx, k_in, k_out, bias=bias, act=O.ACT_RELU))
+    errs = group_errors(got, ref, idx, k_out, T)
+    assert max(errs.values()) <= TOL_BF16, errs
+    assert_tail_untouched(got, idx, k_out)
+
+
 def test_bf16_linear_vit_base_shape_sampled(dsn, ctx):
     """ViT-B width (768 -> 3072, 8 diagonal paths), Zipf routing; the oracle checks whole samples."""
     cfg = wl.config5(B=64, routing="zipf")
