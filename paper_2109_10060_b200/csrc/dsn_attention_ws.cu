@@ -265,6 +265,13 @@ __global__ void __launch_bounds__(kWsThreads, 1) attention_ws_kernel(const __gri
       bool store_pending = false;   // lane 0: a TMA store of the previous item may still be reading its staging tile
       for (int it = blockIdx.x; it < total; it += stride, ++n) {
         const uint32_t s = n & 1u;
+        // the previous item's store has read its staging tile by the time S of this item is ready (or shortly after): that
+        // stage goes back to the loader before the maximum pass, which then has all of this item to refill it
+        if (lane == 0 && store_pending) {
+          bulk_wait_read0();
+          mbar_arrive(bar_kv_empty + 8 * (s ^ 1u));
+          store_pending = false;
+        }
         if (!mbar_wait(bar_s_full + 8 * h, n & 1u, abort_flag, p.status, 36)) break;
         tc_fence_after();
         float sum = 0.f;
@@ -295,13 +302,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attention_ws_kernel(const __gri
               max_block(va, 32 * c);
               if (c + 1 < nb32) max_block(vb, 32 * (c + 1));
             }
-          }
-          // the previous item's store has read its staging tile by now (it was issued a whole maximum pass ago):
-          // that stage goes back to the loader, which then has the rest of this item to refill it
-          if (lane == 0 && store_pending) {
-            bulk_wait_read0();
-            mbar_arrive(bar_kv_empty + 8 * (s ^ 1u));
-            store_pending = false;
           }
           // pass 2: exp2(s * c - max * c); probabilities rounded to bf16 and written over columns of S this thread
           // has already read (P block c: 16 columns at 16 c).  Two keys per instruction where the hardware has a
