@@ -252,9 +252,10 @@ cudaError_t dsn_launch_depthwise(const int32_t* c, const int32_t* ksize, int T, 
   }
   p.H = H; p.W = W; p.K = K; p.stride = stride; p.C = C; p.T = T; p.G = G;
   p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
-  // about four (pixel, 8-channel) outputs per thread: each costs one round trip to memory, and many small CTAs fill
-  // the SMs more evenly than few long-running ones (measured on 14 x 14 x 640, 256 samples: 91 us with 3 bands)
-  int bands = (int)(((int64_t)p.Ho * p.Wo * ((C + 7) / 8)) / (4 * kThreads));
+  // about eight (pixel, 8-channel) outputs per thread: many small CTAs fill the SMs more evenly than few long-running
+  // ones, but every CTA pays its group lookup (measured on 14 x 14 x 640, 256 samples: 3 bands 61 us, 7 bands 55 us,
+  // 14 bands 58 us)
+  int bands = (int)(((int64_t)p.Ho * p.Wo * ((C + 7) / 8)) / (8 * kThreads));
   if (bands < 1) bands = 1;
   if (bands > p.Ho) bands = p.Ho;   // bands are whole output rows on the 3 x 3 fast path
   if (bands > 64) bands = 64;
